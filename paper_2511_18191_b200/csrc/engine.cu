@@ -1,0 +1,715 @@
+// Host side of the decoder library: handle, weight-blob layout, forward-pass assembly,
+// the speculative round loop (Algorithm 1 looped), target-only decoding (Eq. 1) and the
+// C ABI declared in include/tsfm.h.
+#include "../../include/tsfm.h"
+
+#include <cuda_runtime.h>
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "kernels_simt.cuh"
+#include "accept.cuh"
+#include "gemm_tc.cuh"
+
+using namespace tsfm;
+
+namespace {
+
+std::atomic<long long> g_launches{0};
+thread_local std::string g_cuda_err;
+
+#define CU_TRY(expr)                                                            \
+  do {                                                                          \
+    cudaError_t e_ = (expr);                                                    \
+    if (e_ != cudaSuccess) {                                                    \
+      g_cuda_err = std::string(#expr) + ": " + cudaGetErrorString(e_);          \
+      return TSFM_ERR_CUDA;                                                     \
+    }                                                                           \
+  } while (0)
+
+#define LAUNCHED() (g_launches.fetch_add(1, std::memory_order_relaxed))
+
+inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+inline size_t elt_bytes(int dtype) { return dtype == TSFM_BF16 ? 2 : 4; }
+
+bool arch_ok(const tsfm_arch &a, int P) {
+  if (a.n_layers < 1 || a.d_model < 64 || a.n_heads < 1 || a.d_ff < 64) return false;
+  if (a.d_model % a.n_heads) return false;
+  const int dh = a.d_model / a.n_heads;
+  if (dh != 32 && dh != 64 && dh != 128) return false;
+  if (a.d_model % 64 || a.d_ff % 64) return false;
+  if (P < 16 || P > 256 || P % 16) return false;
+  return true;
+}
+
+// Offsets of the tensors of one model inside its blob (canonical order, 256-byte aligned).
+struct BlobLayout {
+  size_t W_emb = 0, g_f = 0, W_head = 0, total = 0;
+  struct L { size_t g1, Wq, Wk, Wv, Wo, g2, W1, W2; };
+  std::vector<L> layers;
+};
+
+BlobLayout blob_layout(const tsfm_arch &a, int P, int dtype) {
+  BlobLayout b;
+  const size_t e = elt_bytes(dtype), d = a.d_model, f = a.d_ff;
+  size_t off = 256;
+  auto take = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return o; };
+  b.W_emb = take(d * P * e);
+  for (int l = 0; l < a.n_layers; ++l) {
+    BlobLayout::L x;
+    x.g1 = take(d * 4);
+    x.Wq = take(d * d * e);
+    x.Wk = take(d * d * e);
+    x.Wv = take(d * d * e);
+    x.Wo = take(d * d * e);
+    x.g2 = take(d * 4);
+    x.W1 = take(f * d * e);
+    x.W2 = take(d * f * e);
+    b.layers.push_back(x);
+  }
+  b.g_f = take(d * 4);
+  b.W_head = take((size_t)P * d * e);
+  b.total = off;
+  return b;
+}
+
+struct LayerDev {
+  const float *g1, *g2;
+  const void *Wqkv, *Wo, *W1, *W2;
+  GemmTcPlan tc_qkv, tc_o, tc_1, tc_2;
+};
+
+struct ModelDev {
+  tsfm_arch arch{};
+  int dh = 0;
+  const void *W_emb = nullptr, *W_head = nullptr;
+  const float *g_f = nullptr;
+  std::vector<LayerDev> layers;
+  void *Kc = nullptr, *Vc = nullptr;     // [L][B][heads][cap][dh]
+  size_t kv_layer_elems = 0;
+  float2 *rope = nullptr;                // [cap][dh/2] (cos, sin)
+};
+
+}  // namespace
+
+struct tsfm_spec {
+  tsfm_cfg cfg{};
+  cudaStream_t stream = nullptr;
+  int cap = 0;
+  bool use_tc = false;
+  ModelDev tgt, drf;
+  // activations (sized for M_max rows)
+  int M_max = 0;
+  float *x = nullptr, *qkv = nullptr;
+  void *a = nullptr, *ao = nullptr, *hbuf = nullptr;
+  // decoding state
+  float *hist = nullptr, *vout = nullptr, *mean = nullptr, *sd = nullptr;
+  int *done = nullptr;
+  AcceptCounters *ctr = nullptr;
+  int *unfinished = nullptr;             // [max_T + 1]
+  int *h_unfinished = nullptr;           // pinned
+  int *dev_status = nullptr;
+  int *tr_nacc = nullptr;                // [max_T][B]
+  float *tr_ell = nullptr, *tr_logu = nullptr;   // [max_T][B][K]
+  float *stage_in = nullptr, *stage_out = nullptr;   // device staging for the *_host entry points
+  int last_B = 0, last_K = 0, last_rounds = 0;
+  std::vector<cudaEvent_t> ev;
+  std::vector<void *> owned;
+};
+
+namespace {
+
+template <typename T>
+int dev_alloc(tsfm_spec *h, T **p, size_t count) {
+  void *q = nullptr;
+  CU_TRY(cudaMalloc(&q, count * sizeof(T) ? count * sizeof(T) : 256));
+  h->owned.push_back(q);
+  *p = (T *)q;
+  return TSFM_OK;
+}
+
+int read_header(const tsfm_weights *w, const tsfm_arch &a, int P, int dtype, cudaStream_t s) {
+  if (!w || !w->blob) return TSFM_ERR_ARG;
+  int32_t hd[8];
+  CU_TRY(cudaMemcpyAsync(hd, w->blob, sizeof(hd), cudaMemcpyDeviceToHost, s));
+  CU_TRY(cudaStreamSynchronize(s));
+  if (hd[0] != 0x4D465354 || hd[1] != 1 || hd[2] != dtype || hd[3] < a.n_layers ||
+      hd[4] != a.d_model || hd[5] != a.n_heads || hd[6] != a.d_ff || hd[7] != P)
+    return TSFM_ERR_SHAPE;
+  return TSFM_OK;
+}
+
+// Wire a model's tensor pointers.  `blob_arch` is the shape the blob was written for (a
+// layer-skip draft reads the first layers of the target's blob).
+void wire_model(ModelDev &m, const tsfm_arch &arch, const tsfm_arch &blob_arch, const void *blob,
+                int P, int dtype) {
+  const BlobLayout lay = blob_layout(blob_arch, P, dtype);
+  const char *base = (const char *)blob;
+  m.arch = arch;
+  m.dh = arch.d_model / arch.n_heads;
+  m.W_emb = base + lay.W_emb;
+  m.g_f = (const float *)(base + lay.g_f);
+  m.W_head = base + lay.W_head;
+  m.layers.clear();
+  for (int l = 0; l < arch.n_layers; ++l) {
+    LayerDev L{};
+    L.g1 = (const float *)(base + lay.layers[l].g1);
+    L.g2 = (const float *)(base + lay.layers[l].g2);
+    L.Wqkv = base + lay.layers[l].Wq;    // Wq, Wk, Wv are adjacent: one [3d, d] matrix
+    L.Wo = base + lay.layers[l].Wo;
+    L.W1 = base + lay.layers[l].W1;
+    L.W2 = base + lay.layers[l].W2;
+    m.layers.push_back(L);
+  }
+}
+
+int make_rope(tsfm_spec *h, ModelDev &m) {
+  const int half = m.dh / 2;
+  std::vector<float2> t((size_t)h->cap * half);
+  for (int p = 0; p < h->cap; ++p)
+    for (int i = 0; i < half; ++i) {
+      const double theta = std::pow((double)h->cfg.rope_base, -2.0 * i / m.dh);
+      t[(size_t)p * half + i] = make_float2((float)std::cos(p * theta), (float)std::sin(p * theta));
+    }
+  if (int rc = dev_alloc(h, &m.rope, t.size())) return rc;
+  CU_TRY(cudaMemcpyAsync(m.rope, t.data(), t.size() * sizeof(float2), cudaMemcpyHostToDevice, h->stream));
+  CU_TRY(cudaStreamSynchronize(h->stream));
+  return TSFM_OK;
+}
+
+template <typename T> size_t attn_smem_bytes(int dh, int nk) {
+  const int kp = dh + KPad<T>::v;
+  return (size_t)nk * (kp + dh) * sizeof(T) + (size_t)4 * nk * sizeof(float) + 4 * dh * sizeof(float);
+}
+
+template <typename T, int DH>
+int attn_set_attr(size_t bytes) {
+  CU_TRY(cudaFuncSetAttribute(attn_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+  return TSFM_OK;
+}
+template <typename T>
+int attn_prepare(int dh, int cap) {
+  const size_t bytes = attn_smem_bytes<T>(dh, cap);
+  if (bytes > 227 * 1024) return TSFM_ERR_SHAPE;
+  const size_t optin = 227 * 1024;        // opt in once to the per-CTA maximum; launches size themselves
+  if (dh == 32) return attn_set_attr<T, 32>(optin);
+  if (dh == 64) return attn_set_attr<T, 64>(optin);
+  return attn_set_attr<T, 128>(optin);
+}
+
+template <typename T>
+void launch_gemm_simt(cudaStream_t s, const T *A, const T *W, void *C, int M, int N, int K, int epi) {
+  dim3 grid((N + 63) / 64, (M + 63) / 64), block(256);
+  switch (epi) {
+    case EPI_F32: gemm_simt_kernel<T, EPI_F32><<<grid, block, 0, s>>>(A, W, C, M, N, K); break;
+    case EPI_T: gemm_simt_kernel<T, EPI_T><<<grid, block, 0, s>>>(A, W, C, M, N, K); break;
+    case EPI_GELU_T: gemm_simt_kernel<T, EPI_GELU_T><<<grid, block, 0, s>>>(A, W, C, M, N, K); break;
+    default: gemm_simt_kernel<T, EPI_RESID><<<grid, block, 0, s>>>(A, W, C, M, N, K); break;
+  }
+  LAUNCHED();
+}
+
+// C (op)= A . W^T through the tensor-core kernel when a plan exists, else the FMA kernel.
+template <typename T>
+void gemm(tsfm_spec *h, const GemmTcPlan *plan, const void *A, const void *W, void *C, int M, int N,
+          int K, int epi) {
+  if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
+    if (gemm_tc_launch(h->stream, *plan, A, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
+  }
+  launch_gemm_simt<T>(h->stream, (const T *)A, (const T *)W, C, M, N, K, epi);
+}
+
+template <typename T, int DH>
+void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
+  const int QT = g.q_len <= 16 ? g.q_len : 16;
+  dim3 grid(m.arch.n_heads, B, (g.q_len + QT - 1) / QT);
+  const size_t smem = attn_smem_bytes<T>(DH, h->cap);
+  T *Kc = (T *)m.Kc + (size_t)l * m.kv_layer_elems;
+  T *Vc = (T *)m.Vc + (size_t)l * m.kv_layer_elems;
+  attn_kernel<T, DH><<<grid, 128, smem, h->stream>>>(h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
+                                                     h->cap, (T *)h->ao);
+  LAUNCHED();
+}
+
+enum { HEAD_NONE = 0, HEAD_LAST_TO_HIST = 1, HEAD_ALL_TO_VOUT = 2 };
+
+// One causal pass of a model over q_len new tokens per series (appends to its KV cache).
+template <typename T>
+void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout) {
+  const int M = B * g.q_len, d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len;
+  cudaStream_t s = h->stream;
+  const float eps = h->cfg.rms_eps;
+  embed_kernel<T><<<M, 128, P * sizeof(float), s>>>(h->hist, g, P, d, (const T *)m.W_emb, h->x);
+  LAUNCHED();
+  const int L = m.arch.n_layers;
+  for (int l = 0; l < L; ++l) {
+    LayerDev &ly = m.layers[l];
+    rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g1, d, eps, (T *)h->a);
+    LAUNCHED();
+    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32);
+    if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
+    else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
+    else launch_attn<T, 128>(h, m, l, B, g);
+    if (l == L - 1 && head_mode == HEAD_NONE) break;   // prefill: only the cache is needed
+    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID);
+    rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g2, d, eps, (T *)h->a);
+    LAUNCHED();
+    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T);
+    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID);
+  }
+  if (head_mode == HEAD_LAST_TO_HIST) {
+    head_kernel<T><<<B, 128, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 1,
+                                                     h->hist, nullptr);
+    LAUNCHED();
+  } else if (head_mode == HEAD_ALL_TO_VOUT) {
+    head_kernel<T><<<M, 128, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 0,
+                                                     nullptr, vout);
+    LAUNCHED();
+  }
+}
+
+void pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout = nullptr) {
+  if (g.q_len < 1) return;
+  if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout);
+  else run_pass<float>(h, m, B, g, head_mode, vout);
+}
+
+int check_call(tsfm_spec *h, const float *series, int B, int ctx_len, int H, float *out, int K) {
+  if (!h || !series || !out) return TSFM_ERR_ARG;
+  if (B < 1 || H < 1 || ctx_len < 1) return TSFM_ERR_ARG;
+  const int P = h->cfg.patch_len;
+  if (ctx_len % P) return TSFM_ERR_SHAPE;
+  const int N = ctx_len / P, T = (H + P - 1) / P;
+  if (N < 2) return TSFM_ERR_SHAPE;
+  if (B > h->cfg.max_batch || N > h->cfg.max_ctx_tokens || T > h->cfg.max_horizon_patches ||
+      K > h->cfg.max_K)
+    return TSFM_ERR_SHAPE;
+  return TSFM_OK;
+}
+
+int begin_forecast(tsfm_spec *h, const float *series, int B, int ctx_len) {
+  const int P = h->cfg.patch_len;
+  instnorm_kernel<<<B, 256, 0, h->stream>>>(series, ctx_len, P, h->cap, h->cfg.norm_eps, h->hist,
+                                            h->mean, h->sd, h->done);
+  LAUNCHED();
+  CU_TRY(cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream));
+  return TSFM_OK;
+}
+
+int finish_call(tsfm_spec *h) {
+  CU_TRY(cudaGetLastError());
+  return TSFM_OK;
+}
+
+int read_status(tsfm_spec *h, int *status) {
+  CU_TRY(cudaMemcpyAsync(status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(cudaStreamSynchronize(h->stream));
+  return TSFM_OK;
+}
+
+}  // namespace
+
+// ====================================================================================
+// C ABI
+// ====================================================================================
+extern "C" {
+
+size_t tsfm_weights_bytes(const tsfm_arch *arch, int32_t patch_len, int32_t dtype) {
+  if (!arch || !arch_ok(*arch, patch_len) || (dtype != TSFM_F32 && dtype != TSFM_BF16)) return 0;
+  return blob_layout(*arch, patch_len, dtype).total;
+}
+
+size_t tsfm_weights_offset(const tsfm_arch *arch, int32_t patch_len, int32_t dtype, int32_t layer,
+                           const char *name) {
+  if (!arch || !name || !arch_ok(*arch, patch_len) || (dtype != TSFM_F32 && dtype != TSFM_BF16)) return 0;
+  const BlobLayout b = blob_layout(*arch, patch_len, dtype);
+  const std::string n(name);
+  if (n == "W_emb") return b.W_emb;
+  if (n == "g_f") return b.g_f;
+  if (n == "W_head") return b.W_head;
+  if (layer < 0 || layer >= arch->n_layers) return 0;
+  const BlobLayout::L &l = b.layers[layer];
+  if (n == "g1") return l.g1;
+  if (n == "Wq") return l.Wq;
+  if (n == "Wk") return l.Wk;
+  if (n == "Wv") return l.Wv;
+  if (n == "Wo") return l.Wo;
+  if (n == "g2") return l.g2;
+  if (n == "W1") return l.W1;
+  if (n == "W2") return l.W2;
+  return 0;
+}
+
+int tsfm_spec_destroy(tsfm_spec *h) {
+  if (!h) return TSFM_ERR_ARG;
+  cudaStreamSynchronize(h->stream);
+  for (void *p : h->owned) cudaFree(p);
+  if (h->h_unfinished) cudaFreeHost(h->h_unfinished);
+  for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
+  delete h;
+  return TSFM_OK;
+}
+
+int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, const tsfm_cfg *cfg,
+                     tsfm_spec **out_h) {
+  if (!target_w || !cfg || !out_h) return TSFM_ERR_ARG;
+  *out_h = nullptr;
+  const int P = cfg->patch_len;
+  if (cfg->dtype != TSFM_F32 && cfg->dtype != TSFM_BF16) return TSFM_ERR_ARG;
+  if (cfg->draft_mode != TSFM_DRAFT_SEPARATE && cfg->draft_mode != TSFM_DRAFT_LAYER_SKIP) return TSFM_ERR_ARG;
+  if (cfg->max_batch < 1 || cfg->max_ctx_tokens < 2 || cfg->max_horizon_patches < 1 || cfg->max_K < 1 ||
+      cfg->max_K > TSFM_MAX_K)
+    return TSFM_ERR_ARG;
+  if (!(cfg->rms_eps > 0.f) || !(cfg->norm_eps > 0.f) || !(cfg->rope_base > 1.f)) return TSFM_ERR_ARG;
+  if (!arch_ok(cfg->target, P) || !arch_ok(cfg->draft, P)) return TSFM_ERR_SHAPE;
+  if (cfg->draft_mode == TSFM_DRAFT_LAYER_SKIP) {
+    if (draft_w && draft_w->blob) return TSFM_ERR_ARG;
+    if (cfg->draft.d_model != cfg->target.d_model || cfg->draft.n_heads != cfg->target.n_heads ||
+        cfg->draft.d_ff != cfg->target.d_ff || cfg->draft.n_layers > cfg->target.n_layers)
+      return TSFM_ERR_SHAPE;
+  } else if (!draft_w || !draft_w->blob) {
+    return TSFM_ERR_ARG;
+  }
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CU_TRY(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return TSFM_ERR_ARCH;
+
+  tsfm_spec *h = new (std::nothrow) tsfm_spec();
+  if (!h) return TSFM_ERR_INTERNAL;
+  h->cfg = *cfg;
+  h->stream = (cudaStream_t)cfg->stream;
+  h->cap = cfg->max_ctx_tokens + cfg->max_horizon_patches + cfg->max_K + 1;
+  h->use_tc = cfg->dtype == TSFM_BF16 && cfg->gemm_backend == TSFM_GEMM_AUTO;
+  int rc = TSFM_OK;
+  auto fail = [&](int code) { tsfm_spec_destroy(h); return code; };
+
+  if (target_w->bytes < blob_layout(cfg->target, P, cfg->dtype).total) return fail(TSFM_ERR_SHAPE);
+  if ((rc = read_header(target_w, cfg->target, P, cfg->dtype, h->stream))) return fail(rc);
+  wire_model(h->tgt, cfg->target, cfg->target, target_w->blob, P, cfg->dtype);
+  if (cfg->draft_mode == TSFM_DRAFT_LAYER_SKIP) {
+    wire_model(h->drf, cfg->draft, cfg->target, target_w->blob, P, cfg->dtype);
+  } else {
+    if (draft_w->bytes < blob_layout(cfg->draft, P, cfg->dtype).total) return fail(TSFM_ERR_SHAPE);
+    if ((rc = read_header(draft_w, cfg->draft, P, cfg->dtype, h->stream))) return fail(rc);
+    wire_model(h->drf, cfg->draft, cfg->draft, draft_w->blob, P, cfg->dtype);
+  }
+
+  const size_t e = elt_bytes(cfg->dtype);
+  const int Bm = cfg->max_batch;
+  for (ModelDev *m : {&h->tgt, &h->drf}) {
+    m->kv_layer_elems = (size_t)Bm * m->arch.d_model * h->cap;
+    const size_t bytes = m->kv_layer_elems * m->arch.n_layers * e;
+    if ((rc = dev_alloc(h, (char **)&m->Kc, bytes))) return fail(rc);
+    if ((rc = dev_alloc(h, (char **)&m->Vc, bytes))) return fail(rc);
+    if ((rc = make_rope(h, *m))) return fail(rc);
+    rc = cfg->dtype == TSFM_BF16 ? attn_prepare<bf16>(m->dh, h->cap) : attn_prepare<float>(m->dh, h->cap);
+    if (rc) return fail(rc);
+  }
+  h->M_max = Bm * std::max(std::max(cfg->max_ctx_tokens, cfg->max_K + 1), 2);
+  const int dmax = std::max(cfg->target.d_model, cfg->draft.d_model);
+  const int fmax = std::max(cfg->target.d_ff, cfg->draft.d_ff);
+  const size_t Mx = h->M_max;
+  if ((rc = dev_alloc(h, &h->x, Mx * dmax))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->qkv, Mx * 3 * dmax))) return fail(rc);
+  if ((rc = dev_alloc(h, (char **)&h->a, Mx * dmax * e))) return fail(rc);
+  if ((rc = dev_alloc(h, (char **)&h->ao, Mx * dmax * e))) return fail(rc);
+  if ((rc = dev_alloc(h, (char **)&h->hbuf, Mx * fmax * e))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->hist, (size_t)Bm * h->cap * P))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->vout, (size_t)Bm * (cfg->max_K + 1) * P))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->mean, Bm))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->sd, Bm))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->done, Bm))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->ctr, 1))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->unfinished, cfg->max_horizon_patches + 1))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->dev_status, 1))) return fail(rc);
+  const size_t tr = (size_t)cfg->max_horizon_patches * Bm;
+  if ((rc = dev_alloc(h, &h->tr_nacc, tr))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->tr_ell, tr * cfg->max_K))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->tr_logu, tr * cfg->max_K))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->stage_in, (size_t)Bm * cfg->max_ctx_tokens * P))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->stage_out, (size_t)Bm * cfg->max_horizon_patches * P))) return fail(rc);
+  if (cudaMallocHost((void **)&h->h_unfinished, sizeof(int)) != cudaSuccess) return fail(TSFM_ERR_CUDA);
+  h->ev.resize(2 + 4 * (size_t)cfg->max_horizon_patches + 4);
+  for (auto &ev : h->ev)
+    if (cudaEventCreate(&ev) != cudaSuccess) { ev = nullptr; return fail(TSFM_ERR_CUDA); }
+  if (cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream) != cudaSuccess) return fail(TSFM_ERR_CUDA);
+
+  if (h->use_tc) {
+    if ((rc = gemm_tc_init())) return fail(rc);
+    for (ModelDev *m : {&h->tgt, &h->drf}) {
+      const int d = m->arch.d_model, f = m->arch.d_ff;
+      for (LayerDev &ly : m->layers) {
+        if ((rc = gemm_tc_plan(&ly.tc_qkv, ly.Wqkv, 3 * d, d, h->a, h->M_max))) return fail(rc);
+        if ((rc = gemm_tc_plan(&ly.tc_o, ly.Wo, d, d, h->ao, h->M_max))) return fail(rc);
+        if ((rc = gemm_tc_plan(&ly.tc_1, ly.W1, f, d, h->a, h->M_max))) return fail(rc);
+        if ((rc = gemm_tc_plan(&ly.tc_2, ly.W2, d, f, h->hbuf, h->M_max))) return fail(rc);
+      }
+    }
+  }
+  if (cudaStreamSynchronize(h->stream) != cudaSuccess) return fail(TSFM_ERR_CUDA);
+  *out_h = h;
+  return TSFM_OK;
+}
+
+int tsfm_target_only_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H,
+                              float *out, tsfm_stats *stats) {
+  if (int rc = check_call(h, series, B, ctx_len, H, out, 1)) return rc;
+  const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
+  cudaStream_t s = h->stream;
+  if (stats) CU_TRY(cudaEventRecord(h->ev[0], s));
+  if (int rc = begin_forecast(h, series, B, ctx_len)) return rc;
+  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
+  if (stats) CU_TRY(cudaEventRecord(h->ev[2], s));
+  for (int t = 0; t < T; ++t)       // Eq. 1: one target pass per committed patch
+    pass(h, h->tgt, B, PassGeom{nullptr, N - 1 + t, 1, h->cap}, HEAD_LAST_TO_HIST);
+  denorm_kernel<<<B, 256, 0, s>>>(h->hist, N, P, h->cap, H, h->mean, h->sd, out);
+  LAUNCHED();
+  if (int rc = finish_call(h)) return rc;
+  if (stats) {
+    CU_TRY(cudaEventRecord(h->ev[1], s));
+    std::memset(stats, 0, sizeof(*stats));
+    if (int rc = read_status(h, &stats->device_status)) return rc;
+    CU_TRY(cudaEventElapsedTime(&stats->ms_total, h->ev[0], h->ev[1]));
+    CU_TRY(cudaEventElapsedTime(&stats->ms_prefill, h->ev[0], h->ev[2]));
+    CU_TRY(cudaEventElapsedTime(&stats->ms_verify, h->ev[2], h->ev[1]));
+    stats->rounds = T;
+    stats->patches_committed = (int64_t)B * T;
+    if (stats->device_status) return TSFM_ERR_TIMEOUT;
+  }
+  return TSFM_OK;
+}
+
+int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H, int32_t K,
+                       float tau, uint64_t seed, float *out, tsfm_stats *stats) {
+  if (K < 1) return TSFM_ERR_ARG;
+  if (!(tau > 0.f) || !std::isfinite(tau)) return TSFM_ERR_ARG;
+  if (int rc = check_call(h, series, B, ctx_len, H, out, K)) return rc;
+  const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
+  cudaStream_t s = h->stream;
+  const bool timed = stats != nullptr;
+  if (timed) CU_TRY(cudaEventRecord(h->ev[0], s));
+  if (int rc = begin_forecast(h, series, B, ctx_len)) return rc;
+  CU_TRY(cudaMemsetAsync(h->ctr, 0, sizeof(AcceptCounters), s));
+  CU_TRY(cudaMemsetAsync(h->unfinished, 0, sizeof(int) * (T + 1), s));
+  CU_TRY(cudaMemsetAsync(h->tr_nacc, 0xff, sizeof(int) * (size_t)T * B, s));
+  CU_TRY(cudaMemsetAsync(h->tr_ell, 0, sizeof(float) * (size_t)T * B * K, s));
+  CU_TRY(cudaMemsetAsync(h->tr_logu, 0, sizeof(float) * (size_t)T * B * K, s));
+  // both caches ingest the context except its last patch (target) / last two (draft)
+  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
+  pass(h, h->drf, B, PassGeom{nullptr, 0, N - 2, h->cap}, HEAD_NONE);
+  if (timed) CU_TRY(cudaEventRecord(h->ev[2], s));
+
+  AcceptArgs a{};
+  a.x = a.mu_q = h->hist + (size_t)N * P;       // slot N + done[b] holds x_1
+  a.x_stride_b = (long long)h->cap * P;
+  a.mu_p = h->vout;
+  a.commit = h->hist + (size_t)N * P;
+  a.commit_stride_b = a.x_stride_b;
+  a.commit_accepted = 0;
+  a.commit_follows_done = 1;
+  a.done = h->done;
+  a.B = B; a.K = K; a.P = P; a.T = T;
+  a.sigma_p = a.sigma_q = tau;
+  a.margin = h->cfg.dtype == TSFM_BF16 ? 5e-2f : 1e-3f;
+  a.key = make_uint2((uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32));
+  a.series0 = 0;
+  a.forced_u = nullptr;
+  a.ctr = h->ctr;
+
+  int rounds = 0;
+  for (int r = 0; r < T; ++r) {
+    size_t e0 = 3 + 4 * (size_t)r;
+    // draft rollout: step 1 re-ingests the last two committed patches (the draft cache may
+    // lack the last accepted proposal), steps 2..K ingest the previous proposal
+    pass(h, h->drf, B, PassGeom{h->done, N - 2, 2, h->cap}, HEAD_LAST_TO_HIST);
+    for (int i = 2; i <= K; ++i)
+      pass(h, h->drf, B, PassGeom{h->done, N - 1 + (i - 1), 1, h->cap}, HEAD_LAST_TO_HIST);
+    if (timed) CU_TRY(cudaEventRecord(h->ev[e0], s));
+    // single-pass verification over [pending, x_1..x_K]
+    pass(h, h->tgt, B, PassGeom{h->done, N - 1, K + 1, h->cap}, HEAD_ALL_TO_VOUT, h->vout);
+    if (timed) CU_TRY(cudaEventRecord(h->ev[e0 + 1], s));
+    a.round_idx = r;
+    a.n_accept = h->tr_nacc + (size_t)r * B;
+    a.ell = h->tr_ell + (size_t)r * B * K;
+    a.log_u = h->tr_logu + (size_t)r * B * K;
+    a.unfinished = h->unfinished + r;
+    accept_kernel<<<(B + 3) / 4, 128, 0, s>>>(a);
+    LAUNCHED();
+    if (timed) CU_TRY(cudaEventRecord(h->ev[e0 + 2], s));
+    ++rounds;
+    CU_TRY(cudaMemcpyAsync(h->h_unfinished, h->unfinished + r, sizeof(int), cudaMemcpyDeviceToHost, s));
+    CU_TRY(cudaStreamSynchronize(s));
+    if (*h->h_unfinished == 0) break;
+  }
+  denorm_kernel<<<B, 256, 0, s>>>(h->hist, N, P, h->cap, H, h->mean, h->sd, out);
+  LAUNCHED();
+  h->last_B = B; h->last_K = K; h->last_rounds = rounds;
+  if (int rc = finish_call(h)) return rc;
+  if (stats) {
+    CU_TRY(cudaEventRecord(h->ev[1], s));
+    std::memset(stats, 0, sizeof(*stats));
+    AcceptCounters c;
+    CU_TRY(cudaMemcpyAsync(&c, h->ctr, sizeof(c), cudaMemcpyDeviceToHost, s));
+    if (int rc = read_status(h, &stats->device_status)) return rc;
+    stats->rounds = rounds;
+    stats->proposals_drafted = (int64_t)c.drafted;
+    stats->proposals_tested = (int64_t)c.tested;
+    stats->proposals_accepted = (int64_t)c.accepted;
+    stats->patches_committed = (int64_t)c.committed;
+    stats->near_margin_decisions = (int64_t)c.near_margin;
+    for (int i = 0; i < TSFM_MAX_K; ++i) {
+      stats->tested_by_pos[i] = (int64_t)c.tested_by_pos[i];
+      stats->accepted_by_pos[i] = (int64_t)c.accepted_by_pos[i];
+    }
+    for (int i = 0; i < TSFM_MAX_K + 2; ++i) stats->L_hist[i] = (int64_t)c.L_hist[i];
+    CU_TRY(cudaEventElapsedTime(&stats->ms_total, h->ev[0], h->ev[1]));
+    CU_TRY(cudaEventElapsedTime(&stats->ms_prefill, h->ev[0], h->ev[2]));
+    float ms = 0.f;
+    for (int r = 0; r < rounds; ++r) {
+      size_t e0 = 3 + 4 * (size_t)r;
+      cudaEvent_t start = r == 0 ? h->ev[2] : h->ev[e0 - 4 + 2];
+      CU_TRY(cudaEventElapsedTime(&ms, start, h->ev[e0]));
+      stats->ms_draft += ms;
+      CU_TRY(cudaEventElapsedTime(&ms, h->ev[e0], h->ev[e0 + 1]));
+      stats->ms_verify += ms;
+      CU_TRY(cudaEventElapsedTime(&ms, h->ev[e0 + 1], h->ev[e0 + 2]));
+      stats->ms_accept += ms;
+    }
+    if (stats->device_status) return TSFM_ERR_TIMEOUT;
+  }
+  return TSFM_OK;
+}
+
+int tsfm_spec_forecast_host(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H,
+                            int32_t K, float tau, uint64_t seed, float *out, tsfm_stats *stats) {
+  if (K < 1) return TSFM_ERR_ARG;
+  if (int rc = check_call(h, series, B, ctx_len, H, out, K)) return rc;
+  CU_TRY(cudaMemcpyAsync(h->stage_in, series, sizeof(float) * (size_t)B * ctx_len, cudaMemcpyHostToDevice, h->stream));
+  if (int rc = tsfm_spec_forecast(h, h->stage_in, B, ctx_len, H, K, tau, seed, h->stage_out, stats)) return rc;
+  CU_TRY(cudaMemcpyAsync(out, h->stage_out, sizeof(float) * (size_t)B * H, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(cudaStreamSynchronize(h->stream));
+  return TSFM_OK;
+}
+
+int tsfm_target_only_forecast_host(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H,
+                                   float *out, tsfm_stats *stats) {
+  if (int rc = check_call(h, series, B, ctx_len, H, out, 1)) return rc;
+  CU_TRY(cudaMemcpyAsync(h->stage_in, series, sizeof(float) * (size_t)B * ctx_len, cudaMemcpyHostToDevice, h->stream));
+  if (int rc = tsfm_target_only_forecast(h, h->stage_in, B, ctx_len, H, h->stage_out, stats)) return rc;
+  CU_TRY(cudaMemcpyAsync(out, h->stage_out, sizeof(float) * (size_t)B * H, cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(cudaStreamSynchronize(h->stream));
+  return TSFM_OK;
+}
+
+int tsfm_spec_last_trace(tsfm_spec *h, int32_t cap_rounds, int32_t *rounds, int32_t *n_accept, float *ell,
+                         float *log_u) {
+  if (!h || !rounds) return TSFM_ERR_ARG;
+  *rounds = h->last_rounds;
+  if (cap_rounds < h->last_rounds) return TSFM_ERR_ARG;
+  const size_t nb = (size_t)h->last_rounds * h->last_B, nk = nb * h->last_K;
+  cudaStream_t s = h->stream;
+  if (n_accept && nb) CU_TRY(cudaMemcpyAsync(n_accept, h->tr_nacc, nb * sizeof(int), cudaMemcpyDeviceToHost, s));
+  if (ell && nk) CU_TRY(cudaMemcpyAsync(ell, h->tr_ell, nk * sizeof(float), cudaMemcpyDeviceToHost, s));
+  if (log_u && nk) CU_TRY(cudaMemcpyAsync(log_u, h->tr_logu, nk * sizeof(float), cudaMemcpyDeviceToHost, s));
+  CU_TRY(cudaStreamSynchronize(s));
+  return TSFM_OK;
+}
+
+int tsfm_accept_round(void *stream, const float *x, const float *mu_q, const float *mu_p, int32_t B,
+                      int32_t K, int32_t P, int32_t T, float sigma_p, float sigma_q, uint64_t seed,
+                      int32_t round_idx, int32_t series0, const float *forced_u, int32_t *done,
+                      float *commit, int32_t *n_accept, float *ell, float *log_u) {
+  if (!x || !mu_q || !mu_p || !done || !commit) return TSFM_ERR_ARG;
+  if (B < 1 || K < 1 || K > TSFM_MAX_K || P < 1 || T < 1) return TSFM_ERR_ARG;
+  if (!(sigma_p > 0.f) || !(sigma_q > 0.f) || !std::isfinite(sigma_p) || !std::isfinite(sigma_q))
+    return TSFM_ERR_ARG;
+  AcceptArgs a{};
+  a.x = x; a.mu_q = mu_q; a.x_stride_b = (long long)K * P;
+  a.mu_p = mu_p;
+  a.commit = commit; a.commit_stride_b = (long long)(K + 1) * P;
+  a.commit_accepted = 1; a.commit_follows_done = 0;
+  a.done = done;
+  a.B = B; a.K = K; a.P = P; a.T = T;
+  a.sigma_p = sigma_p; a.sigma_q = sigma_q; a.margin = 0.f;
+  a.key = make_uint2((uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32));
+  a.round_idx = round_idx; a.series0 = series0;
+  a.forced_u = forced_u;
+  a.n_accept = n_accept; a.ell = ell; a.log_u = log_u;
+  accept_kernel<<<(B + 3) / 4, 128, 0, (cudaStream_t)stream>>>(a);
+  LAUNCHED();
+  CU_TRY(cudaGetLastError());
+  return TSFM_OK;
+}
+
+int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t B, int32_t n, float *out) {
+  if (!h || !tokens || !out || (which != 0 && which != 1)) return TSFM_ERR_ARG;
+  if (B < 1 || n < 1) return TSFM_ERR_ARG;
+  if (B > h->cfg.max_batch || n > h->cfg.max_ctx_tokens || B * n > h->M_max) return TSFM_ERR_SHAPE;
+  const int P = h->cfg.patch_len;
+  CU_TRY(cudaMemcpy2DAsync(h->hist, (size_t)h->cap * P * sizeof(float), tokens, (size_t)n * P * sizeof(float),
+                           (size_t)n * P * sizeof(float), B, cudaMemcpyDeviceToDevice, h->stream));
+  CU_TRY(cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream));
+  pass(h, which == 0 ? h->tgt : h->drf, B, PassGeom{nullptr, 0, n, h->cap}, HEAD_ALL_TO_VOUT, out);
+  if (int rc = finish_call(h)) return rc;
+  int status = 0;
+  if (int rc = read_status(h, &status)) return rc;
+  return status ? TSFM_ERR_TIMEOUT : TSFM_OK;
+}
+
+int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t M, int32_t N, int32_t Kd,
+                   int32_t backend) {
+  if (!A || !W || !C) return TSFM_ERR_ARG;
+  if (M < 1 || N < 1 || Kd < 16 || Kd % 16) return TSFM_ERR_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (backend == TSFM_GEMM_SIMT) {
+    launch_gemm_simt<bf16>(s, (const bf16 *)A, (const bf16 *)W, C, M, N, Kd, EPI_F32);
+    CU_TRY(cudaGetLastError());
+    return TSFM_OK;
+  }
+  if (Kd % 64) return TSFM_ERR_SHAPE;
+  if (int rc = gemm_tc_init()) return rc;
+  GemmTcPlan plan;
+  if (int rc = gemm_tc_plan(&plan, W, N, Kd, A, M)) return rc;
+  if (!plan.valid) return TSFM_ERR_SHAPE;
+  int *status = nullptr;
+  CU_TRY(cudaMalloc((void **)&status, sizeof(int)));
+  CU_TRY(cudaMemsetAsync(status, 0, sizeof(int), s));
+  const bool ok = gemm_tc_launch(s, plan, A, C, M, EPI_F32, status);
+  if (ok) LAUNCHED();
+  int hs = 0;
+  cudaError_t e1 = cudaMemcpyAsync(&hs, status, sizeof(int), cudaMemcpyDeviceToHost, s);
+  cudaError_t e2 = cudaStreamSynchronize(s);
+  cudaFree(status);
+  CU_TRY(e1);
+  CU_TRY(e2);
+  CU_TRY(cudaGetLastError());
+  if (!ok) return TSFM_ERR_INTERNAL;
+  return hs ? TSFM_ERR_TIMEOUT : TSFM_OK;
+}
+
+int64_t tsfm_launch_count(void) { return g_launches.load(); }
+
+const char *tsfm_strerror(int code) {
+  switch (code) {
+    case TSFM_OK: return "ok";
+    case TSFM_ERR_ARG: return "invalid argument";
+    case TSFM_ERR_SHAPE: return "unsupported shape or capacity exceeded";
+    case TSFM_ERR_ARCH: return "device is not sm_100";
+    case TSFM_ERR_CUDA: return "CUDA call failed";
+    case TSFM_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case TSFM_ERR_INTERNAL: return "internal error";
+    default: return "unknown error code";
+  }
+}
+
+const char *tsfm_last_cuda_error(void) { return g_cuda_err.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,328 @@
+// Plain CUDA-core kernels of the forward pass: instance norm, patch embedding, RMSNorm,
+// FMA GEMM, RoPE causal attention over the contiguous KV cache, final norm + mean head,
+// de-normalisation.  Everything is templated on the storage type T (float | bf16) of
+// weights, MMA-operand activations and the KV cache; the residual stream, norms, softmax
+// and head output are always fp32.
+#pragma once
+#include "common.cuh"
+
+namespace tsfm {
+
+// Where the tokens of one pass sit.  Token j of series b is history slot
+// pos0(b) + j with pos0(b) = done[b] + base (done may be NULL = 0).  Activations are
+// stored row-major with row = b * q_len + j.
+struct PassGeom {
+  const int *done;   // [B] patches committed so far, or NULL
+  int base;          // pos0 = done[b] + base
+  int q_len;         // tokens per series in this pass
+  int cap;           // token capacity of history / KV cache per series
+};
+__device__ __forceinline__ int pos0_of(const PassGeom &g, int b) {
+  return (g.done ? g.done[b] : 0) + g.base;
+}
+
+// ----------------------------------------------------------------------------------
+// Instance statistics frozen on the context (Sec. 3.4) and history initialisation.
+// grid = B, block = 256.  hist[b, t, :] = (series - mean) / sd for the N context
+// patches; the remaining slots are zeroed.  Sums in fp64 (8 K values, one pass each).
+// ----------------------------------------------------------------------------------
+__global__ void instnorm_kernel(const float *__restrict__ series, int ctx_len, int P, int cap,
+                                float norm_eps, float *__restrict__ hist,
+                                float *__restrict__ mean_out, float *__restrict__ sd_out,
+                                int *__restrict__ done) {
+  __shared__ double red[32];
+  const int b = blockIdx.x;
+  const float *s = series + (size_t)b * ctx_len;
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < ctx_len; i += blockDim.x) acc += (double)s[i];
+  const double mean = block_sum_d(acc, red) / ctx_len;
+  acc = 0.0;
+  for (int i = threadIdx.x; i < ctx_len; i += blockDim.x) {
+    const double c = (double)s[i] - mean;
+    acc += c * c;
+  }
+  const double var = block_sum_d(acc, red) / ctx_len;
+  const double sd = sqrt(var + (double)norm_eps);
+  float *hb = hist + (size_t)b * cap * P;
+  for (int i = threadIdx.x; i < cap * P; i += blockDim.x)
+    hb[i] = (i < ctx_len) ? (float)(((double)s[i] - mean) / sd) : 0.f;
+  if (threadIdx.x == 0) {
+    mean_out[b] = (float)mean;
+    sd_out[b] = (float)sd;
+    done[b] = 0;
+  }
+}
+
+// out[b, s] = hist[b, N + s / P, s % P] * sd + mean, s < H.   grid = B.
+__global__ void denorm_kernel(const float *__restrict__ hist, int N, int P, int cap, int H,
+                              const float *__restrict__ mean, const float *__restrict__ sd,
+                              float *__restrict__ out) {
+  const int b = blockIdx.x;
+  const float m = mean[b], s = sd[b];
+  const float *hb = hist + ((size_t)b * cap + N) * P;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) out[(size_t)b * H + i] = hb[i] * s + m;
+}
+
+// ----------------------------------------------------------------------------------
+// Patch embedding x[row, :] = W_emb[d, P] . z, z = history token (fp32).  grid = M rows,
+// block = 128.  A warp takes output features f, f + 4, ...; lanes stride over P.
+// ----------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d,
+                             const T *__restrict__ W, float *__restrict__ x) {
+  extern __shared__ float zs[];
+  const int row = blockIdx.x, b = row / g.q_len, j = row % g.q_len;
+  const float *z = hist + ((size_t)b * g.cap + pos0_of(g, b) + j) * P;
+  for (int i = threadIdx.x; i < P; i += blockDim.x) zs[i] = z[i];
+  __syncthreads();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  for (int f = w; f < d; f += nw) {
+    const T *wr = W + (size_t)f * P;
+    float acc = 0.f;
+    for (int i = lane; i < P; i += 32) acc = fmaf(to_f32(wr[i]), zs[i], acc);
+    acc = warp_sum(acc);
+    if (lane == 0) x[(size_t)row * d + f] = acc;
+  }
+}
+
+// ----------------------------------------------------------------------------------
+// RMSNorm: a[row, :] = g * x / sqrt(mean(x^2) + eps), rounded to T.  grid = M, block 128.
+// ----------------------------------------------------------------------------------
+template <typename T>
+__global__ void rmsnorm_kernel(const float *__restrict__ x, const float *__restrict__ gain, int d,
+                               float eps, T *__restrict__ a) {
+  __shared__ float red[32];
+  const size_t row = blockIdx.x;
+  const float *xr = x + row * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = xr[i];
+    ss = fmaf(v, v, ss);
+  }
+  const float rstd = rsqrtf(block_sum(ss, red) / d + eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x) a[row * d + i] = from_f32<T>(gain[i] * xr[i] * rstd);
+}
+
+// ----------------------------------------------------------------------------------
+// FMA GEMM  C[M, N] (op)= A[M, K] . W[N, K]^T, fp32 accumulate.  64x64 tile, BK = 16,
+// 256 threads, 4x4 outputs per thread.  K must be a multiple of 16.
+// Epilogues: store fp32 | store T | GELU -> T | residual add into fp32.
+// ----------------------------------------------------------------------------------
+enum { EPI_F32 = 0, EPI_T = 1, EPI_GELU_T = 2, EPI_RESID = 3 };
+
+template <typename T, int EPI>
+__global__ void __launch_bounds__(256)
+gemm_simt_kernel(const T *__restrict__ A, const T *__restrict__ W, void *__restrict__ Cout,
+                 int M, int N, int K) {
+  __shared__ float As[16][64 + 4];
+  __shared__ float Ws[16][64 + 4];
+  const int tid = threadIdx.x;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const int lr = tid >> 2;          // 0..63: tile row loaded by this thread
+  const int lk = (tid & 3) * 4;     // 0,4,8,12: first of 4 k's loaded
+  const int tm = (tid >> 4) * 4;    // output rows tm..tm+3
+  const int tn = (tid & 15) * 4;    // output cols tn..tn+3
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < K; k0 += 16) {
+    float av[4], wv[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      av[i] = (m0 + lr < M) ? to_f32(A[(size_t)(m0 + lr) * K + k0 + lk + i]) : 0.f;
+      wv[i] = (n0 + lr < N) ? to_f32(W[(size_t)(n0 + lr) * K + k0 + lk + i]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      As[lk + i][lr] = av[i];
+      Ws[lk + i][lr] = wv[i];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      float a4[4], w4[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        a4[i] = As[kk][tm + i];
+        w4[i] = Ws[kk][tn + i];
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a4[i], w4[j], acc[i][j]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + tm + i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tn + j;
+      if (n >= N) continue;
+      const size_t o = (size_t)m * N + n;
+      if (EPI == EPI_F32) ((float *)Cout)[o] = acc[i][j];
+      else if (EPI == EPI_T) ((T *)Cout)[o] = from_f32<T>(acc[i][j]);
+      else if (EPI == EPI_GELU_T) ((T *)Cout)[o] = from_f32<T>(gelu_erf(acc[i][j]));
+      else ((float *)Cout)[o] += acc[i][j];
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------------
+// RoPE + KV append + causal attention for one (head, series, query tile).
+//   qkv   [M, 3 d] fp32: q | k | v of this pass's tokens (row = b * q_len + j)
+//   Kc,Vc [B, heads, cap, DH] T: this layer's cache; positions < pos0 are valid
+//   rope  [cap, DH/2] float2 (cos, sin), rotate-half pairing (i, i + DH/2)
+//   out   [M, d] T
+// The CTA loads keys 0..pos0-1 from the cache and keys of this pass (rotated here) up to
+// its last query into shared memory once; all queries of the tile share that read.  The
+// tile that owns a token writes its rotated key and its value to the cache.
+// grid = (heads, B, ceil(q_len / QT)), block = 128 (one query per warp at a time).
+// Dynamic smem: K tile [nk][DH + 2] T, V tile [nk][DH] T, scores [4][nk] f32, q [4][DH] f32.
+// ----------------------------------------------------------------------------------
+template <typename T> struct KPad { static constexpr int v = 2; };
+template <> struct KPad<float> { static constexpr int v = 1; };
+
+template <typename T, int DH>
+__global__ void __launch_bounds__(128)
+attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
+            const float2 *__restrict__ rope, PassGeom g, int n_heads, int QT, int nk_max,
+            T *__restrict__ out) {
+  constexpr int KP = DH + KPad<T>::v;
+  constexpr int HALF = DH / 2;
+  constexpr int DPL = DH / 32;                 // output dims per lane
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  T *Ks = reinterpret_cast<T *>(smem_raw);
+  T *Vs = Ks + (size_t)nk_max * KP;
+  float *sc = reinterpret_cast<float *>(Vs + (size_t)nk_max * DH);
+  float *qs = sc + 4 * nk_max;
+
+  const int h = blockIdx.x, b = blockIdx.y, qt = blockIdx.z;
+  const int d = n_heads * DH;
+  const int p0 = pos0_of(g, b);
+  const int j_lo = qt * QT;
+  const int j_hi = min(g.q_len, j_lo + QT);          // queries [j_lo, j_hi)
+  const size_t row0 = (size_t)b * g.q_len;
+  T *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
+  T *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
+
+  // cached keys/values
+  for (int i = threadIdx.x; i < p0 * DH; i += blockDim.x) {
+    const int t = i / DH, c = i % DH;
+    Ks[t * KP + c] = Kb[i];
+    Vs[t * DH + c] = Vb[i];
+  }
+  // keys/values of this pass (rotate keys; the owning tile appends to the cache)
+  for (int i = threadIdx.x; i < j_hi * HALF; i += blockDim.x) {
+    const int j = i / HALF, c = i % HALF;
+    const float *src = qkv + (row0 + j) * 3 * d + h * DH;
+    const float2 cs = rope[(size_t)(p0 + j) * HALF + c];
+    const float k1 = src[d + c], k2 = src[d + c + HALF];
+    const T r1 = from_f32<T>(k1 * cs.x - k2 * cs.y), r2 = from_f32<T>(k2 * cs.x + k1 * cs.y);
+    const T v1 = from_f32<T>(src[2 * d + c]), v2 = from_f32<T>(src[2 * d + c + HALF]);
+    const int t = p0 + j;
+    Ks[t * KP + c] = r1;
+    Ks[t * KP + c + HALF] = r2;
+    Vs[t * DH + c] = v1;
+    Vs[t * DH + c + HALF] = v2;
+    if (j >= j_lo) {
+      Kb[(size_t)t * DH + c] = r1;
+      Kb[(size_t)t * DH + c + HALF] = r2;
+      Vb[(size_t)t * DH + c] = v1;
+      Vb[(size_t)t * DH + c + HALF] = v2;
+    }
+  }
+  __syncthreads();
+
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const float scale = rsqrtf((float)DH);
+  float *my_sc = sc + (size_t)w * nk_max;
+  float *my_q = qs + w * DH;
+  for (int j = j_lo + w; j < j_hi; j += 4) {
+    const float *src = qkv + (row0 + j) * 3 * d + h * DH;
+    for (int c = lane; c < HALF; c += 32) {
+      const float2 cs = rope[(size_t)(p0 + j) * HALF + c];
+      const float q1 = src[c], q2 = src[c + HALF];
+      my_q[c] = (q1 * cs.x - q2 * cs.y) * scale;
+      my_q[c + HALF] = (q2 * cs.x + q1 * cs.y) * scale;
+    }
+    __syncwarp();
+    const int nv = p0 + j + 1;                       // causal: keys 0..p0+j
+    float mx = -INFINITY;
+    for (int t = lane; t < nv; t += 32) {
+      const T *kr = Ks + (size_t)t * KP;
+      float s = 0.f;
+#pragma unroll 8
+      for (int c = 0; c < DH; ++c) s = fmaf(my_q[c], to_f32(kr[c]), s);
+      my_sc[t] = s;
+      mx = fmaxf(mx, s);
+    }
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int t = lane; t < nv; t += 32) {
+      const float p = expf(my_sc[t] - mx);
+      my_sc[t] = p;
+      sum += p;
+    }
+    sum = warp_sum(sum);
+    __syncwarp();
+    float acc[DPL];
+#pragma unroll
+    for (int c = 0; c < DPL; ++c) acc[c] = 0.f;
+    for (int t = 0; t < nv; ++t) {
+      const float p = my_sc[t];
+#pragma unroll
+      for (int c = 0; c < DPL; ++c) acc[c] = fmaf(p, to_f32(Vs[(size_t)t * DH + lane * DPL + c]), acc[c]);
+    }
+    const float inv = 1.f / sum;
+#pragma unroll
+    for (int c = 0; c < DPL; ++c)
+      out[(row0 + j) * d + h * DH + lane * DPL + c] = from_f32<T>(acc[c] * inv);
+    __syncwarp();
+  }
+}
+
+// ----------------------------------------------------------------------------------
+// Final RMSNorm + mean head for selected tokens: o = W_head[P, d] . (g_f * x * rstd).
+// Normalised activations stay fp32 here.  grid = (rows), block = 128.
+// only_last = 1: one row per series, the pass's last token, written to the series' next
+//   history slot hist[b, pos0 + q_len, :]  (draft steps, target-only steps);
+// only_last = 0: every token, written to vout[b, j, :]  (verification; vout [B, q_len, P]).
+// ----------------------------------------------------------------------------------
+template <typename T>
+__global__ void head_kernel(const float *__restrict__ x, const float *__restrict__ gain,
+                            const T *__restrict__ Wh, int d, int P, float eps, PassGeom g,
+                            int only_last, float *__restrict__ hist, float *__restrict__ vout) {
+  extern __shared__ float xs[];
+  __shared__ float red[32];
+  int b, j;
+  if (only_last) { b = blockIdx.x; j = g.q_len - 1; }
+  else { b = blockIdx.x / g.q_len; j = blockIdx.x % g.q_len; }
+  const float *xr = x + ((size_t)b * g.q_len + j) * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = xr[i];
+    xs[i] = v;
+    ss = fmaf(v, v, ss);
+  }
+  const float rstd = rsqrtf(block_sum(ss, red) / d + eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x) xs[i] = gain[i] * xs[i] * rstd;
+  __syncthreads();
+  float *dst = only_last ? hist + ((size_t)b * g.cap + pos0_of(g, b) + g.q_len) * P
+                         : vout + ((size_t)b * g.q_len + j) * P;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  for (int p = w; p < P; p += nw) {
+    const T *wr = Wh + (size_t)p * d;
+    float acc = 0.f;
+    for (int i = lane; i < d; i += 32) acc = fmaf(to_f32(wr[i]), xs[i], acc);
+    acc = warp_sum(acc);
+    if (lane == 0) dst[p] = acc;
+  }
+}
+
+}  // namespace tsfm

@@ -1,0 +1,149 @@
+"""End-to-end parity of the CUDA decoder with the oracle on the five workloads (and small
+ragged variants), through the C ABI, plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import tests.parity as parity
+from tests.gpu_common import make_decoder, series_on_device
+from oracle import tsfm_oracle as orc
+from tsfm_inputs import Arch, WORKLOADS, workload
+
+pytestmark = pytest.mark.gpu
+
+
+def check_stats(st, B, T, K):
+    d = st.as_dict()
+    assert d["device_status"] == 0
+    assert d["patches_committed"] == B * T
+    assert 1 <= d["rounds"] <= T
+    assert d["proposals_accepted"] <= d["proposals_tested"] <= d["proposals_drafted"]
+    n_rounds = sum(d["L_hist"])
+    assert d["proposals_drafted"] == K * n_rounds
+    assert sum(d["L_hist"][K + 2:]) == 0 and d["L_hist"][0] == 0
+    assert sum(l * c for l, c in enumerate(d["L_hist"])) == n_rounds + d["proposals_accepted"]
+    tested, acc = np.array(d["tested_by_pos"][:K], float), np.array(d["accepted_by_pos"][:K], float)
+    assert tested[0] == n_rounds and np.all(tested[1:] == acc[:-1])
+    # the capped-geometric identity on the run's own counts: mean(L) = sum_l prod_{i<l} a_i
+    rate = np.divide(acc, tested, out=np.zeros(K), where=tested > 0)
+    mean_L = sum(l * c for l, c in enumerate(d["L_hist"])) / n_rounds
+    assert mean_L == pytest.approx(sum(np.prod(rate[:l]) for l in range(K + 1)), rel=1e-9)
+    return d
+
+
+def run_and_compare(wl, K, tau, seed, ids, backend=0, batch=None, H=None):
+    H = H or wl.horizon
+    B = batch or wl.batch
+    dec, tw, dw = make_decoder(wl, backend=backend, max_K=max(K, wl.K), batch=B)
+    s, ctx = series_on_device(wl, B)
+    out, st = dec.forecast(ctx, H, K, tau, seed)
+    T = -(-H // wl.patch_len)
+    d = check_stats(st, B, T, K)
+    nacc, ell, logu = dec.last_trace(B, K)
+    assert nacc.shape[0] == d["rounds"]
+    ref, st0 = dec.target_only(ctx, H)
+    got = out.cpu().numpy()
+    tgt_only = ref.cpu().numpy()
+    dec.close()
+    tm, dm = parity.oracle_models(wl, tw, dw)
+    res = parity.compare_forecast(wl, tm, dm, s, H, K, tau, seed, got, nacc, ids)
+    want_t = orc.forecast_target_only(tm, s[list(ids)], wl.ctx_len, H)
+    kind, tol = parity.VALUE_TOL[wl.dtype]
+    res["target_only_error"] = parity.value_error(kind, tgt_only[list(ids)], want_t)
+    assert res["target_only_error"] <= tol
+    res["stats"] = d
+    print(wl.name, K, tau, {k: v for k, v in res.items() if k != "stats"},
+          "acc", d["proposals_accepted"], "/", d["proposals_tested"], "rounds", d["rounds"])
+    return res
+
+
+def test_c0_full():
+    wl = workload("C0")
+    run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, range(wl.batch))
+
+
+@pytest.mark.parametrize("K,tau,H", [(1, 1.0, 384), (3, 2.0, 400), (4, 4.0, 96 * 7 + 5)])
+def test_c0_shape_ragged_batch_fp32(K, tau, H):
+    """C0's models on a ragged batch: several series, acceptance in the middle range, truncated last patch."""
+    wl = workload("C0", batch=6, series_recipe="c1", horizon=H)
+    run_and_compare(wl, K, tau, 7, range(6))
+
+
+@pytest.mark.parametrize("backend", [1, 0], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("tau", [0.5, 1.0, 2.0])
+def test_c1_full(tau, backend):
+    wl = workload("C1")
+    run_and_compare(wl, wl.K, tau, wl.forecast_seed, range(wl.batch), backend=backend)
+
+
+def test_c2_subset():
+    wl = workload("C2")
+    run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, [0, 1, 100, 255])
+
+
+@pytest.mark.parametrize("K,eps", [(1, 1e-2), (2, 1e-1), (4, 1e-2), (8, 1e-3), (4, 0.0)])
+def test_c3_sweep_subset(K, eps):
+    wl = workload("C3", draft_eps=eps)
+    res = run_and_compare(wl, K, wl.tau, wl.forecast_seed, [0, 513, 1023])
+    d = res["stats"]
+    if eps == 0.0:                       # draft == target: everything accepted, every round yields K+1
+        assert d["proposals_accepted"] == d["proposals_tested"]
+        assert d["rounds"] == -(-wl.n_patches // (K + 1))
+
+
+def test_c4_subset():
+    wl = workload("C4")
+    run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, [0, 63])
+
+
+def test_tiny_tau_recovers_target_only_and_result_is_independent_of_batch_composition():
+    wl = workload("C1")
+    dec, tw, dw = make_decoder(wl)
+    s, ctx = series_on_device(wl)
+    ref, _ = dec.target_only(ctx, wl.horizon)
+    out, st = dec.forecast(ctx, wl.horizon, wl.K, 1e-4, 5)
+    d = st.as_dict()
+    assert d["proposals_accepted"] == 0 and d["rounds"] == wl.n_patches
+    assert parity.value_error("rel_rms", out.cpu().numpy(), ref.cpu().numpy().astype(np.float64)) < 1e-2
+    # a series decoded alone (same series id 0) gives the same forecast as inside the batch
+    full, _ = dec.forecast(ctx, wl.horizon, wl.K, 1.0, 5)
+    solo, _ = dec.forecast(ctx[:1].contiguous(), wl.horizon, wl.K, 1.0, 5)
+    assert parity.value_error("rel_rms", solo.cpu().numpy(), full[:1].cpu().numpy().astype(np.float64)) < 1e-2
+    dec.close()
+
+
+def test_argument_errors_are_reported_not_fatal():
+    import paper_2511_18191_b200 as tsfm
+    wl = workload("C0")
+    dec, tw, dw = make_decoder(wl)
+    s, ctx = series_on_device(wl)
+    out = torch.empty((1, wl.horizon), device="cuda")
+    for kw, code in [(dict(K=0), tsfm.TSFM_ERR_ARG), (dict(K=3), tsfm.TSFM_ERR_SHAPE),
+                     (dict(tau=0.0), tsfm.TSFM_ERR_ARG), (dict(tau=float("nan")), tsfm.TSFM_ERR_ARG),
+                     (dict(H=0), tsfm.TSFM_ERR_ARG), (dict(H=96 * 5), tsfm.TSFM_ERR_SHAPE),
+                     (dict(ctx_len=100), tsfm.TSFM_ERR_SHAPE), (dict(ctx_len=96), tsfm.TSFM_ERR_SHAPE),
+                     (dict(B=2), tsfm.TSFM_ERR_SHAPE)]:
+        a = dict(B=1, ctx_len=wl.ctx_len, H=wl.horizon, K=2, tau=1.0)
+        a.update(kw)
+        with pytest.raises(tsfm.TsfmError) as e:
+            tsfm.tsfm_spec_forecast(dec.h, ctx, a["B"], a["ctx_len"], a["H"], a["K"], a["tau"], 1, out, None)
+        assert e.value.code == code, kw
+    # the handle still works afterwards
+    dec.forecast(ctx, wl.horizon, 2, 1.0, 1)
+    dec.close()
+
+
+def test_host_buffer_entry_points_match_device_ones():
+    import paper_2511_18191_b200 as tsfm
+    wl = workload("C1")
+    dec, tw, dw = make_decoder(wl)
+    s, ctx = series_on_device(wl)
+    out, _ = dec.forecast(ctx, wl.horizon, wl.K, 1.0, 3)
+    h_in = torch.from_numpy(np.ascontiguousarray(s[:, :wl.ctx_len])).pin_memory()
+    h_out = torch.empty((wl.batch, wl.horizon)).pin_memory()
+    tsfm.tsfm_spec_forecast_host(dec.h, h_in, wl.batch, wl.ctx_len, wl.horizon, wl.K, 1.0, 3, h_out, None)
+    np.testing.assert_array_equal(h_out.numpy(), out.cpu().numpy())
+    ref, _ = dec.target_only(ctx, wl.horizon)
+    tsfm.tsfm_target_only_forecast_host(dec.h, h_in, wl.batch, wl.ctx_len, wl.horizon, h_out, None)
+    np.testing.assert_array_equal(h_out.numpy(), ref.cpu().numpy())
+    dec.close()
