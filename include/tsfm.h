@@ -204,6 +204,23 @@ int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t
 int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C,
                    int32_t M, int32_t N, int32_t Kd, int32_t backend);
 
+/* Per-launch timing, for roofline accounting.  While enabled, every kernel launch of the handle
+ * is bracketed by two CUDA events on the handle's stream (this perturbs end-to-end time: do not
+ * quote throughput from a profiled call).  tsfm_spec_set_profiling clears the records.
+ * tsfm_spec_kernel_profile synchronises and aggregates them per kernel: launches, total device
+ * milliseconds, and the algorithmic bytes and flops of those launches (what the operation must
+ * move / compute: operands read once, results written once).  out: host array of `cap` entries;
+ * *n receives the number of kernels with at least one launch. */
+typedef struct {
+  char    name[24];
+  int64_t launches;
+  double  ms_total;
+  double  bytes;
+  double  flops;
+} tsfm_kernel_stat;
+int tsfm_spec_set_profiling(tsfm_spec *h, int32_t enable);
+int tsfm_spec_kernel_profile(tsfm_spec *h, int32_t cap, int32_t *n, tsfm_kernel_stat *out);
+
 int tsfm_spec_destroy(tsfm_spec *h);
 
 /* Number of kernels this library has launched in this process (all handles, all streams). */

@@ -25,7 +25,7 @@ EXPORTS = [
     "tsfm_weights_bytes", "tsfm_weights_offset", "tsfm_spec_create", "tsfm_spec_forecast",
     "tsfm_target_only_forecast", "tsfm_spec_forecast_host", "tsfm_target_only_forecast_host",
     "tsfm_spec_last_trace", "tsfm_accept_round", "tsfm_model_forward", "tsfm_gemm_bf16",
-    "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
+    "tsfm_spec_set_profiling", "tsfm_spec_kernel_profile", "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
 ]
 
 
@@ -64,6 +64,11 @@ class tsfm_stats(C.Structure):
         return d
 
 
+class tsfm_kernel_stat(C.Structure):
+    _fields_ = [("name", C.c_char * 24), ("launches", C.c_int64), ("ms_total", C.c_double),
+                ("bytes", C.c_double), ("flops", C.c_double)]
+
+
 def _load() -> C.CDLL:
     path = _build.LIB
     if not os.path.exists(path):
@@ -93,6 +98,10 @@ def _load() -> C.CDLL:
     lib.tsfm_model_forward.argtypes = [vp, i32, vp, i32, i32, vp]
     lib.tsfm_gemm_bf16.restype = C.c_int
     lib.tsfm_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
+    lib.tsfm_spec_set_profiling.restype = C.c_int
+    lib.tsfm_spec_set_profiling.argtypes = [vp, i32]
+    lib.tsfm_spec_kernel_profile.restype = C.c_int
+    lib.tsfm_spec_kernel_profile.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(tsfm_kernel_stat)]
     lib.tsfm_spec_destroy.restype = C.c_int
     lib.tsfm_spec_destroy.argtypes = [vp]
     lib.tsfm_launch_count.restype = C.c_int64
@@ -236,6 +245,19 @@ def tsfm_model_forward(h, which: int, tokens, B: int, n: int, out) -> None:
 
 def tsfm_gemm_bf16(stream, A, W, Cout, M: int, N: int, Kd: int, backend: int) -> None:
     _check(lib.tsfm_gemm_bf16(stream, _ptr(A), _ptr(W), _ptr(Cout), M, N, Kd, backend), "tsfm_gemm_bf16")
+
+
+def tsfm_spec_set_profiling(h, enable: bool) -> None:
+    _check(lib.tsfm_spec_set_profiling(h, int(bool(enable))), "tsfm_spec_set_profiling")
+
+
+def tsfm_spec_kernel_profile(h):
+    """Per-kernel {name: dict(launches, ms_total, bytes, flops)} of the launches since profiling was enabled."""
+    arr = (tsfm_kernel_stat * 32)()
+    n = C.c_int32(0)
+    _check(lib.tsfm_spec_kernel_profile(h, 32, C.byref(n), arr), "tsfm_spec_kernel_profile")
+    return {arr[i].name.decode(): dict(launches=arr[i].launches, ms_total=arr[i].ms_total, bytes=arr[i].bytes,
+                                       flops=arr[i].flops) for i in range(n.value)}
 
 
 def tsfm_launch_count() -> int:

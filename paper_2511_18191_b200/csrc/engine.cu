@@ -119,11 +119,50 @@ struct tsfm_spec {
   float *tr_ell = nullptr, *tr_logu = nullptr;   // [max_T][B][K]
   float *stage_in = nullptr, *stage_out = nullptr;   // device staging for the *_host entry points
   int last_B = 0, last_K = 0, last_rounds = 0;
+  // optional per-launch timing (tsfm_spec_set_profiling)
+  bool profiling = false;
+  struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
+  std::vector<ProfRec> prof;
+  std::vector<cudaEvent_t> prof_pool;
+  size_t prof_pool_used = 0;
   std::vector<cudaEvent_t> ev;
   std::vector<void *> owned;
 };
 
 namespace {
+
+// Kernel classes for per-launch timing.
+enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_TC, KC_GEMM_SIMT, KC_ATTN, KC_HEAD, KC_ACCEPT, KC_DENORM,
+       KC_COUNT };
+const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_tc", "gemm_simt", "attn",
+                                            "head", "accept", "denorm"};
+
+// Brackets one launch with two events when profiling is on (no-op otherwise).
+struct KTimer {
+  tsfm_spec *h;
+  size_t idx = 0;
+  bool on = false;
+  KTimer(tsfm_spec *h_, int cls, double bytes, double flops) : h(h_) {
+    if (!h->profiling || cls < 0) return;
+    auto get = [&]() -> cudaEvent_t {
+      if (h->prof_pool_used == h->prof_pool.size()) {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+        h->prof_pool.push_back(e);
+      }
+      return h->prof_pool[h->prof_pool_used++];
+    };
+    tsfm_spec::ProfRec r{cls, get(), get(), bytes, flops};
+    if (!r.e0 || !r.e1) return;
+    cudaEventRecord(r.e0, h->stream);
+    h->prof.push_back(r);
+    idx = h->prof.size() - 1;
+    on = true;
+  }
+  ~KTimer() {
+    if (on) cudaEventRecord(h->prof[idx].e1, h->stream);
+  }
+};
 
 template <typename T>
 int dev_alloc(tsfm_spec *h, T **p, size_t count) {
@@ -219,9 +258,15 @@ void launch_gemm_simt(cudaStream_t s, const T *A, const T *W, void *C, int M, in
 template <typename T>
 void gemm(tsfm_spec *h, const GemmTcPlan *plan, const void *A, const void *W, void *C, int M, int N,
           int K, int epi) {
+  const double e = sizeof(T);
+  const double out_b = epi == EPI_F32 ? 4.0 : epi == EPI_RESID ? 8.0 : e;
+  const double bytes = ((double)N * K + (double)M * K) * e + (double)M * N * out_b;
+  const double flops = 2.0 * M * N * K;
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
+    KTimer kt(h, KC_GEMM_TC, bytes, flops);
     if (gemm_tc_launch(h->stream, *plan, A, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
   }
+  KTimer kt(h, KC_GEMM_SIMT, bytes, flops);
   launch_gemm_simt<T>(h->stream, (const T *)A, (const T *)W, C, M, N, K, epi);
 }
 
@@ -232,6 +277,11 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   const size_t smem = attn_smem_bytes<T>(DH, h->cap);
   T *Kc = (T *)m.Kc + (size_t)l * m.kv_layer_elems;
   T *Vc = (T *)m.Vc + (size_t)l * m.kv_layer_elems;
+  // algorithmic bytes: q/k/v of the pass + the cached keys and values (lower bound: done = 0)
+  const double kv = (double)B * std::max(g.base, 0) * 2.0 * m.arch.d_model * sizeof(T);
+  const double Mr = (double)B * g.q_len;
+  KTimer kt(h, KC_ATTN, Mr * 3 * m.arch.d_model * 4 + kv + Mr * m.arch.d_model * (2.0 * sizeof(T) + sizeof(T)),
+            4.0 * Mr * (std::max(g.base, 0) + 0.5 * g.q_len) * m.arch.d_model);
   attn_kernel<T, DH><<<grid, 128, smem, h->stream>>>(h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
                                                      h->cap, (T *)h->ao);
   LAUNCHED();
@@ -245,24 +295,37 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   const int M = B * g.q_len, d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len;
   cudaStream_t s = h->stream;
   const float eps = h->cfg.rms_eps;
-  embed_kernel<T><<<M, 128, P * sizeof(float), s>>>(h->hist, g, P, d, (const T *)m.W_emb, h->x);
-  LAUNCHED();
+  {
+    KTimer kt(h, KC_EMBED, (double)M * P * 4 + (double)d * P * sizeof(T) + (double)M * d * 4, 2.0 * M * P * d);
+    embed_kernel<T><<<M, 128, P * sizeof(float), s>>>(h->hist, g, P, d, (const T *)m.W_emb, h->x);
+    LAUNCHED();
+  }
+  const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
   const int L = m.arch.n_layers;
   for (int l = 0; l < L; ++l) {
     LayerDev &ly = m.layers[l];
-    rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g1, d, eps, (T *)h->a);
-    LAUNCHED();
+    {
+      KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
+      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g1, d, eps, (T *)h->a);
+      LAUNCHED();
+    }
     gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
     else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
     else launch_attn<T, 128>(h, m, l, B, g);
     if (l == L - 1 && head_mode == HEAD_NONE) break;   // prefill: only the cache is needed
     gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID);
-    rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g2, d, eps, (T *)h->a);
-    LAUNCHED();
+    {
+      KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
+      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g2, d, eps, (T *)h->a);
+      LAUNCHED();
+    }
     gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T);
     gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID);
   }
+  const double rows = head_mode == HEAD_LAST_TO_HIST ? B : M;
+  KTimer kt(h, head_mode == HEAD_NONE ? -1 : KC_HEAD, rows * d * 4 + (double)P * d * sizeof(T) + rows * P * 4,
+            2.0 * rows * P * d);
   if (head_mode == HEAD_LAST_TO_HIST) {
     head_kernel<T><<<B, 128, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 1,
                                                      h->hist, nullptr);
@@ -295,9 +358,12 @@ int check_call(tsfm_spec *h, const float *series, int B, int ctx_len, int H, flo
 
 int begin_forecast(tsfm_spec *h, const float *series, int B, int ctx_len) {
   const int P = h->cfg.patch_len;
-  instnorm_kernel<<<B, 256, 0, h->stream>>>(series, ctx_len, P, h->cap, h->cfg.norm_eps, h->hist,
-                                            h->mean, h->sd, h->done);
-  LAUNCHED();
+  {
+    KTimer kt(h, KC_INSTNORM, (double)B * (ctx_len + (double)h->cap * P) * 4, 4.0 * B * ctx_len);
+    instnorm_kernel<<<B, 256, 0, h->stream>>>(series, ctx_len, P, h->cap, h->cfg.norm_eps, h->hist,
+                                              h->mean, h->sd, h->done);
+    LAUNCHED();
+  }
   CU_TRY(cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream));
   return TSFM_OK;
 }
@@ -349,6 +415,7 @@ size_t tsfm_weights_offset(const tsfm_arch *arch, int32_t patch_len, int32_t dty
 int tsfm_spec_destroy(tsfm_spec *h) {
   if (!h) return TSFM_ERR_ARG;
   cudaStreamSynchronize(h->stream);
+  for (cudaEvent_t e : h->prof_pool) cudaEventDestroy(e);
   for (void *p : h->owned) cudaFree(p);
   if (h->h_unfinished) cudaFreeHost(h->h_unfinished);
   for (cudaEvent_t e : h->ev) cudaEventDestroy(e);
@@ -470,8 +537,11 @@ int tsfm_target_only_forecast(tsfm_spec *h, const float *series, int32_t B, int3
   if (stats) CU_TRY(cudaEventRecord(h->ev[2], s));
   for (int t = 0; t < T; ++t)       // Eq. 1: one target pass per committed patch
     pass(h, h->tgt, B, PassGeom{nullptr, N - 1 + t, 1, h->cap}, HEAD_LAST_TO_HIST);
-  denorm_kernel<<<B, 256, 0, s>>>(h->hist, N, P, h->cap, H, h->mean, h->sd, out);
-  LAUNCHED();
+  {
+    KTimer kt(h, KC_DENORM, 8.0 * B * H, 2.0 * B * H);
+    denorm_kernel<<<B, 256, 0, s>>>(h->hist, N, P, h->cap, H, h->mean, h->sd, out);
+    LAUNCHED();
+  }
   if (int rc = finish_call(h)) return rc;
   if (stats) {
     CU_TRY(cudaEventRecord(h->ev[1], s));
@@ -541,16 +611,22 @@ int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx
     a.ell = h->tr_ell + (size_t)r * B * K;
     a.log_u = h->tr_logu + (size_t)r * B * K;
     a.unfinished = h->unfinished + r;
-    accept_kernel<<<(B + 3) / 4, 128, 0, s>>>(a);
-    LAUNCHED();
+    {
+      KTimer kt(h, KC_ACCEPT, (double)B * (2 * K + 2) * P * 4, 4.0 * B * K * P);
+      accept_kernel<<<(B + 3) / 4, 128, 0, s>>>(a);
+      LAUNCHED();
+    }
     if (timed) CU_TRY(cudaEventRecord(h->ev[e0 + 2], s));
     ++rounds;
     CU_TRY(cudaMemcpyAsync(h->h_unfinished, h->unfinished + r, sizeof(int), cudaMemcpyDeviceToHost, s));
     CU_TRY(cudaStreamSynchronize(s));
     if (*h->h_unfinished == 0) break;
   }
-  denorm_kernel<<<B, 256, 0, s>>>(h->hist, N, P, h->cap, H, h->mean, h->sd, out);
-  LAUNCHED();
+  {
+    KTimer kt(h, KC_DENORM, 8.0 * B * H, 2.0 * B * H);
+    denorm_kernel<<<B, 256, 0, s>>>(h->hist, N, P, h->cap, H, h->mean, h->sd, out);
+    LAUNCHED();
+  }
   h->last_B = B; h->last_K = K; h->last_rounds = rounds;
   if (int rc = finish_call(h)) return rc;
   if (stats) {
@@ -693,6 +769,39 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t
   CU_TRY(cudaGetLastError());
   if (!ok) return TSFM_ERR_INTERNAL;
   return hs ? TSFM_ERR_TIMEOUT : TSFM_OK;
+}
+
+int tsfm_spec_set_profiling(tsfm_spec *h, int32_t enable) {
+  if (!h) return TSFM_ERR_ARG;
+  CU_TRY(cudaStreamSynchronize(h->stream));
+  h->profiling = enable != 0;
+  h->prof.clear();
+  h->prof_pool_used = 0;
+  return TSFM_OK;
+}
+
+int tsfm_spec_kernel_profile(tsfm_spec *h, int32_t cap, int32_t *n, tsfm_kernel_stat *out) {
+  if (!h || !n || (cap > 0 && !out)) return TSFM_ERR_ARG;
+  CU_TRY(cudaStreamSynchronize(h->stream));
+  tsfm_kernel_stat acc[KC_COUNT];
+  std::memset(acc, 0, sizeof(acc));
+  for (int c = 0; c < KC_COUNT; ++c) std::snprintf(acc[c].name, sizeof(acc[c].name), "%s", kKernelNames[c]);
+  for (const tsfm_spec::ProfRec &r : h->prof) {
+    float ms = 0.f;
+    CU_TRY(cudaEventElapsedTime(&ms, r.e0, r.e1));
+    acc[r.cls].launches += 1;
+    acc[r.cls].ms_total += ms;
+    acc[r.cls].bytes += r.bytes;
+    acc[r.cls].flops += r.flops;
+  }
+  int k = 0;
+  for (int c = 0; c < KC_COUNT; ++c)
+    if (acc[c].launches) {
+      if (k < cap) out[k] = acc[c];
+      ++k;
+    }
+  *n = k;
+  return k <= cap ? TSFM_OK : TSFM_ERR_ARG;
 }
 
 int64_t tsfm_launch_count(void) { return g_launches.load(); }
