@@ -223,8 +223,8 @@ int make_rope(tsfm_spec *h, ModelDev &m) {
 }
 
 template <typename T> size_t attn_smem_bytes(int dh, int nk) {
-  const int kp = dh + KPad<T>::v;
-  return (size_t)nk * (kp + dh) * sizeof(T) + (size_t)4 * nk * sizeof(float) + 4 * dh * sizeof(float);
+  const int vw = AttnWords<T>::per_row(dh);
+  return (size_t)nk * (2 * vw + 1) * 4 + (size_t)4 * nk * sizeof(float) + 4 * dh * sizeof(float);
 }
 
 template <typename T, int DH>
@@ -234,7 +234,7 @@ int attn_set_attr(size_t bytes) {
 }
 template <typename T>
 int attn_prepare(int dh, int cap) {
-  const size_t bytes = attn_smem_bytes<T>(dh, cap);
+  const size_t bytes = attn_smem_bytes<T>(dh, (cap + 3) & ~3);
   if (bytes > 227 * 1024) return TSFM_ERR_SHAPE;
   const size_t optin = 227 * 1024;        // opt in once to the per-CTA maximum; launches size themselves
   if (dh == 32) return attn_set_attr<T, 32>(optin);
@@ -259,7 +259,7 @@ template <typename T>
 void gemm(tsfm_spec *h, const GemmTcPlan *plan, const void *A, const void *W, void *C, int M, int N,
           int K, int epi) {
   const double e = sizeof(T);
-  const double out_b = epi == EPI_F32 ? 4.0 : epi == EPI_RESID ? 8.0 : e;
+  const double out_b = (epi == EPI_F32 || epi == EPI_ATOMIC) ? 4.0 : epi == EPI_RESID ? 8.0 : e;
   const double bytes = ((double)N * K + (double)M * K) * e + (double)M * N * out_b;
   const double flops = 2.0 * M * N * K;
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
@@ -274,7 +274,8 @@ template <typename T, int DH>
 void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   const int QT = g.q_len <= 16 ? g.q_len : 16;
   dim3 grid(m.arch.n_heads, B, (g.q_len + QT - 1) / QT);
-  const size_t smem = attn_smem_bytes<T>(DH, h->cap);
+  const int nk_max = (h->cap + 3) & ~3;        // keeps every shared-memory region 16-byte aligned
+  const size_t smem = attn_smem_bytes<T>(DH, nk_max);
   T *Kc = (T *)m.Kc + (size_t)l * m.kv_layer_elems;
   T *Vc = (T *)m.Vc + (size_t)l * m.kv_layer_elems;
   // algorithmic bytes: q/k/v of the pass + the cached keys and values (lower bound: done = 0)
@@ -283,7 +284,7 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   KTimer kt(h, KC_ATTN, Mr * 3 * m.arch.d_model * 4 + kv + Mr * m.arch.d_model * (2.0 * sizeof(T) + sizeof(T)),
             4.0 * Mr * (std::max(g.base, 0) + 0.5 * g.q_len) * m.arch.d_model);
   attn_kernel<T, DH><<<grid, 128, smem, h->stream>>>(h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
-                                                     h->cap, (T *)h->ao);
+                                                     nk_max, (T *)h->ao);
   LAUNCHED();
 }
 
@@ -297,19 +298,23 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   const float eps = h->cfg.rms_eps;
   {
     KTimer kt(h, KC_EMBED, (double)M * P * 4 + (double)d * P * sizeof(T) + (double)M * d * 4, 2.0 * M * P * d);
-    embed_kernel<T><<<M, 128, P * sizeof(float), s>>>(h->hist, g, P, d, (const T *)m.W_emb, h->x);
+    embed_kernel<T><<<dim3(M, (d + 127) / 128), 128, P * sizeof(float), s>>>(h->hist, g, P, d, (const T *)m.W_emb, h->x);
     LAUNCHED();
   }
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
   const int L = m.arch.n_layers;
+  // The QKV contraction is split along K (atomic accumulation) when its grid would be small;
+  // the preceding RMSNorm kernel then clears the accumulator.
+  const bool qkv_split = sizeof(T) == 2 && h->use_tc && gemm_tc_splits(3 * d, d, M, true) > 1;
+  float *qkv_zero = qkv_split ? h->qkv : nullptr;
   for (int l = 0; l < L; ++l) {
     LayerDev &ly = m.layers[l];
     {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g1, d, eps, (T *)h->a);
+      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g1, d, eps, (T *)h->a, qkv_zero, 3 * d);
       LAUNCHED();
     }
-    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32);
+    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, qkv_split ? EPI_ATOMIC : EPI_F32);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
     else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
     else launch_attn<T, 128>(h, m, l, B, g);
@@ -317,7 +322,7 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID);
     {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g2, d, eps, (T *)h->a);
+      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g2, d, eps, (T *)h->a, nullptr, 0);
       LAUNCHED();
     }
     gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T);
@@ -327,11 +332,11 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   KTimer kt(h, head_mode == HEAD_NONE ? -1 : KC_HEAD, rows * d * 4 + (double)P * d * sizeof(T) + rows * P * 4,
             2.0 * rows * P * d);
   if (head_mode == HEAD_LAST_TO_HIST) {
-    head_kernel<T><<<B, 128, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 1,
+    head_kernel<T><<<dim3(B, (P + 7) / 8), 256, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 1,
                                                      h->hist, nullptr);
     LAUNCHED();
   } else if (head_mode == HEAD_ALL_TO_VOUT) {
-    head_kernel<T><<<M, 128, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 0,
+    head_kernel<T><<<dim3(M, (P + 7) / 8), 256, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 0,
                                                      nullptr, vout);
     LAUNCHED();
   }
@@ -750,7 +755,7 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t
     CU_TRY(cudaGetLastError());
     return TSFM_OK;
   }
-  if (Kd % 64) return TSFM_ERR_SHAPE;
+  if (Kd % 8) return TSFM_ERR_SHAPE;
   if (int rc = gemm_tc_init()) return rc;
   GemmTcPlan plan;
   if (int rc = gemm_tc_plan(&plan, W, N, Kd, A, M)) return rc;

@@ -118,7 +118,9 @@ template <int BN> struct TcShape {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
 };
 
-// grid = (ceil(N / 128), ceil(M / BN)), block = 192, dynamic smem = TcShape<BN>::SMEM_BYTES.
+// grid = (ceil(N / 128), ceil(M / BN), splits), block = 192, dynamic smem = TcShape<BN>::SMEM_BYTES.
+// With splits > 1 CTA z reduces K blocks [z * KB / splits, (z + 1) * KB / splits) and the epilogue
+// must be additive (EPI_RESID / EPI_ATOMIC): partial sums are added with fp32 atomics.
 template <int BN>
 __global__ void __launch_bounds__(192, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
@@ -133,7 +135,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int f0 = blockIdx.x * TC_BM, t0 = blockIdx.y * BN;
-  const int KB = K / TC_BK;
+  const int KB_all = (K + TC_BK - 1) / TC_BK;
+  const int kb_lo = (int)(((long long)KB_all * blockIdx.z) / gridDim.z);
+  const int kb_hi = (int)(((long long)KB_all * (blockIdx.z + 1)) / gridDim.z);
+  const int KB = kb_hi - kb_lo;
+  const bool atomic = epi == EPI_ATOMIC || (epi == EPI_RESID && gridDim.z > 1);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::STAGES; ++s) {
@@ -160,8 +166,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { atomicExch(status, DEV_TIMEOUT_TMA); break; }
       const uint32_t dst = tiles + s * S::STAGE_BYTES;
       mbar_expect_tx(full0 + 8 * s, S::STAGE_BYTES);
-      tma_load_2d(dst, &mapW, kb * TC_BK, f0, full0 + 8 * s);
-      tma_load_2d(dst + TC_W_BYTES, &mapA, kb * TC_BK, t0, full0 + 8 * s);
+      tma_load_2d(dst, &mapW, (kb_lo + kb) * TC_BK, f0, full0 + 8 * s);
+      tma_load_2d(dst + TC_W_BYTES, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * s);
     }
   } else if (warp == 5 && lane == 0) {
     // ---------------- MMA issuer
@@ -197,7 +203,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
             const int t = t0 + c0 + j;
             if (t < M) {
               const size_t o = (size_t)t * N + f;
-              if (epi == EPI_F32) ((float *)C)[o] = v[j];
+              if (atomic) atomicAdd((float *)C + o, v[j]);
+              else if (epi == EPI_F32) ((float *)C)[o] = v[j];
               else if (epi == EPI_T) ((bf16 *)C)[o] = __float2bfloat16_rn(v[j]);
               else if (epi == EPI_GELU_T) ((bf16 *)C)[o] = __float2bfloat16_rn(gelu_erf(v[j]));
               else ((float *)C)[o] += v[j];
@@ -261,7 +268,7 @@ static int gemm_tc_plan(GemmTcPlan *plan, const void *W, int N, int K, const voi
   plan->valid = false;
   plan->N = N;
   plan->K = K;
-  if (K % TC_BK || K < TC_BK || N < 1 || M_max < 1) return 0;
+  if (K % 8 || K < 16 || N < 1 || M_max < 1) return 0;   // row pitch must be a multiple of 16 bytes
   if (((uintptr_t)W & 15) || ((uintptr_t)A & 15)) return 0;
   if (!g_encode) return -4;
   if (tc_encode(&plan->mapW, W, N, K, TC_BM)) return -4;
@@ -271,9 +278,33 @@ static int gemm_tc_plan(GemmTcPlan *plan, const void *W, int N, int K, const voi
   return 0;
 }
 
+// Token-tile width for M tokens.
+static int gemm_tc_bn(int N, int M) {
+  (void)N;
+  if (M <= 16) return 16;
+  if (M <= 32) return 32;
+  if (M <= 64) return 64;
+  if (M <= 128) return 128;
+  return 256;
+}
+
+// Number of K splits: fill the SMs when the (feature tile x token tile) grid is small.  Only
+// additive epilogues can be split.
+static int gemm_tc_splits(int N, int K, int M, bool additive) {
+  if (!additive) return 1;
+  const int bn = gemm_tc_bn(N, M);
+  const int tiles = ((N + TC_BM - 1) / TC_BM) * ((M + bn - 1) / bn);
+  const int KB = (K + TC_BK - 1) / TC_BK;
+  if (tiles >= 96 || KB < 2) return 1;
+  int s = 148 / tiles;
+  if (s > KB) s = KB;
+  return s < 1 ? 1 : s;
+}
+
 template <int BN>
 static void gemm_tc_launch_bn(cudaStream_t s, const GemmTcPlan &p, int idx, void *C, int M, int epi, int *status) {
-  dim3 grid((p.N + TC_BM - 1) / TC_BM, (M + BN - 1) / BN);
+  const bool additive = epi == EPI_RESID || epi == EPI_ATOMIC;
+  dim3 grid((p.N + TC_BM - 1) / TC_BM, (M + BN - 1) / BN, gemm_tc_splits(p.N, p.K, M, additive));
   gemm_tc_kernel<BN><<<grid, 192, TcShape<BN>::SMEM_BYTES, s>>>(p.mapW, p.mapA[idx], C, M, p.N, p.K, epi, status);
 }
 
@@ -282,12 +313,13 @@ static bool gemm_tc_launch(cudaStream_t s, const GemmTcPlan &p, const void *A, v
                            int *status) {
   (void)A;
   if (!p.valid) return false;
-  const int ftiles = (p.N + TC_BM - 1) / TC_BM;
-  if (M <= 16) gemm_tc_launch_bn<16>(s, p, 0, C, M, epi, status);
-  else if (M <= 32) gemm_tc_launch_bn<32>(s, p, 1, C, M, epi, status);
-  else if (M <= 64) gemm_tc_launch_bn<64>(s, p, 2, C, M, epi, status);
-  else if (M <= 128 || ftiles * ((M + 127) / 128) <= 2 * 148) gemm_tc_launch_bn<128>(s, p, 3, C, M, epi, status);
-  else gemm_tc_launch_bn<256>(s, p, 4, C, M, epi, status);
+  switch (gemm_tc_bn(p.N, M)) {
+    case 16: gemm_tc_launch_bn<16>(s, p, 0, C, M, epi, status); break;
+    case 32: gemm_tc_launch_bn<32>(s, p, 1, C, M, epi, status); break;
+    case 64: gemm_tc_launch_bn<64>(s, p, 2, C, M, epi, status); break;
+    case 128: gemm_tc_launch_bn<128>(s, p, 3, C, M, epi, status); break;
+    default: gemm_tc_launch_bn<256>(s, p, 4, C, M, epi, status); break;
+  }
   return true;
 }
 

@@ -63,44 +63,88 @@ __global__ void denorm_kernel(const float *__restrict__ hist, int N, int P, int 
   for (int i = threadIdx.x; i < H; i += blockDim.x) out[(size_t)b * H + i] = hb[i] * s + m;
 }
 
+// 16-byte vector loads of T (8 bf16 or 4 fp32) unpacked to floats.
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+  static constexpr int N = 4;
+  static __device__ __forceinline__ void load(const float *p, float *v) {
+    const float4 t = *reinterpret_cast<const float4 *>(p);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  }
+};
+template <> struct Vec16<bf16> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void load(const bf16 *p, float *v) {
+    const uint4 t = *reinterpret_cast<const uint4 *>(p);
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+};
+
 // ----------------------------------------------------------------------------------
-// Patch embedding x[row, :] = W_emb[d, P] . z, z = history token (fp32).  grid = M rows,
-// block = 128.  A warp takes output features f, f + 4, ...; lanes stride over P.
+// Patch embedding x[row, f] = sum_i W_emb[f, i] * z[i], z = history token (fp32).
+// grid = (M rows, ceil(d / 128)), block = 128: one output feature per thread, its weight
+// row (P elements, a multiple of 16) read with independent 16-byte loads.
 // ----------------------------------------------------------------------------------
 template <typename T>
-__global__ void embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d,
-                             const T *__restrict__ W, float *__restrict__ x) {
+__global__ void __launch_bounds__(128)
+embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *__restrict__ W,
+             float *__restrict__ x) {
   extern __shared__ float zs[];
   const int row = blockIdx.x, b = row / g.q_len, j = row % g.q_len;
   const float *z = hist + ((size_t)b * g.cap + pos0_of(g, b) + j) * P;
   for (int i = threadIdx.x; i < P; i += blockDim.x) zs[i] = z[i];
   __syncthreads();
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
-  for (int f = w; f < d; f += nw) {
-    const T *wr = W + (size_t)f * P;
-    float acc = 0.f;
-    for (int i = lane; i < P; i += 32) acc = fmaf(to_f32(wr[i]), zs[i], acc);
-    acc = warp_sum(acc);
-    if (lane == 0) x[(size_t)row * d + f] = acc;
+  const int f = blockIdx.y * 128 + threadIdx.x;
+  if (f >= d) return;
+  const T *wr = W + (size_t)f * P;
+  constexpr int V = Vec16<T>::N;
+  float acc = 0.f;
+#pragma unroll 4
+  for (int i = 0; i < P; i += V) {
+    float w[V];
+    Vec16<T>::load(wr + i, w);
+#pragma unroll
+    for (int c = 0; c < V; ++c) acc = fmaf(w[c], zs[i + c], acc);
   }
+  x[(size_t)row * d + f] = acc;
 }
 
 // ----------------------------------------------------------------------------------
 // RMSNorm: a[row, :] = g * x / sqrt(mean(x^2) + eps), rounded to T.  grid = M, block 128.
+// Optionally clears zero_cols floats of row `row` of a scratch matrix (the accumulator of
+// a following split-K contraction).
 // ----------------------------------------------------------------------------------
 template <typename T>
-__global__ void rmsnorm_kernel(const float *__restrict__ x, const float *__restrict__ gain, int d,
-                               float eps, T *__restrict__ a) {
+__global__ void __launch_bounds__(128)
+rmsnorm_kernel(const float *__restrict__ x, const float *__restrict__ gain, int d, float eps,
+               T *__restrict__ a, float *__restrict__ zero, int zero_cols) {
   __shared__ float red[32];
   const size_t row = blockIdx.x;
-  const float *xr = x + row * d;
+  const float4 *xr = reinterpret_cast<const float4 *>(x + row * d);
+  const float4 *gr = reinterpret_cast<const float4 *>(gain);
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const float v = xr[i];
-    ss = fmaf(v, v, ss);
+  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+    const float4 v = xr[i];
+    ss = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, ss))));
+  }
+  if (zero) {
+    float4 *zr = reinterpret_cast<float4 *>(zero + row * zero_cols);
+    for (int i = threadIdx.x; i < zero_cols / 4; i += blockDim.x) zr[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
   const float rstd = rsqrtf(block_sum(ss, red) / d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x) a[row * d + i] = from_f32<T>(gain[i] * xr[i] * rstd);
+  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
+    const float4 v = xr[i], gg = gr[i];
+    T *o = a + row * d + 4 * i;
+    o[0] = from_f32<T>(gg.x * v.x * rstd);
+    o[1] = from_f32<T>(gg.y * v.y * rstd);
+    o[2] = from_f32<T>(gg.z * v.z * rstd);
+    o[3] = from_f32<T>(gg.w * v.w * rstd);
+  }
 }
 
 // ----------------------------------------------------------------------------------
@@ -108,7 +152,7 @@ __global__ void rmsnorm_kernel(const float *__restrict__ x, const float *__restr
 // 256 threads, 4x4 outputs per thread.  K must be a multiple of 16.
 // Epilogues: store fp32 | store T | GELU -> T | residual add into fp32.
 // ----------------------------------------------------------------------------------
-enum { EPI_F32 = 0, EPI_T = 1, EPI_GELU_T = 2, EPI_RESID = 3 };
+enum { EPI_F32 = 0, EPI_T = 1, EPI_GELU_T = 2, EPI_RESID = 3, EPI_ATOMIC = 4 };   // ATOMIC: fp32 atomic add
 
 template <typename T, int EPI>
 __global__ void __launch_bounds__(256)
@@ -179,27 +223,41 @@ gemm_simt_kernel(const T *__restrict__ A, const T *__restrict__ W, void *__restr
 //   Kc,Vc [B, heads, cap, DH] T: this layer's cache; positions < pos0 are valid
 //   rope  [cap, DH/2] float2 (cos, sin), rotate-half pairing (i, i + DH/2)
 //   out   [M, d] T
-// The CTA loads keys 0..pos0-1 from the cache and keys of this pass (rotated here) up to
-// its last query into shared memory once; all queries of the tile share that read.  The
-// tile that owns a token writes its rotated key and its value to the cache.
+// The CTA loads keys 0..pos0-1 from the cache (16-byte loads) and the keys of this pass
+// (rotated here) up to its last query into shared memory once; all queries of the tile share
+// that read.  The tile that owns a token writes its rotated key and its value to the cache.
 // grid = (heads, B, ceil(q_len / QT)), block = 128 (one query per warp at a time).
-// Dynamic smem: K tile [nk][DH + 2] T, V tile [nk][DH] T, scores [4][nk] f32, q [4][DH] f32.
+// Shared memory is addressed in 32-bit words: K rows are padded by one word so that lanes
+// reading different keys hit different banks.
+//   K tile [nk][KW] words, V tile [nk][VW] words, scores [4][nk] f32, q [4][DH] f32.
 // ----------------------------------------------------------------------------------
-template <typename T> struct KPad { static constexpr int v = 2; };
-template <> struct KPad<float> { static constexpr int v = 1; };
+template <typename T> struct AttnWords;                 // words per DH elements
+template <> struct AttnWords<float> {
+  static __host__ __device__ constexpr int per_row(int dh) { return dh; }
+};
+template <> struct AttnWords<bf16> {
+  static __host__ __device__ constexpr int per_row(int dh) { return dh / 2; }
+};
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t *>(&v);
+}
 
 template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
             const float2 *__restrict__ rope, PassGeom g, int n_heads, int QT, int nk_max,
             T *__restrict__ out) {
-  constexpr int KP = DH + KPad<T>::v;
+  constexpr bool BF = sizeof(T) == 2;
+  constexpr int VW = AttnWords<T>::per_row(DH);   // words per value row
+  constexpr int KW = VW + 1;                      // padded key row
   constexpr int HALF = DH / 2;
-  constexpr int DPL = DH / 32;                 // output dims per lane
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  T *Ks = reinterpret_cast<T *>(smem_raw);
-  T *Vs = Ks + (size_t)nk_max * KP;
-  float *sc = reinterpret_cast<float *>(Vs + (size_t)nk_max * DH);
+  constexpr int DPL = DH / 32;                    // output dims per lane
+  constexpr int EPV = 16 / sizeof(T);             // elements per 16-byte vector
+  extern __shared__ __align__(16) uint32_t smem_w[];
+  uint32_t *Vs = smem_w;                          // [nk_max][VW], 16-byte aligned rows
+  uint32_t *Ks = Vs + (size_t)nk_max * VW;        // [nk_max][KW]
+  float *sc = reinterpret_cast<float *>(Ks + (size_t)nk_max * KW);
   float *qs = sc + 4 * nk_max;
 
   const int h = blockIdx.x, b = blockIdx.y, qt = blockIdx.z;
@@ -211,30 +269,52 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   T *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
   T *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
 
-  // cached keys/values
-  for (int i = threadIdx.x; i < p0 * DH; i += blockDim.x) {
-    const int t = i / DH, c = i % DH;
-    Ks[t * KP + c] = Kb[i];
-    Vs[t * DH + c] = Vb[i];
+  // cached keys/values: p0 rows of DH elements, 16 bytes at a time
+  for (int i = threadIdx.x; i < p0 * (DH / EPV); i += blockDim.x) {
+    const int t = i / (DH / EPV), c = i % (DH / EPV);
+    const uint4 kv = *reinterpret_cast<const uint4 *>(Kb + (size_t)t * DH + c * EPV);
+    const uint4 vv = *reinterpret_cast<const uint4 *>(Vb + (size_t)t * DH + c * EPV);
+    uint32_t *kd = Ks + (size_t)t * KW + c * 4;
+    kd[0] = kv.x; kd[1] = kv.y; kd[2] = kv.z; kd[3] = kv.w;
+    *reinterpret_cast<uint4 *>(Vs + (size_t)t * VW + c * 4) = vv;
   }
-  // keys/values of this pass (rotate keys; the owning tile appends to the cache)
-  for (int i = threadIdx.x; i < j_hi * HALF; i += blockDim.x) {
-    const int j = i / HALF, c = i % HALF;
+  // keys/values of this pass (rotate keys; the owning tile appends to the cache).
+  // One thread handles the element pair (c, c + 1) of the first half and its rotation partners.
+  for (int i = threadIdx.x; i < j_hi * (HALF / 2); i += blockDim.x) {
+    const int j = i / (HALF / 2), c = (i % (HALF / 2)) * 2;
     const float *src = qkv + (row0 + j) * 3 * d + h * DH;
-    const float2 cs = rope[(size_t)(p0 + j) * HALF + c];
-    const float k1 = src[d + c], k2 = src[d + c + HALF];
-    const T r1 = from_f32<T>(k1 * cs.x - k2 * cs.y), r2 = from_f32<T>(k2 * cs.x + k1 * cs.y);
-    const T v1 = from_f32<T>(src[2 * d + c]), v2 = from_f32<T>(src[2 * d + c + HALF]);
     const int t = p0 + j;
-    Ks[t * KP + c] = r1;
-    Ks[t * KP + c + HALF] = r2;
-    Vs[t * DH + c] = v1;
-    Vs[t * DH + c + HALF] = v2;
-    if (j >= j_lo) {
-      Kb[(size_t)t * DH + c] = r1;
-      Kb[(size_t)t * DH + c + HALF] = r2;
-      Vb[(size_t)t * DH + c] = v1;
-      Vb[(size_t)t * DH + c + HALF] = v2;
+    const float4 cs = *reinterpret_cast<const float4 *>(rope + (size_t)t * HALF + c);   // cos0 sin0 cos1 sin1
+    const float2 ka = *reinterpret_cast<const float2 *>(src + d + c);
+    const float2 kb = *reinterpret_cast<const float2 *>(src + d + c + HALF);
+    const float2 va = *reinterpret_cast<const float2 *>(src + 2 * d + c);
+    const float2 vb = *reinterpret_cast<const float2 *>(src + 2 * d + c + HALF);
+    const float r1a = ka.x * cs.x - kb.x * cs.y, r1b = ka.y * cs.z - kb.y * cs.w;    // first half
+    const float r2a = kb.x * cs.x + ka.x * cs.y, r2b = kb.y * cs.z + ka.y * cs.w;    // second half
+    if (BF) {
+      const uint32_t k1 = pack_bf16x2(r1a, r1b), k2 = pack_bf16x2(r2a, r2b);
+      const uint32_t v1 = pack_bf16x2(va.x, va.y), v2 = pack_bf16x2(vb.x, vb.y);
+      Ks[(size_t)t * KW + c / 2] = k1;
+      Ks[(size_t)t * KW + (c + HALF) / 2] = k2;
+      Vs[(size_t)t * VW + c / 2] = v1;
+      Vs[(size_t)t * VW + (c + HALF) / 2] = v2;
+      if (j >= j_lo) {
+        uint32_t *kg = reinterpret_cast<uint32_t *>(Kb + (size_t)t * DH);
+        uint32_t *vg = reinterpret_cast<uint32_t *>(Vb + (size_t)t * DH);
+        kg[c / 2] = k1; kg[(c + HALF) / 2] = k2;
+        vg[c / 2] = v1; vg[(c + HALF) / 2] = v2;
+      }
+    } else {
+      float *kf = reinterpret_cast<float *>(Ks + (size_t)t * KW);
+      float *vf = reinterpret_cast<float *>(Vs + (size_t)t * VW);
+      kf[c] = r1a; kf[c + 1] = r1b; kf[c + HALF] = r2a; kf[c + HALF + 1] = r2b;
+      vf[c] = va.x; vf[c + 1] = va.y; vf[c + HALF] = vb.x; vf[c + HALF + 1] = vb.y;
+      if (j >= j_lo) {
+        float *kg = reinterpret_cast<float *>(Kb + (size_t)t * DH);
+        float *vg = reinterpret_cast<float *>(Vb + (size_t)t * DH);
+        kg[c] = r1a; kg[c + 1] = r1b; kg[c + HALF] = r2a; kg[c + HALF + 1] = r2b;
+        vg[c] = va.x; vg[c + 1] = va.y; vg[c + HALF] = vb.x; vg[c + HALF + 1] = vb.y;
+      }
     }
   }
   __syncthreads();
@@ -255,10 +335,20 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
     const int nv = p0 + j + 1;                       // causal: keys 0..p0+j
     float mx = -INFINITY;
     for (int t = lane; t < nv; t += 32) {
-      const T *kr = Ks + (size_t)t * KP;
+      const uint32_t *kr = Ks + (size_t)t * KW;
       float s = 0.f;
+      if (BF) {
 #pragma unroll 8
-      for (int c = 0; c < DH; ++c) s = fmaf(my_q[c], to_f32(kr[c]), s);
+        for (int c = 0; c < DH / 2; ++c) {
+          const uint32_t kk = kr[c];
+          const float2 qq = *reinterpret_cast<const float2 *>(my_q + 2 * c);
+          s = fmaf(qq.x, __uint_as_float(kk << 16), s);
+          s = fmaf(qq.y, __uint_as_float(kk & 0xffff0000u), s);
+        }
+      } else {
+#pragma unroll 8
+        for (int c = 0; c < DH; ++c) s = fmaf(my_q[c], __uint_as_float(kr[c]), s);
+      }
       my_sc[t] = s;
       mx = fmaxf(mx, s);
     }
@@ -274,10 +364,27 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
     float acc[DPL];
 #pragma unroll
     for (int c = 0; c < DPL; ++c) acc[c] = 0.f;
-    for (int t = 0; t < nv; ++t) {
-      const float p = my_sc[t];
+    if (BF) {
+      // lane owns DPL consecutive dims = DPL / 2 words of each value row
+      for (int t = 0; t < nv; ++t) {
+        const float p = my_sc[t];
 #pragma unroll
-      for (int c = 0; c < DPL; ++c) acc[c] = fmaf(p, to_f32(Vs[(size_t)t * DH + lane * DPL + c]), acc[c]);
+        for (int c = 0; c < DPL / 2; ++c) {
+          const uint32_t vv = Vs[(size_t)t * VW + lane * (DPL / 2) + c];
+          acc[2 * c] = fmaf(p, __uint_as_float(vv << 16), acc[2 * c]);
+          acc[2 * c + 1] = fmaf(p, __uint_as_float(vv & 0xffff0000u), acc[2 * c + 1]);
+        }
+        if (DPL == 1) {                              // DH = 32: half a word per lane
+          const uint32_t vv = Vs[(size_t)t * VW + lane / 2];
+          acc[0] = fmaf(p, __uint_as_float((lane & 1) ? (vv & 0xffff0000u) : (vv << 16)), acc[0]);
+        }
+      }
+    } else {
+      for (int t = 0; t < nv; ++t) {
+        const float p = my_sc[t];
+#pragma unroll
+        for (int c = 0; c < DPL; ++c) acc[c] = fmaf(p, __uint_as_float(Vs[(size_t)t * VW + lane * DPL + c]), acc[c]);
+      }
     }
     const float inv = 1.f / sum;
 #pragma unroll
@@ -289,16 +396,18 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
 
 // ----------------------------------------------------------------------------------
 // Final RMSNorm + mean head for selected tokens: o = W_head[P, d] . (g_f * x * rstd).
-// Normalised activations stay fp32 here.  grid = (rows), block = 128.
+// Normalised activations stay fp32 here.  grid = (rows, ceil(P / 8)), block = 256: each warp
+// produces one output element with 16-byte weight loads.
 // only_last = 1: one row per series, the pass's last token, written to the series' next
 //   history slot hist[b, pos0 + q_len, :]  (draft steps, target-only steps);
 // only_last = 0: every token, written to vout[b, j, :]  (verification; vout [B, q_len, P]).
 // ----------------------------------------------------------------------------------
 template <typename T>
-__global__ void head_kernel(const float *__restrict__ x, const float *__restrict__ gain,
-                            const T *__restrict__ Wh, int d, int P, float eps, PassGeom g,
-                            int only_last, float *__restrict__ hist, float *__restrict__ vout) {
-  extern __shared__ float xs[];
+__global__ void __launch_bounds__(256)
+head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T *__restrict__ Wh, int d,
+            int P, float eps, PassGeom g, int only_last, float *__restrict__ hist,
+            float *__restrict__ vout) {
+  extern __shared__ __align__(16) float xs[];
   __shared__ float red[32];
   int b, j;
   if (only_last) { b = blockIdx.x; j = g.q_len - 1; }
@@ -315,14 +424,20 @@ __global__ void head_kernel(const float *__restrict__ x, const float *__restrict
   __syncthreads();
   float *dst = only_last ? hist + ((size_t)b * g.cap + pos0_of(g, b) + g.q_len) * P
                          : vout + ((size_t)b * g.q_len + j) * P;
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
-  for (int p = w; p < P; p += nw) {
-    const T *wr = Wh + (size_t)p * d;
-    float acc = 0.f;
-    for (int i = lane; i < d; i += 32) acc = fmaf(to_f32(wr[i]), xs[i], acc);
-    acc = warp_sum(acc);
-    if (lane == 0) dst[p] = acc;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int p = blockIdx.y * 8 + w;
+  if (p >= P) return;
+  const T *wr = Wh + (size_t)p * d;
+  constexpr int V = Vec16<T>::N;
+  float acc = 0.f;
+  for (int i = lane * V; i < d; i += 32 * V) {
+    float wv[V];
+    Vec16<T>::load(wr + i, wv);
+#pragma unroll
+    for (int c = 0; c < V; ++c) acc = fmaf(wv[c], xs[i + c], acc);
   }
+  acc = warp_sum(acc);
+  if (lane == 0) dst[p] = acc;
 }
 
 }  // namespace tsfm

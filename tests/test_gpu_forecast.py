@@ -135,7 +135,7 @@ def test_argument_errors_are_reported_not_fatal():
 
 def test_host_buffer_entry_points_match_device_ones():
     import paper_2511_18191_b200 as tsfm
-    wl = workload("C1")
+    wl = workload("C0", batch=4, series_recipe="c1")      # fp32 path: bit-reproducible
     dec, tw, dw = make_decoder(wl)
     s, ctx = series_on_device(wl)
     out, _ = dec.forecast(ctx, wl.horizon, wl.K, 1.0, 3)

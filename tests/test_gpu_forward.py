@@ -58,7 +58,7 @@ def test_bf16_forward_matches_oracle(backend, target, draft, P, n, mode):
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (16, 128, 64), (32, 1536, 512), (160, 512, 2048), (33, 96, 128),
-                                   (200, 200, 192), (960, 2048, 512), (300, 384, 1280), (2048, 768, 768)])
+                                   (200, 200, 192), (40, 512, 96), (7, 130, 16), (960, 2048, 512), (300, 384, 1280), (2048, 768, 768)])
 def test_tensor_core_gemm_matches_fp64_product_and_fma_kernel(M, N, K):
     import paper_2511_18191_b200 as tsfm
     g = torch.Generator(device="cpu").manual_seed(M * 7 + N)
