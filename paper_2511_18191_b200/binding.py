@@ -72,7 +72,7 @@ class tsfm_kernel_stat(C.Structure):
 def _load() -> C.CDLL:
     path = _build.LIB
     if not os.path.exists(path):
-        raise ImportError(f"{path} is missing: build it with `python -m paper_2511_18191_b200.build` "
+        raise ImportError(f"{path} is missing: build it with `python paper_2511_18191_b200/build.py` "
                           "(nvcc, sm_100a); there is no fallback implementation")
     lib = C.CDLL(path)
     i32, f32, u64, vp, sz = C.c_int32, C.c_float, C.c_uint64, C.c_void_p, C.c_size_t
