@@ -204,6 +204,29 @@ int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t
 int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C,
                    int32_t M, int32_t N, int32_t Kd, int32_t backend);
 
+/* The same contraction as tsfm_gemm_bf16 (tensor-core kernel, K split across CTAs with fp32
+ * atomic accumulation) for callers that must not allocate device memory.  The paper has no
+ * counterpart to this entry point; it exists for the library's users.  Who they are: a
+ * serving loop that checks the contraction while forecasts are in flight on other streams
+ * (cudaMalloc and cudaFree synchronise the whole device and would stall those forecasts), and
+ * a process that has handed all device memory to a pooling allocator, where a raw cudaMalloc
+ * can simply fail.  This call makes no cudaMalloc, cudaFree or other allocating call.
+ *   - Scratch (the split-K accumulator and a status word) is a fixed array of
+ *     256 + 4 * TSFM_STATIC_GEMM_MAX_ELEMS bytes (4 MiB + 256 B) inside the library image; every
+ *     GPU that loads the library holds it until the process exits.
+ *   - M * N must not exceed TSFM_STATIC_GEMM_MAX_ELEMS: larger outputs are rejected with
+ *     TSFM_ERR_SHAPE and a message available from tsfm_last_cuda_error().
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside of any stream capture.
+ *   - Every call on a device shares the one array, which still holds the previous call's
+ *     contents: the call clears the part it uses before accumulating.  Two calls that overlap
+ *     on the GPU (different streams, or threads) race on it; serialise them.
+ * A, W dev bf16 row-major, C dev fp32 [M, N] row-major (written last, by a device-to-device
+ * copy); synchronises `stream` before returning. */
+#define TSFM_STATIC_GEMM_MAX_ELEMS (1 << 20)
+int tsfm_gemm_bf16_static(void *stream, const void *A, const void *W, float *C,
+                          int32_t M, int32_t N, int32_t Kd);
+
 /* Per-launch timing, for roofline accounting.  While enabled, every kernel launch of the handle
  * is bracketed by two CUDA events on the handle's stream (this perturbs end-to-end time: do not
  * quote throughput from a profiled call).  tsfm_spec_set_profiling clears the records.

@@ -24,7 +24,7 @@ TSFM_MAX_K = 32
 EXPORTS = [
     "tsfm_weights_bytes", "tsfm_weights_offset", "tsfm_spec_create", "tsfm_spec_forecast",
     "tsfm_target_only_forecast", "tsfm_spec_forecast_host", "tsfm_target_only_forecast_host",
-    "tsfm_spec_last_trace", "tsfm_accept_round", "tsfm_model_forward", "tsfm_gemm_bf16",
+    "tsfm_spec_last_trace", "tsfm_accept_round", "tsfm_model_forward", "tsfm_gemm_bf16", "tsfm_gemm_bf16_static",
     "tsfm_spec_set_profiling", "tsfm_spec_kernel_profile", "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
 ]
 
@@ -98,6 +98,8 @@ def _load() -> C.CDLL:
     lib.tsfm_model_forward.argtypes = [vp, i32, vp, i32, i32, vp]
     lib.tsfm_gemm_bf16.restype = C.c_int
     lib.tsfm_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
+    lib.tsfm_gemm_bf16_static.restype = C.c_int
+    lib.tsfm_gemm_bf16_static.argtypes = [vp, vp, vp, vp, i32, i32, i32]
     lib.tsfm_spec_set_profiling.restype = C.c_int
     lib.tsfm_spec_set_profiling.argtypes = [vp, i32]
     lib.tsfm_spec_kernel_profile.restype = C.c_int
@@ -245,6 +247,18 @@ def tsfm_model_forward(h, which: int, tokens, B: int, n: int, out) -> None:
 
 def tsfm_gemm_bf16(stream, A, W, Cout, M: int, N: int, Kd: int, backend: int) -> None:
     _check(lib.tsfm_gemm_bf16(stream, _ptr(A), _ptr(W), _ptr(Cout), M, N, Kd, backend), "tsfm_gemm_bf16")
+
+
+TSFM_STATIC_GEMM_MAX_ELEMS = 1 << 20
+
+
+def tsfm_gemm_bf16_static(stream, A, W, Cout, M: int, N: int, Kd: int) -> None:
+    """The contraction of tsfm_gemm_bf16 without any device allocation (scratch is a fixed array inside
+    the library; M * N <= TSFM_STATIC_GEMM_MAX_ELEMS; calls on one device must not overlap)."""
+    code = lib.tsfm_gemm_bf16_static(stream, _ptr(A), _ptr(W), _ptr(Cout), M, N, Kd)
+    if code == TSFM_ERR_SHAPE:
+        raise TsfmError(code, "tsfm_gemm_bf16_static: " + lib.tsfm_last_cuda_error().decode())
+    _check(code, "tsfm_gemm_bf16_static")
 
 
 def tsfm_spec_set_profiling(h, enable: bool) -> None:

@@ -8,6 +8,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -771,6 +772,67 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t
   cudaFree(status);
   CU_TRY(e1);
   CU_TRY(e2);
+  CU_TRY(cudaGetLastError());
+  if (!ok) return TSFM_ERR_INTERNAL;
+  return hs ? TSFM_ERR_TIMEOUT : TSFM_OK;
+}
+
+// ------------------------------------------------------------------------------------
+// Allocation-free variant of the tensor-core contraction (see include/tsfm.h).
+// The accumulator of the K-split partial sums and the kernel's status word live in a
+// file-scope device array instead of cudaMalloc'd memory.  The array's name is only a
+// host-side handle for the symbol: its device address is looked up once per device with
+// cudaGetSymbolAddress and that pointer is what the kernels receive.
+// ------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[256 + sizeof(float) * TSFM_STATIC_GEMM_MAX_ELEMS];
+
+static int static_scratch_ptr(unsigned char **out) {
+  static std::mutex mu;
+  static unsigned char *per_device[64] = {nullptr};
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return TSFM_ERR_INTERNAL;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!per_device[dev]) {
+    unsigned char *p = nullptr;
+    CU_TRY(cudaGetSymbolAddress((void **)&p, g_static_scratch));
+    if (!p) return TSFM_ERR_INTERNAL;
+    per_device[dev] = p;
+  }
+  *out = per_device[dev];
+  return TSFM_OK;
+}
+
+int tsfm_gemm_bf16_static(void *stream, const void *A, const void *W, float *C, int32_t M, int32_t N,
+                          int32_t Kd) {
+  if (!A || !W || !C) return TSFM_ERR_ARG;
+  if (M < 1 || N < 1 || Kd < 16 || Kd % 16) return TSFM_ERR_ARG;
+  if ((long long)M * N > (long long)TSFM_STATIC_GEMM_MAX_ELEMS) {
+    g_cuda_err = "tsfm_gemm_bf16_static: M * N = " + std::to_string((long long)M * N) +
+                 " output elements exceed the static scratch capacity of " +
+                 std::to_string((long long)TSFM_STATIC_GEMM_MAX_ELEMS);
+    return TSFM_ERR_SHAPE;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  unsigned char *scratch = nullptr;
+  if (int rc = static_scratch_ptr(&scratch)) return rc;
+  if (int rc = gemm_tc_init()) return rc;
+  GemmTcPlan plan;
+  if (int rc = gemm_tc_plan(&plan, W, N, Kd, A, M)) return rc;
+  if (!plan.valid) return TSFM_ERR_SHAPE;
+  int *status = (int *)scratch;
+  float *acc = (float *)(scratch + 256);
+  const size_t out_bytes = sizeof(float) * (size_t)M * N;
+  // the array keeps whatever the previous call left: the status word and the part of the
+  // accumulator this call adds into must start at zero
+  CU_TRY(cudaMemsetAsync(status, 0, 256, s));
+  CU_TRY(cudaMemsetAsync(acc, 0, out_bytes, s));
+  const bool ok = gemm_tc_launch(s, plan, A, acc, M, EPI_ATOMIC, status);
+  if (ok) LAUNCHED();
+  int hs = 0;
+  CU_TRY(cudaMemcpyAsync(C, acc, out_bytes, cudaMemcpyDeviceToDevice, s));
+  CU_TRY(cudaMemcpyAsync(&hs, status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CU_TRY(cudaStreamSynchronize(s));
   CU_TRY(cudaGetLastError());
   if (!ok) return TSFM_ERR_INTERNAL;
   return hs ? TSFM_ERR_TIMEOUT : TSFM_OK;
