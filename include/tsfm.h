@@ -57,6 +57,11 @@ extern "C" {
 #define TSFM_GEMM_AUTO  0       /* bf16 contractions on tcgen05 tensor cores where shapes allow     */
 #define TSFM_GEMM_SIMT  1       /* force the plain FMA kernels everywhere (differential reference)  */
 
+#define TSFM_EXEC_GRAPH   0       /* a forecast is one CUDA-graph launch: prologue, a device-side WHILE
+                                   over the rounds, de-normalisation; no host round trip             */
+#define TSFM_EXEC_STREAM  1       /* kernels are launched one by one and the host checks for completion
+                                   after every round (reference behaviour; also used while profiling) */
+
 #define TSFM_MAX_K 32           /* hard upper bound on the block size K                             */
 
 typedef struct tsfm_spec tsfm_spec;   /* opaque decoder handle */
@@ -82,7 +87,7 @@ typedef struct {
   float   rms_eps;              /* RMSNorm epsilon (1e-6)                                        */
   float   norm_eps;             /* instance-norm variance epsilon (1e-5)                         */
   float   rope_base;            /* RoPE base (1e4)                                               */
-  int32_t reserved0;
+  int32_t exec_mode;            /* TSFM_EXEC_*                                                   */
   void   *stream;               /* cudaStream_t, borrowed for the handle's lifetime              */
 } tsfm_cfg;
 
@@ -246,7 +251,9 @@ int tsfm_spec_kernel_profile(tsfm_spec *h, int32_t cap, int32_t *n, tsfm_kernel_
 
 int tsfm_spec_destroy(tsfm_spec *h);
 
-/* Number of kernels this library has launched in this process (all handles, all streams). */
+/* Number of kernels this library has launched in this process (all handles, all streams).  The
+ * rounds of a graph-mode forecast count their launches on the device: the call waits for the
+ * streams of all live handles to read those counters. */
 int64_t tsfm_launch_count(void);
 
 const char *tsfm_strerror(int code);

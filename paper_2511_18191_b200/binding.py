@@ -19,6 +19,7 @@ TSFM_ERR_ARG, TSFM_ERR_SHAPE, TSFM_ERR_ARCH, TSFM_ERR_CUDA, TSFM_ERR_TIMEOUT, TS
 TSFM_F32, TSFM_BF16 = 0, 1
 TSFM_DRAFT_SEPARATE, TSFM_DRAFT_LAYER_SKIP = 0, 1
 TSFM_GEMM_AUTO, TSFM_GEMM_SIMT = 0, 1
+TSFM_EXEC_GRAPH, TSFM_EXEC_STREAM = 0, 1
 TSFM_MAX_K = 32
 
 EXPORTS = [
@@ -39,7 +40,7 @@ class tsfm_cfg(C.Structure):
                 ("max_batch", C.c_int32), ("max_ctx_tokens", C.c_int32),
                 ("max_horizon_patches", C.c_int32), ("max_K", C.c_int32), ("gemm_backend", C.c_int32),
                 ("rms_eps", C.c_float), ("norm_eps", C.c_float), ("rope_base", C.c_float),
-                ("reserved0", C.c_int32), ("stream", C.c_void_p)]
+                ("exec_mode", C.c_int32), ("stream", C.c_void_p)]
 
 
 class tsfm_weights(C.Structure):
@@ -284,7 +285,7 @@ class SpecDecoder:
 
     def __init__(self, target_w, draft_w, target_arch, draft_arch, patch_len: int, dtype: str,
                  draft_mode: str, max_batch: int, max_ctx_tokens: int, max_horizon_patches: int, max_K: int,
-                 gemm_backend: int = TSFM_GEMM_AUTO, device: str = "cuda:0"):
+                 gemm_backend: int = TSFM_GEMM_AUTO, exec_mode: int = TSFM_EXEC_GRAPH, device: str = "cuda:0"):
         import torch
         self.torch = torch
         self.device = torch.device(device)
@@ -301,6 +302,7 @@ class SpecDecoder:
         cfg.max_batch, cfg.max_ctx_tokens = max_batch, max_ctx_tokens
         cfg.max_horizon_patches, cfg.max_K = max_horizon_patches, max_K
         cfg.gemm_backend = gemm_backend
+        cfg.exec_mode = exec_mode
         cfg.rms_eps, cfg.norm_eps, cfg.rope_base = 1e-6, 1e-5, 1e4
         cfg.stream = torch.cuda.current_stream(self.device).cuda_stream
         self.cfg = cfg

@@ -54,12 +54,45 @@ struct AcceptArgs {
   float *ell, *log_u;              // [B, K] (or NULL)
   AcceptCounters *ctr;             // or NULL
   int *unfinished;                 // or NULL: += 1 per series still short of T after this round
+  // When st is non-NULL the scales (tau), the Philox key and the round index come from it, and
+  // n_accept / ell / log_u / unfinished are per-round arrays indexed by that round.
+  DevState *st;
 };
+
+// Closes a round: accumulates the phase clocks, advances the round counter, adds the round's
+// kernel launches to the device-side launch counter and, inside a captured graph, tells the
+// WHILE node whether another round is needed.  One thread.
+__global__ void round_end_kernel(DevState *st, const int *unfinished, int T,
+                                 cudaGraphConditionalHandle handle, int use_handle,
+                                 const int *body_launches, unsigned long long *launch_ctr) {
+  const int r = st->round;
+  const unsigned long long now = globaltimer_ns();
+  if (r == 0) st->ns_prefill = st->t_phase[0] - st->t_call;
+  st->ns_draft += st->t_phase[1] - st->t_phase[0];
+  st->ns_verify += st->t_phase[2] - st->t_phase[1];
+  st->ns_accept += now - st->t_phase[2];
+  st->round = r + 1;
+  if (body_launches && launch_ctr) *launch_ctr += (unsigned long long)*body_launches;
+  // every round commits at least one patch per unfinished series, so T rounds always suffice:
+  // the second condition bounds the loop whatever the counters say
+  if (use_handle) cudaGraphSetConditional(handle, (unfinished[r] > 0 && r + 1 < T) ? 1u : 0u);
+}
 
 // block = 128 (4 series per CTA), grid = ceil(B / 4).
 __global__ void __launch_bounds__(128) accept_kernel(AcceptArgs a) {
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (a.st) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) a.st->t_phase[2] = globaltimer_ns();
+    const int r = a.st->round;
+    a.sigma_p = a.sigma_q = a.st->tau;
+    a.key = make_uint2(a.st->key0, a.st->key1);
+    a.round_idx = r;
+    if (a.n_accept) a.n_accept += (size_t)r * a.B;
+    if (a.ell) a.ell += (size_t)r * a.B * a.K;
+    if (a.log_u) a.log_u += (size_t)r * a.B * a.K;
+    if (a.unfinished) a.unfinished += r;
+  }
   if (b >= a.B) return;
   const int m = a.done[b];
   if (m >= a.T) {                                   // finished earlier: nothing to decide

@@ -11,6 +11,27 @@ typedef __nv_bfloat16 bf16;
 // Device status codes written by kernels whose bounded waits expire (0 = fine).
 enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPILOGUE = 3 };
 
+// Per-forecast state in device memory.  The first block holds the call's parameters (written
+// by the host before the work is enqueued, so that a captured graph can be replayed with new
+// ones); the rest is loop state and phase clocks kept by the kernels themselves.
+struct DevState {
+  const float *series;            // [B, ctx_len] raw context values
+  float *out;                     // [B, H] forecast
+  float tau;                      // acceptance temperature (the paper's sigma)
+  uint32_t key0, key1;            // Philox key = forecast seed
+  int round;                      // index of the round in flight
+  unsigned long long t_call;      // %globaltimer stamps: call start, ...
+  unsigned long long t_phase[3];  // ... start of this round's draft / verify / accept phase
+  unsigned long long t_end;
+  unsigned long long ns_prefill, ns_draft, ns_verify, ns_accept;   // accumulated phase times
+};
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
 

@@ -8,9 +8,11 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
 #include <string>
+#include <tuple>
 #include <vector>
 
 #include "common.cuh"
@@ -24,6 +26,9 @@ namespace {
 
 std::atomic<long long> g_launches{0};
 thread_local std::string g_cuda_err;
+std::mutex g_handles_mu;
+std::vector<tsfm_spec *> g_handles;           // live handles (their replayed rounds count launches on the device)
+constexpr int kMaxGraphs = 16;                // captured forecast geometries kept per handle
 
 #define CU_TRY(expr)                                                            \
   do {                                                                          \
@@ -99,9 +104,26 @@ struct ModelDev {
 
 }  // namespace
 
+struct GraphKey {
+  int mode, B, N, H, K;
+  bool operator<(const GraphKey &o) const {
+    return std::tie(mode, B, N, H, K) < std::tie(o.mode, o.B, o.N, o.H, o.K);
+  }
+};
+struct GraphInfo {
+  cudaGraphExec_t exec = nullptr;
+  long long n_fixed = 0;                 // kernel launches outside the round loop, per replay
+};
+
 struct tsfm_spec {
   tsfm_cfg cfg{};
-  cudaStream_t stream = nullptr;
+  cudaStream_t stream = nullptr;         // the caller's stream: all work is ordered on it
+  cudaStream_t ls = nullptr;             // stream the launches go to (== stream, or a capturing stream)
+  cudaStream_t cap_stream = nullptr, cap_stream2 = nullptr;   // capture-only streams
+  std::map<GraphKey, GraphInfo> graphs;
+  unsigned long long *dev_launches = nullptr;   // launches made by replayed round bodies
+  int *dev_body_launches = nullptr;             // [kMaxGraphs] launches of one round body, per cached graph
+  DevState *st = nullptr;
   int cap = 0;
   bool use_tc = false;
   ModelDev tgt, drf;
@@ -119,7 +141,7 @@ struct tsfm_spec {
   int *tr_nacc = nullptr;                // [max_T][B]
   float *tr_ell = nullptr, *tr_logu = nullptr;   // [max_T][B][K]
   float *stage_in = nullptr, *stage_out = nullptr;   // device staging for the *_host entry points
-  int last_B = 0, last_K = 0, last_rounds = 0;
+  int last_B = 0, last_K = 0;
   // optional per-launch timing (tsfm_spec_set_profiling)
   bool profiling = false;
   struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
@@ -155,13 +177,13 @@ struct KTimer {
     };
     tsfm_spec::ProfRec r{cls, get(), get(), bytes, flops};
     if (!r.e0 || !r.e1) return;
-    cudaEventRecord(r.e0, h->stream);
+    cudaEventRecord(r.e0, h->ls);
     h->prof.push_back(r);
     idx = h->prof.size() - 1;
     on = true;
   }
   ~KTimer() {
-    if (on) cudaEventRecord(h->prof[idx].e1, h->stream);
+    if (on) cudaEventRecord(h->prof[idx].e1, h->ls);
   }
 };
 
@@ -265,10 +287,10 @@ void gemm(tsfm_spec *h, const GemmTcPlan *plan, const void *A, const void *W, vo
   const double flops = 2.0 * M * N * K;
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
     KTimer kt(h, KC_GEMM_TC, bytes, flops);
-    if (gemm_tc_launch(h->stream, *plan, A, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
+    if (gemm_tc_launch(h->ls, *plan, A, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
   }
   KTimer kt(h, KC_GEMM_SIMT, bytes, flops);
-  launch_gemm_simt<T>(h->stream, (const T *)A, (const T *)W, C, M, N, K, epi);
+  launch_gemm_simt<T>(h->ls, (const T *)A, (const T *)W, C, M, N, K, epi);
 }
 
 template <typename T, int DH>
@@ -284,7 +306,7 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   const double Mr = (double)B * g.q_len;
   KTimer kt(h, KC_ATTN, Mr * 3 * m.arch.d_model * 4 + kv + Mr * m.arch.d_model * (2.0 * sizeof(T) + sizeof(T)),
             4.0 * Mr * (std::max(g.base, 0) + 0.5 * g.q_len) * m.arch.d_model);
-  attn_kernel<T, DH><<<grid, 128, smem, h->stream>>>(h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
+  attn_kernel<T, DH><<<grid, 128, smem, h->ls>>>(h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
                                                      nk_max, (T *)h->ao);
   LAUNCHED();
 }
@@ -293,13 +315,14 @@ enum { HEAD_NONE = 0, HEAD_LAST_TO_HIST = 1, HEAD_ALL_TO_VOUT = 2 };
 
 // One causal pass of a model over q_len new tokens per series (appends to its KV cache).
 template <typename T>
-void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout) {
+void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout,
+              unsigned long long *stamp) {
   const int M = B * g.q_len, d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len;
-  cudaStream_t s = h->stream;
+  cudaStream_t s = h->ls;
   const float eps = h->cfg.rms_eps;
   {
     KTimer kt(h, KC_EMBED, (double)M * P * 4 + (double)d * P * sizeof(T) + (double)M * d * 4, 2.0 * M * P * d);
-    embed_kernel<T><<<dim3(M, (d + 127) / 128), 128, P * sizeof(float), s>>>(h->hist, g, P, d, (const T *)m.W_emb, h->x);
+    embed_kernel<T><<<dim3(M, (d + 127) / 128), 128, P * sizeof(float), s>>>(h->hist, g, P, d, (const T *)m.W_emb, h->x, stamp);
     LAUNCHED();
   }
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
@@ -343,10 +366,11 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   }
 }
 
-void pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout = nullptr) {
+void pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout = nullptr,
+          unsigned long long *stamp = nullptr) {
   if (g.q_len < 1) return;
-  if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout);
-  else run_pass<float>(h, m, B, g, head_mode, vout);
+  if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout, stamp);
+  else run_pass<float>(h, m, B, g, head_mode, vout, stamp);
 }
 
 int check_call(tsfm_spec *h, const float *series, int B, int ctx_len, int H, float *out, int K) {
@@ -362,26 +386,216 @@ int check_call(tsfm_spec *h, const float *series, int B, int ctx_len, int H, flo
   return TSFM_OK;
 }
 
-int begin_forecast(tsfm_spec *h, const float *series, int B, int ctx_len) {
+// ---------------------------------------------------------------- enqueue helpers
+// Each of these only enqueues work on h->ls; none synchronises, so that they can run under
+// stream capture.
+
+void enqueue_begin(tsfm_spec *h, int B, int ctx_len) {
   const int P = h->cfg.patch_len;
+  cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->ls);
+  KTimer kt(h, KC_INSTNORM, (double)B * (ctx_len + (double)h->cap * P) * 4, 4.0 * B * ctx_len);
+  instnorm_kernel<<<B, 256, 0, h->ls>>>(h->st, ctx_len, P, h->cap, h->cfg.norm_eps, h->hist, h->mean, h->sd,
+                                        h->done);
+  LAUNCHED();
+}
+
+void enqueue_denorm(tsfm_spec *h, int B, int N, int H) {
+  KTimer kt(h, KC_DENORM, 8.0 * B * H, 2.0 * B * H);
+  denorm_kernel<<<B, 256, 0, h->ls>>>(h->hist, N, h->cfg.patch_len, h->cap, H, h->mean, h->sd, h->st);
+  LAUNCHED();
+}
+
+// Everything of a speculative forecast that precedes the round loop: counters, traces,
+// instance norm, and the prefill of both caches (the target ingests the context except its
+// last patch, the draft except its last two: those are re-read by the first round).
+void enqueue_spec_prologue(tsfm_spec *h, int B, int N, int T, int K) {
+  cudaStream_t s = h->ls;
+  cudaMemsetAsync(h->ctr, 0, sizeof(AcceptCounters), s);
+  cudaMemsetAsync(h->unfinished, 0, sizeof(int) * (T + 1), s);
+  cudaMemsetAsync(h->tr_nacc, 0xff, sizeof(int) * (size_t)T * B, s);
+  cudaMemsetAsync(h->tr_ell, 0, sizeof(float) * (size_t)T * B * K, s);
+  cudaMemsetAsync(h->tr_logu, 0, sizeof(float) * (size_t)T * B * K, s);
+  enqueue_begin(h, B, N * h->cfg.patch_len);
+  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
+  pass(h, h->drf, B, PassGeom{nullptr, 0, N - 2, h->cap}, HEAD_NONE);
+}
+
+// One round of Algorithm 1 for the whole batch: K draft steps, one verification pass over
+// [pending, x_1..x_K], the fused accept, and the round bookkeeping.  The round index, tau and
+// the Philox key are read from device state, so the same enqueued work serves every round.
+void enqueue_round(tsfm_spec *h, int B, int N, int T, int K, cudaGraphConditionalHandle handle, int use_handle,
+                   const int *body_launches = nullptr) {
+  const int P = h->cfg.patch_len;
+  // step 1 re-ingests the last two committed patches (the draft cache may lack the last
+  // accepted proposal), steps 2..K ingest the previous proposal
+  pass(h, h->drf, B, PassGeom{h->done, N - 2, 2, h->cap}, HEAD_LAST_TO_HIST, nullptr, &h->st->t_phase[0]);
+  for (int i = 2; i <= K; ++i)
+    pass(h, h->drf, B, PassGeom{h->done, N - 1 + (i - 1), 1, h->cap}, HEAD_LAST_TO_HIST);
+  // single-pass verification over [pending, x_1..x_K]
+  pass(h, h->tgt, B, PassGeom{h->done, N - 1, K + 1, h->cap}, HEAD_ALL_TO_VOUT, h->vout, &h->st->t_phase[1]);
+
+  AcceptArgs a{};
+  a.x = a.mu_q = h->hist + (size_t)N * P;       // slot N + done[b] holds x_1
+  a.x_stride_b = (long long)h->cap * P;
+  a.mu_p = h->vout;
+  a.commit = h->hist + (size_t)N * P;
+  a.commit_stride_b = a.x_stride_b;
+  a.commit_accepted = 0;
+  a.commit_follows_done = 1;
+  a.done = h->done;
+  a.B = B; a.K = K; a.P = P; a.T = T;
+  a.margin = h->cfg.dtype == TSFM_BF16 ? 5e-2f : 1e-3f;
+  a.series0 = 0;
+  a.forced_u = nullptr;
+  a.ctr = h->ctr;
+  a.n_accept = h->tr_nacc;
+  a.ell = h->tr_ell;
+  a.log_u = h->tr_logu;
+  a.unfinished = h->unfinished;
+  a.st = h->st;
   {
-    KTimer kt(h, KC_INSTNORM, (double)B * (ctx_len + (double)h->cap * P) * 4, 4.0 * B * ctx_len);
-    instnorm_kernel<<<B, 256, 0, h->stream>>>(series, ctx_len, P, h->cap, h->cfg.norm_eps, h->hist,
-                                              h->mean, h->sd, h->done);
+    KTimer kt(h, KC_ACCEPT, (double)B * (2 * K + 2) * P * 4, 4.0 * B * K * P);
+    accept_kernel<<<(B + 3) / 4, 128, 0, h->ls>>>(a);
     LAUNCHED();
   }
-  CU_TRY(cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream));
+  round_end_kernel<<<1, 1, 0, h->ls>>>(h->st, h->unfinished, T, handle, use_handle, body_launches, h->dev_launches);
+  LAUNCHED();
+}
+
+void enqueue_target_only(tsfm_spec *h, int B, int N, int T, int H) {
+  enqueue_begin(h, B, N * h->cfg.patch_len);
+  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
+  for (int t = 0; t < T; ++t)       // Eq. 1: one target pass per committed patch
+    pass(h, h->tgt, B, PassGeom{nullptr, N - 1 + t, 1, h->cap}, HEAD_LAST_TO_HIST, nullptr,
+         t == 0 ? &h->st->t_phase[0] : nullptr);
+  enqueue_denorm(h, B, N, H);
+}
+
+// ---------------------------------------------------------------- graph capture
+// A forecast of a given geometry is captured once into a CUDA graph and replayed: the
+// prologue, a WHILE node whose body is one round (the round-end kernel sets the condition),
+// and the de-normalisation.  Capture runs on the handle's own streams (the caller's stream
+// may be the legacy default stream, which cannot capture); the graph is launched on the
+// caller's stream.
+int capture_graph(tsfm_spec *h, const GraphKey &k, int slot, GraphInfo *out) {
+  const int P = h->cfg.patch_len, T = (k.H + P - 1) / P;
+  cudaStream_t cs = h->cap_stream, cs2 = h->cap_stream2;
+  cudaGraph_t graph = nullptr;
+  const cudaStreamCaptureMode mode = cudaStreamCaptureModeThreadLocal;
+  const long long launches0 = g_launches.load();
+  long long n_body = 0;
+  CU_TRY(cudaStreamBeginCapture(cs, mode));
+  int rc = TSFM_OK;
+  auto step = [&](cudaError_t e, const char *what) {
+    if (rc == TSFM_OK && e != cudaSuccess) {
+      g_cuda_err = std::string(what) + ": " + cudaGetErrorString(e);
+      rc = TSFM_ERR_CUDA;
+    }
+    return rc == TSFM_OK;
+  };
+  h->ls = cs;
+  if (k.mode == 1) {
+    enqueue_target_only(h, k.B, k.N, T, k.H);
+  } else {
+    enqueue_spec_prologue(h, k.B, k.N, T, k.K);
+    cudaStreamCaptureStatus status;
+    cudaGraph_t g = nullptr;
+    const cudaGraphNode_t *deps = nullptr;
+    size_t ndeps = 0;
+    cudaGraphConditionalHandle handle{};
+    cudaGraphNode_t node = nullptr;
+    cudaGraphNodeParams np{};
+    np.type = cudaGraphNodeTypeConditional;
+    if (step(cudaStreamGetCaptureInfo(cs, &status, nullptr, &g, &deps, &ndeps), "cudaStreamGetCaptureInfo") &&
+        step(cudaGraphConditionalHandleCreate(&handle, g, 1, cudaGraphCondAssignDefault),
+             "cudaGraphConditionalHandleCreate")) {
+      np.conditional.handle = handle;
+      np.conditional.type = cudaGraphCondTypeWhile;
+      np.conditional.size = 1;
+      if (step(cudaGraphAddNode(&node, g, deps, ndeps, &np), "cudaGraphAddNode(conditional)") &&
+          step(cudaStreamUpdateCaptureDependencies(cs, &node, 1, cudaStreamSetCaptureDependencies),
+               "cudaStreamUpdateCaptureDependencies")) {
+        cudaGraph_t body = np.conditional.phGraph_out[0];
+        if (step(cudaStreamBeginCaptureToGraph(cs2, body, nullptr, nullptr, 0, mode), "cudaStreamBeginCaptureToGraph")) {
+          h->ls = cs2;
+          const long long before = g_launches.load();
+          enqueue_round(h, k.B, k.N, T, k.K, handle, 1, h->dev_body_launches + slot);
+          n_body = g_launches.load() - before;
+          cudaGraph_t same = nullptr;
+          step(cudaStreamEndCapture(cs2, &same), "cudaStreamEndCapture(body)");
+          h->ls = cs;
+        }
+      }
+    }
+    if (rc == TSFM_OK) enqueue_denorm(h, k.B, k.N, k.H);
+  }
+  h->ls = h->stream;
+  step(cudaStreamEndCapture(cs, &graph), "cudaStreamEndCapture");
+  out->n_fixed = g_launches.load() - launches0 - n_body;
+  g_launches.store(launches0);                     // captured launches have not run
+  if (rc == TSFM_OK) step(cudaGetLastError(), "capture");
+  if (rc == TSFM_OK) step(cudaGraphInstantiate(&out->exec, graph, 0), "cudaGraphInstantiate");
+  if (graph) cudaGraphDestroy(graph);
+  if (rc == TSFM_OK) {
+    // the round body reports its own launch count to the device-side launch counter
+    const int nb = (int)n_body;
+    step(cudaMemcpyAsync(h->dev_body_launches + slot, &nb, sizeof(int), cudaMemcpyHostToDevice, h->stream),
+         "cudaMemcpyAsync(body launches)");
+  }
+  return rc;
+}
+
+int get_graph(tsfm_spec *h, const GraphKey &k, GraphInfo *info) {
+  auto it = h->graphs.find(k);
+  if (it != h->graphs.end()) { *info = it->second; return TSFM_OK; }
+  if ((int)h->graphs.size() >= kMaxGraphs) {       // bounded cache: drop everything and start over
+    CU_TRY(cudaStreamSynchronize(h->stream));
+    for (auto &kv : h->graphs) cudaGraphExecDestroy(kv.second.exec);
+    h->graphs.clear();
+  }
+  GraphInfo gi;
+  if (int rc = capture_graph(h, k, (int)h->graphs.size(), &gi)) {
+    if (gi.exec) cudaGraphExecDestroy(gi.exec);
+    return rc;
+  }
+  h->graphs[k] = gi;
+  *info = gi;
   return TSFM_OK;
 }
 
-int finish_call(tsfm_spec *h) {
-  CU_TRY(cudaGetLastError());
+// Writes the call parameters and clears the loop state.  The source is an ordinary host
+// struct: for pageable memory the copy is staged before the call returns.
+int write_call_state(tsfm_spec *h, const float *series, float *out, float tau, uint64_t seed) {
+  DevState st{};
+  st.series = series;
+  st.out = out;
+  st.tau = tau;
+  st.key0 = (uint32_t)(seed & 0xffffffffu);
+  st.key1 = (uint32_t)(seed >> 32);
+  CU_TRY(cudaMemcpyAsync(h->st, &st, sizeof(st), cudaMemcpyHostToDevice, h->stream));
   return TSFM_OK;
 }
 
-int read_status(tsfm_spec *h, int *status) {
-  CU_TRY(cudaMemcpyAsync(status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
-  CU_TRY(cudaStreamSynchronize(h->stream));
+// Launches made so far by this handle's replayed round bodies (waits for its stream).
+long long device_launches(tsfm_spec *h) {
+  unsigned long long v = 0;
+  if (!h->dev_launches) return 0;
+  if (cudaMemcpyAsync(&v, h->dev_launches, sizeof(v), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+      cudaStreamSynchronize(h->stream) != cudaSuccess)
+    return 0;
+  return (long long)v;
+}
+
+bool use_graph(const tsfm_spec *h) { return h->cfg.exec_mode == TSFM_EXEC_GRAPH && !h->profiling; }
+
+// Reads status and phase clocks back (synchronises) and fills ms_total.
+int finish_stats(tsfm_spec *h, tsfm_stats *stats, DevState *st_out) {
+  cudaStream_t s = h->stream;
+  CU_TRY(cudaEventRecord(h->ev[1], s));
+  CU_TRY(cudaMemcpyAsync(st_out, h->st, sizeof(DevState), cudaMemcpyDeviceToHost, s));
+  CU_TRY(cudaMemcpyAsync(&stats->device_status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CU_TRY(cudaStreamSynchronize(s));
+  CU_TRY(cudaEventElapsedTime(&stats->ms_total, h->ev[0], h->ev[1]));
   return TSFM_OK;
 }
 
@@ -421,6 +635,18 @@ size_t tsfm_weights_offset(const tsfm_arch *arch, int32_t patch_len, int32_t dty
 int tsfm_spec_destroy(tsfm_spec *h) {
   if (!h) return TSFM_ERR_ARG;
   cudaStreamSynchronize(h->stream);
+  {
+    std::lock_guard<std::mutex> lock(g_handles_mu);
+    for (size_t i = 0; i < g_handles.size(); ++i)
+      if (g_handles[i] == h) {
+        g_launches.fetch_add(device_launches(h));      // keep what its replayed rounds launched
+        g_handles.erase(g_handles.begin() + i);
+        break;
+      }
+  }
+  for (auto &kv : h->graphs) cudaGraphExecDestroy(kv.second.exec);
+  if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
+  if (h->cap_stream2) cudaStreamDestroy(h->cap_stream2);
   for (cudaEvent_t e : h->prof_pool) cudaEventDestroy(e);
   for (void *p : h->owned) cudaFree(p);
   if (h->h_unfinished) cudaFreeHost(h->h_unfinished);
@@ -435,6 +661,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   *out_h = nullptr;
   const int P = cfg->patch_len;
   if (cfg->dtype != TSFM_F32 && cfg->dtype != TSFM_BF16) return TSFM_ERR_ARG;
+  if (cfg->exec_mode != TSFM_EXEC_GRAPH && cfg->exec_mode != TSFM_EXEC_STREAM) return TSFM_ERR_ARG;
   if (cfg->draft_mode != TSFM_DRAFT_SEPARATE && cfg->draft_mode != TSFM_DRAFT_LAYER_SKIP) return TSFM_ERR_ARG;
   if (cfg->max_batch < 1 || cfg->max_ctx_tokens < 2 || cfg->max_horizon_patches < 1 || cfg->max_K < 1 ||
       cfg->max_K > TSFM_MAX_K)
@@ -458,7 +685,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   tsfm_spec *h = new (std::nothrow) tsfm_spec();
   if (!h) return TSFM_ERR_INTERNAL;
   h->cfg = *cfg;
-  h->stream = (cudaStream_t)cfg->stream;
+  h->stream = h->ls = (cudaStream_t)cfg->stream;
   h->cap = cfg->max_ctx_tokens + cfg->max_horizon_patches + cfg->max_K + 1;
   h->use_tc = cfg->dtype == TSFM_BF16 && cfg->gemm_backend == TSFM_GEMM_AUTO;
   int rc = TSFM_OK;
@@ -503,6 +730,15 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   if ((rc = dev_alloc(h, &h->ctr, 1))) return fail(rc);
   if ((rc = dev_alloc(h, &h->unfinished, cfg->max_horizon_patches + 1))) return fail(rc);
   if ((rc = dev_alloc(h, &h->dev_status, 1))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->st, 1))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->dev_launches, 1))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->dev_body_launches, kMaxGraphs))) return fail(rc);
+  if (cudaMemsetAsync(h->st, 0, sizeof(DevState), h->stream) != cudaSuccess ||
+      cudaMemsetAsync(h->dev_launches, 0, sizeof(unsigned long long), h->stream) != cudaSuccess)
+    return fail(TSFM_ERR_CUDA);
+  if (cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&h->cap_stream2, cudaStreamNonBlocking) != cudaSuccess)
+    return fail(TSFM_ERR_CUDA);
   const size_t tr = (size_t)cfg->max_horizon_patches * Bm;
   if ((rc = dev_alloc(h, &h->tr_nacc, tr))) return fail(rc);
   if ((rc = dev_alloc(h, &h->tr_ell, tr * cfg->max_K))) return fail(rc);
@@ -528,6 +764,10 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
     }
   }
   if (cudaStreamSynchronize(h->stream) != cudaSuccess) return fail(TSFM_ERR_CUDA);
+  {
+    std::lock_guard<std::mutex> lock(g_handles_mu);
+    g_handles.push_back(h);
+  }
   *out_h = h;
   return TSFM_OK;
 }
@@ -538,24 +778,23 @@ int tsfm_target_only_forecast(tsfm_spec *h, const float *series, int32_t B, int3
   const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
   cudaStream_t s = h->stream;
   if (stats) CU_TRY(cudaEventRecord(h->ev[0], s));
-  if (int rc = begin_forecast(h, series, B, ctx_len)) return rc;
-  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
-  if (stats) CU_TRY(cudaEventRecord(h->ev[2], s));
-  for (int t = 0; t < T; ++t)       // Eq. 1: one target pass per committed patch
-    pass(h, h->tgt, B, PassGeom{nullptr, N - 1 + t, 1, h->cap}, HEAD_LAST_TO_HIST);
-  {
-    KTimer kt(h, KC_DENORM, 8.0 * B * H, 2.0 * B * H);
-    denorm_kernel<<<B, 256, 0, s>>>(h->hist, N, P, h->cap, H, h->mean, h->sd, out);
-    LAUNCHED();
+  if (int rc = write_call_state(h, series, out, 1.f, 0)) return rc;
+  if (use_graph(h)) {
+    GraphInfo gi;
+    if (int rc = get_graph(h, GraphKey{1, B, N, H, 0}, &gi)) return rc;
+    CU_TRY(cudaGraphLaunch(gi.exec, s));
+    g_launches.fetch_add(gi.n_fixed, std::memory_order_relaxed);
+  } else {
+    h->ls = s;
+    enqueue_target_only(h, B, N, T, H);
   }
-  if (int rc = finish_call(h)) return rc;
+  CU_TRY(cudaGetLastError());
   if (stats) {
-    CU_TRY(cudaEventRecord(h->ev[1], s));
     std::memset(stats, 0, sizeof(*stats));
-    if (int rc = read_status(h, &stats->device_status)) return rc;
-    CU_TRY(cudaEventElapsedTime(&stats->ms_total, h->ev[0], h->ev[1]));
-    CU_TRY(cudaEventElapsedTime(&stats->ms_prefill, h->ev[0], h->ev[2]));
-    CU_TRY(cudaEventElapsedTime(&stats->ms_verify, h->ev[2], h->ev[1]));
+    DevState st;
+    if (int rc = finish_stats(h, stats, &st)) return rc;
+    stats->ms_prefill = (float)((st.t_phase[0] - st.t_call) * 1e-6);
+    stats->ms_verify = (float)((st.t_end - st.t_phase[0]) * 1e-6);
     stats->rounds = T;
     stats->patches_committed = (int64_t)B * T;
     if (stats->device_status) return TSFM_ERR_TIMEOUT;
@@ -570,78 +809,34 @@ int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx
   if (int rc = check_call(h, series, B, ctx_len, H, out, K)) return rc;
   const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
   cudaStream_t s = h->stream;
-  const bool timed = stats != nullptr;
-  if (timed) CU_TRY(cudaEventRecord(h->ev[0], s));
-  if (int rc = begin_forecast(h, series, B, ctx_len)) return rc;
-  CU_TRY(cudaMemsetAsync(h->ctr, 0, sizeof(AcceptCounters), s));
-  CU_TRY(cudaMemsetAsync(h->unfinished, 0, sizeof(int) * (T + 1), s));
-  CU_TRY(cudaMemsetAsync(h->tr_nacc, 0xff, sizeof(int) * (size_t)T * B, s));
-  CU_TRY(cudaMemsetAsync(h->tr_ell, 0, sizeof(float) * (size_t)T * B * K, s));
-  CU_TRY(cudaMemsetAsync(h->tr_logu, 0, sizeof(float) * (size_t)T * B * K, s));
-  // both caches ingest the context except its last patch (target) / last two (draft)
-  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
-  pass(h, h->drf, B, PassGeom{nullptr, 0, N - 2, h->cap}, HEAD_NONE);
-  if (timed) CU_TRY(cudaEventRecord(h->ev[2], s));
-
-  AcceptArgs a{};
-  a.x = a.mu_q = h->hist + (size_t)N * P;       // slot N + done[b] holds x_1
-  a.x_stride_b = (long long)h->cap * P;
-  a.mu_p = h->vout;
-  a.commit = h->hist + (size_t)N * P;
-  a.commit_stride_b = a.x_stride_b;
-  a.commit_accepted = 0;
-  a.commit_follows_done = 1;
-  a.done = h->done;
-  a.B = B; a.K = K; a.P = P; a.T = T;
-  a.sigma_p = a.sigma_q = tau;
-  a.margin = h->cfg.dtype == TSFM_BF16 ? 5e-2f : 1e-3f;
-  a.key = make_uint2((uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32));
-  a.series0 = 0;
-  a.forced_u = nullptr;
-  a.ctr = h->ctr;
-
-  int rounds = 0;
-  for (int r = 0; r < T; ++r) {
-    size_t e0 = 3 + 4 * (size_t)r;
-    // draft rollout: step 1 re-ingests the last two committed patches (the draft cache may
-    // lack the last accepted proposal), steps 2..K ingest the previous proposal
-    pass(h, h->drf, B, PassGeom{h->done, N - 2, 2, h->cap}, HEAD_LAST_TO_HIST);
-    for (int i = 2; i <= K; ++i)
-      pass(h, h->drf, B, PassGeom{h->done, N - 1 + (i - 1), 1, h->cap}, HEAD_LAST_TO_HIST);
-    if (timed) CU_TRY(cudaEventRecord(h->ev[e0], s));
-    // single-pass verification over [pending, x_1..x_K]
-    pass(h, h->tgt, B, PassGeom{h->done, N - 1, K + 1, h->cap}, HEAD_ALL_TO_VOUT, h->vout);
-    if (timed) CU_TRY(cudaEventRecord(h->ev[e0 + 1], s));
-    a.round_idx = r;
-    a.n_accept = h->tr_nacc + (size_t)r * B;
-    a.ell = h->tr_ell + (size_t)r * B * K;
-    a.log_u = h->tr_logu + (size_t)r * B * K;
-    a.unfinished = h->unfinished + r;
-    {
-      KTimer kt(h, KC_ACCEPT, (double)B * (2 * K + 2) * P * 4, 4.0 * B * K * P);
-      accept_kernel<<<(B + 3) / 4, 128, 0, s>>>(a);
-      LAUNCHED();
+  if (stats) CU_TRY(cudaEventRecord(h->ev[0], s));
+  if (int rc = write_call_state(h, series, out, tau, seed)) return rc;
+  if (use_graph(h)) {
+    // one launch: prologue, WHILE(rounds), de-normalisation; no host round trip
+    GraphInfo gi;
+    if (int rc = get_graph(h, GraphKey{0, B, N, H, K}, &gi)) return rc;
+    CU_TRY(cudaGraphLaunch(gi.exec, s));
+    g_launches.fetch_add(gi.n_fixed, std::memory_order_relaxed);   // the rounds count themselves on the device
+  } else {
+    h->ls = s;
+    enqueue_spec_prologue(h, B, N, T, K);
+    for (int r = 0; r < T; ++r) {
+      enqueue_round(h, B, N, T, K, cudaGraphConditionalHandle{}, 0);
+      CU_TRY(cudaMemcpyAsync(h->h_unfinished, h->unfinished + r, sizeof(int), cudaMemcpyDeviceToHost, s));
+      CU_TRY(cudaStreamSynchronize(s));
+      if (*h->h_unfinished == 0) break;
     }
-    if (timed) CU_TRY(cudaEventRecord(h->ev[e0 + 2], s));
-    ++rounds;
-    CU_TRY(cudaMemcpyAsync(h->h_unfinished, h->unfinished + r, sizeof(int), cudaMemcpyDeviceToHost, s));
-    CU_TRY(cudaStreamSynchronize(s));
-    if (*h->h_unfinished == 0) break;
+    enqueue_denorm(h, B, N, H);
   }
-  {
-    KTimer kt(h, KC_DENORM, 8.0 * B * H, 2.0 * B * H);
-    denorm_kernel<<<B, 256, 0, s>>>(h->hist, N, P, h->cap, H, h->mean, h->sd, out);
-    LAUNCHED();
-  }
-  h->last_B = B; h->last_K = K; h->last_rounds = rounds;
-  if (int rc = finish_call(h)) return rc;
+  h->last_B = B; h->last_K = K;
+  CU_TRY(cudaGetLastError());
   if (stats) {
-    CU_TRY(cudaEventRecord(h->ev[1], s));
     std::memset(stats, 0, sizeof(*stats));
     AcceptCounters c;
+    DevState st;
     CU_TRY(cudaMemcpyAsync(&c, h->ctr, sizeof(c), cudaMemcpyDeviceToHost, s));
-    if (int rc = read_status(h, &stats->device_status)) return rc;
-    stats->rounds = rounds;
+    if (int rc = finish_stats(h, stats, &st)) return rc;
+    stats->rounds = st.round;
     stats->proposals_drafted = (int64_t)c.drafted;
     stats->proposals_tested = (int64_t)c.tested;
     stats->proposals_accepted = (int64_t)c.accepted;
@@ -652,19 +847,10 @@ int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx
       stats->accepted_by_pos[i] = (int64_t)c.accepted_by_pos[i];
     }
     for (int i = 0; i < TSFM_MAX_K + 2; ++i) stats->L_hist[i] = (int64_t)c.L_hist[i];
-    CU_TRY(cudaEventElapsedTime(&stats->ms_total, h->ev[0], h->ev[1]));
-    CU_TRY(cudaEventElapsedTime(&stats->ms_prefill, h->ev[0], h->ev[2]));
-    float ms = 0.f;
-    for (int r = 0; r < rounds; ++r) {
-      size_t e0 = 3 + 4 * (size_t)r;
-      cudaEvent_t start = r == 0 ? h->ev[2] : h->ev[e0 - 4 + 2];
-      CU_TRY(cudaEventElapsedTime(&ms, start, h->ev[e0]));
-      stats->ms_draft += ms;
-      CU_TRY(cudaEventElapsedTime(&ms, h->ev[e0], h->ev[e0 + 1]));
-      stats->ms_verify += ms;
-      CU_TRY(cudaEventElapsedTime(&ms, h->ev[e0 + 1], h->ev[e0 + 2]));
-      stats->ms_accept += ms;
-    }
+    stats->ms_prefill = (float)(st.ns_prefill * 1e-6);
+    stats->ms_draft = (float)(st.ns_draft * 1e-6);
+    stats->ms_verify = (float)(st.ns_verify * 1e-6);
+    stats->ms_accept = (float)(st.ns_accept * 1e-6);
     if (stats->device_status) return TSFM_ERR_TIMEOUT;
   }
   return TSFM_OK;
@@ -694,10 +880,13 @@ int tsfm_target_only_forecast_host(tsfm_spec *h, const float *series, int32_t B,
 int tsfm_spec_last_trace(tsfm_spec *h, int32_t cap_rounds, int32_t *rounds, int32_t *n_accept, float *ell,
                          float *log_u) {
   if (!h || !rounds) return TSFM_ERR_ARG;
-  *rounds = h->last_rounds;
-  if (cap_rounds < h->last_rounds) return TSFM_ERR_ARG;
-  const size_t nb = (size_t)h->last_rounds * h->last_B, nk = nb * h->last_K;
   cudaStream_t s = h->stream;
+  int R = 0;
+  CU_TRY(cudaMemcpyAsync(&R, &h->st->round, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CU_TRY(cudaStreamSynchronize(s));
+  *rounds = R;
+  if (cap_rounds < R) return TSFM_ERR_ARG;
+  const size_t nb = (size_t)R * h->last_B, nk = nb * h->last_K;
   if (n_accept && nb) CU_TRY(cudaMemcpyAsync(n_accept, h->tr_nacc, nb * sizeof(int), cudaMemcpyDeviceToHost, s));
   if (ell && nk) CU_TRY(cudaMemcpyAsync(ell, h->tr_ell, nk * sizeof(float), cudaMemcpyDeviceToHost, s));
   if (log_u && nk) CU_TRY(cudaMemcpyAsync(log_u, h->tr_logu, nk * sizeof(float), cudaMemcpyDeviceToHost, s));
@@ -739,10 +928,12 @@ int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t
   CU_TRY(cudaMemcpy2DAsync(h->hist, (size_t)h->cap * P * sizeof(float), tokens, (size_t)n * P * sizeof(float),
                            (size_t)n * P * sizeof(float), B, cudaMemcpyDeviceToDevice, h->stream));
   CU_TRY(cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream));
+  h->ls = h->stream;
   pass(h, which == 0 ? h->tgt : h->drf, B, PassGeom{nullptr, 0, n, h->cap}, HEAD_ALL_TO_VOUT, out);
-  if (int rc = finish_call(h)) return rc;
+  CU_TRY(cudaGetLastError());
   int status = 0;
-  if (int rc = read_status(h, &status)) return rc;
+  CU_TRY(cudaMemcpyAsync(&status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  CU_TRY(cudaStreamSynchronize(h->stream));
   return status ? TSFM_ERR_TIMEOUT : TSFM_OK;
 }
 
@@ -871,7 +1062,12 @@ int tsfm_spec_kernel_profile(tsfm_spec *h, int32_t cap, int32_t *n, tsfm_kernel_
   return k <= cap ? TSFM_OK : TSFM_ERR_ARG;
 }
 
-int64_t tsfm_launch_count(void) { return g_launches.load(); }
+int64_t tsfm_launch_count(void) {
+  long long n = g_launches.load();
+  std::lock_guard<std::mutex> lock(g_handles_mu);
+  for (tsfm_spec *h : g_handles) n += device_launches(h);
+  return n;
+}
 
 const char *tsfm_strerror(int code) {
   switch (code) {

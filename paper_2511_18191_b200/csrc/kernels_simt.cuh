@@ -26,13 +26,14 @@ __device__ __forceinline__ int pos0_of(const PassGeom &g, int b) {
 // grid = B, block = 256.  hist[b, t, :] = (series - mean) / sd for the N context
 // patches; the remaining slots are zeroed.  Sums in fp64 (8 K values, one pass each).
 // ----------------------------------------------------------------------------------
-__global__ void instnorm_kernel(const float *__restrict__ series, int ctx_len, int P, int cap,
+__global__ void instnorm_kernel(DevState *__restrict__ st, int ctx_len, int P, int cap,
                                 float norm_eps, float *__restrict__ hist,
                                 float *__restrict__ mean_out, float *__restrict__ sd_out,
                                 int *__restrict__ done) {
   __shared__ double red[32];
   const int b = blockIdx.x;
-  const float *s = series + (size_t)b * ctx_len;
+  if (b == 0 && threadIdx.x == 0) st->t_call = globaltimer_ns();
+  const float *s = st->series + (size_t)b * ctx_len;
   double acc = 0.0;
   for (int i = threadIdx.x; i < ctx_len; i += blockDim.x) acc += (double)s[i];
   const double mean = block_sum_d(acc, red) / ctx_len;
@@ -56,8 +57,10 @@ __global__ void instnorm_kernel(const float *__restrict__ series, int ctx_len, i
 // out[b, s] = hist[b, N + s / P, s % P] * sd + mean, s < H.   grid = B.
 __global__ void denorm_kernel(const float *__restrict__ hist, int N, int P, int cap, int H,
                               const float *__restrict__ mean, const float *__restrict__ sd,
-                              float *__restrict__ out) {
+                              DevState *__restrict__ st) {
   const int b = blockIdx.x;
+  float *out = st->out;
+  if (b == 0 && threadIdx.x == 0) st->t_end = globaltimer_ns();
   const float m = mean[b], s = sd[b];
   const float *hb = hist + ((size_t)b * cap + N) * P;
   for (int i = threadIdx.x; i < H; i += blockDim.x) out[(size_t)b * H + i] = hb[i] * s + m;
@@ -93,9 +96,10 @@ template <> struct Vec16<bf16> {
 template <typename T>
 __global__ void __launch_bounds__(128)
 embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *__restrict__ W,
-             float *__restrict__ x) {
+             float *__restrict__ x, unsigned long long *__restrict__ stamp) {
   extern __shared__ float zs[];
   const int row = blockIdx.x, b = row / g.q_len, j = row % g.q_len;
+  if (stamp && row == 0 && blockIdx.y == 0 && threadIdx.x == 0) *stamp = globaltimer_ns();
   const float *z = hist + ((size_t)b * g.cap + pos0_of(g, b) + j) * P;
   for (int i = threadIdx.x; i < P; i += blockDim.x) zs[i] = z[i];
   __syncthreads();

@@ -8,9 +8,10 @@ import paper_2511_18191_b200 as tsfm
 from tsfm_inputs import build_models, make_series
 
 
-def make_decoder(wl, backend=tsfm.TSFM_GEMM_AUTO, max_K=None, batch=None):
+def make_decoder(wl, backend=tsfm.TSFM_GEMM_AUTO, max_K=None, batch=None, exec_mode=tsfm.TSFM_EXEC_GRAPH):
     tw, dw = build_models(wl)
-    dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=max_K, batch=batch, gemm_backend=backend)
+    dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=max_K, batch=batch, gemm_backend=backend,
+                                        exec_mode=exec_mode)
     return dec, tw, dw
 
 

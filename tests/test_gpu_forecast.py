@@ -31,10 +31,10 @@ def check_stats(st, B, T, K):
     return d
 
 
-def run_and_compare(wl, K, tau, seed, ids, backend=0, batch=None, H=None):
+def run_and_compare(wl, K, tau, seed, ids, backend=0, batch=None, H=None, exec_mode=0):
     H = H or wl.horizon
     B = batch or wl.batch
-    dec, tw, dw = make_decoder(wl, backend=backend, max_K=max(K, wl.K), batch=B)
+    dec, tw, dw = make_decoder(wl, backend=backend, max_K=max(K, wl.K), batch=B, exec_mode=exec_mode)
     s, ctx = series_on_device(wl, B)
     out, st = dec.forecast(ctx, H, K, tau, seed)
     T = -(-H // wl.patch_len)
@@ -57,23 +57,70 @@ def run_and_compare(wl, K, tau, seed, ids, backend=0, batch=None, H=None):
     return res
 
 
-def test_c0_full():
+EXEC = pytest.mark.parametrize("exec_mode", [1, 0], ids=["stream", "graph"])
+
+
+@EXEC
+def test_c0_full(exec_mode):
     wl = workload("C0")
-    run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, range(wl.batch))
+    run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, range(wl.batch), exec_mode=exec_mode)
 
 
+@EXEC
 @pytest.mark.parametrize("K,tau,H", [(1, 1.0, 384), (3, 2.0, 400), (4, 4.0, 96 * 7 + 5)])
-def test_c0_shape_ragged_batch_fp32(K, tau, H):
+def test_c0_shape_ragged_batch_fp32(K, tau, H, exec_mode):
     """C0's models on a ragged batch: several series, acceptance in the middle range, truncated last patch."""
     wl = workload("C0", batch=6, series_recipe="c1", horizon=H)
-    run_and_compare(wl, K, tau, 7, range(6))
+    run_and_compare(wl, K, tau, 7, range(6), exec_mode=exec_mode)
 
 
-@pytest.mark.parametrize("backend", [1, 0], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("backend,exec_mode", [(1, 1), (0, 1), (0, 0)], ids=["simt-stream", "tcgen05-stream", "tcgen05-graph"])
 @pytest.mark.parametrize("tau", [0.5, 1.0, 2.0])
-def test_c1_full(tau, backend):
+def test_c1_full(tau, backend, exec_mode):
     wl = workload("C1")
-    run_and_compare(wl, wl.K, tau, wl.forecast_seed, range(wl.batch), backend=backend)
+    run_and_compare(wl, wl.K, tau, wl.forecast_seed, range(wl.batch), backend=backend, exec_mode=exec_mode)
+
+
+def test_graph_and_stream_execution_give_identical_forecasts_and_traces():
+    """The captured graph (device-side WHILE over rounds) replays exactly what the stream path
+    launches: same kernels, same arguments -- so forecasts, decisions and counters are identical,
+    also when one handle replays its graph with other seeds, temperatures and block sizes."""
+    wl = workload("C0", batch=5, series_recipe="c1")          # fp32 path: bit-reproducible
+    s, ctx = series_on_device(wl)
+    decs = [make_decoder(wl, max_K=4, exec_mode=m)[0] for m in (1, 0)]
+    for K, tau, seed in [(2, 1.0, 3), (2, 2.5, 4), (4, 2.5, 4), (1, 0.7, 9), (2, 1.0, 3)]:
+        res = []
+        for dec in decs:
+            out, st = dec.forecast(ctx, wl.horizon, K, tau, seed)
+            nacc, ell, logu = dec.last_trace(wl.batch, K)
+            d = st.as_dict()
+            res.append((out.cpu().numpy(), nacc, ell, logu,
+                        {k: d[k] for k in ("rounds", "proposals_tested", "proposals_accepted", "L_hist")}))
+        for a, b in zip(res[0][:4], res[1][:4]):
+            np.testing.assert_array_equal(a, b)
+        assert res[0][4] == res[1][4]
+        assert res[1][4]["rounds"] == res[1][1].shape[0]
+    ref = [dec.target_only(ctx, wl.horizon)[0].cpu().numpy() for dec in decs]
+    np.testing.assert_array_equal(ref[0], ref[1])
+    for dec in decs:
+        dec.close()
+
+
+def test_launch_counter_counts_replayed_rounds():
+    import paper_2511_18191_b200 as tsfm
+    wl = workload("C0", batch=3, series_recipe="c1")
+    s, ctx = series_on_device(wl)
+    counts = []
+    for mode in (1, 0):
+        dec, _, _ = make_decoder(wl, exec_mode=mode)
+        dec.forecast(ctx, wl.horizon, wl.K, 2.0, 1)            # warm-up (captures the graph in graph mode)
+        n0 = tsfm.tsfm_launch_count()
+        dec.forecast(ctx, wl.horizon, wl.K, 2.0, 1, stats=False)
+        dec.target_only(ctx, wl.horizon, stats=False)
+        counts.append(tsfm.tsfm_launch_count() - n0)
+        dec.close()
+        assert tsfm.tsfm_launch_count() - n0 == counts[-1]      # survives the handle
+    assert counts[0] == counts[1] and counts[0] > 0
 
 
 def test_c2_subset():
