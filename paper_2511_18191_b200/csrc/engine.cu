@@ -19,6 +19,7 @@
 #include "kernels_simt.cuh"
 #include "accept.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_sk.cuh"
 
 using namespace tsfm;
 
@@ -88,7 +89,7 @@ BlobLayout blob_layout(const tsfm_arch &a, int P, int dtype) {
 struct LayerDev {
   const float *g1, *g2;
   const void *Wqkv, *Wo, *W1, *W2;
-  GemmTcPlan tc_qkv, tc_o, tc_1, tc_2;
+  GemmSkPlan tc_qkv, tc_o, tc_1, tc_2;
 };
 
 struct ModelDev {
@@ -265,6 +266,34 @@ int attn_prepare(int dh, int cap) {
   return attn_set_attr<T, 128>(optin);
 }
 
+// Every kernel of the library asks for the same (maximum) shared-memory carve-out, so that the
+// SMs never have to re-partition L1 / shared memory between two consecutive launches of a pass.
+template <typename F> void prefer_max_smem(F *fn) {
+  cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+}
+template <typename T> void prefer_max_smem_typed() {
+  prefer_max_smem(embed_kernel<T>);
+  prefer_max_smem(rmsnorm_kernel<T>);
+  prefer_max_smem(head_kernel<T>);
+  prefer_max_smem(gemm_simt_kernel<T, EPI_F32>);
+  prefer_max_smem(gemm_simt_kernel<T, EPI_T>);
+  prefer_max_smem(gemm_simt_kernel<T, EPI_GELU_T>);
+  prefer_max_smem(gemm_simt_kernel<T, EPI_RESID>);
+  prefer_max_smem(attn_kernel<T, 32>);
+  prefer_max_smem(attn_kernel<T, 64>);
+  prefer_max_smem(attn_kernel<T, 128>);
+}
+void prefer_max_smem_all() {
+  prefer_max_smem_typed<float>();
+  prefer_max_smem_typed<bf16>();
+  prefer_max_smem(instnorm_kernel);
+  prefer_max_smem(denorm_kernel);
+  prefer_max_smem(accept_kernel);
+  prefer_max_smem(round_end_kernel);
+  prefer_max_smem(gemm_sk_kernel);
+  cudaGetLastError();
+}
+
 template <typename T>
 void launch_gemm_simt(cudaStream_t s, const T *A, const T *W, void *C, int M, int N, int K, int epi) {
   dim3 grid((N + 63) / 64, (M + 63) / 64), block(256);
@@ -279,7 +308,7 @@ void launch_gemm_simt(cudaStream_t s, const T *A, const T *W, void *C, int M, in
 
 // C (op)= A . W^T through the tensor-core kernel when a plan exists, else the FMA kernel.
 template <typename T>
-void gemm(tsfm_spec *h, const GemmTcPlan *plan, const void *A, const void *W, void *C, int M, int N,
+void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C, int M, int N,
           int K, int epi) {
   const double e = sizeof(T);
   const double out_b = (epi == EPI_F32 || epi == EPI_ATOMIC) ? 4.0 : epi == EPI_RESID ? 8.0 : e;
@@ -287,7 +316,7 @@ void gemm(tsfm_spec *h, const GemmTcPlan *plan, const void *A, const void *W, vo
   const double flops = 2.0 * M * N * K;
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
     KTimer kt(h, KC_GEMM_TC, bytes, flops);
-    if (gemm_tc_launch(h->ls, *plan, A, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
+    if (gemm_sk_launch(h->ls, *plan, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
   }
   KTimer kt(h, KC_GEMM_SIMT, bytes, flops);
   launch_gemm_simt<T>(h->ls, (const T *)A, (const T *)W, C, M, N, K, epi);
@@ -327,18 +356,14 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   }
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
   const int L = m.arch.n_layers;
-  // The QKV contraction is split along K (atomic accumulation) when its grid would be small;
-  // the preceding RMSNorm kernel then clears the accumulator.
-  const bool qkv_split = sizeof(T) == 2 && h->use_tc && gemm_tc_splits(3 * d, d, M, true) > 1;
-  float *qkv_zero = qkv_split ? h->qkv : nullptr;
   for (int l = 0; l < L; ++l) {
     LayerDev &ly = m.layers[l];
     {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g1, d, eps, (T *)h->a, qkv_zero, 3 * d);
+      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g1, d, eps, (T *)h->a, nullptr, 0);
       LAUNCHED();
     }
-    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, qkv_split ? EPI_ATOMIC : EPI_F32);
+    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
     else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
     else launch_attn<T, 128>(h, m, l, B, g);
@@ -751,15 +776,16 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
     if (cudaEventCreate(&ev) != cudaSuccess) { ev = nullptr; return fail(TSFM_ERR_CUDA); }
   if (cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream) != cudaSuccess) return fail(TSFM_ERR_CUDA);
 
+  prefer_max_smem_all();
   if (h->use_tc) {
-    if ((rc = gemm_tc_init())) return fail(rc);
+    if ((rc = gemm_sk_init())) return fail(rc);
     for (ModelDev *m : {&h->tgt, &h->drf}) {
       const int d = m->arch.d_model, f = m->arch.d_ff;
       for (LayerDev &ly : m->layers) {
-        if ((rc = gemm_tc_plan(&ly.tc_qkv, ly.Wqkv, 3 * d, d, h->a, h->M_max))) return fail(rc);
-        if ((rc = gemm_tc_plan(&ly.tc_o, ly.Wo, d, d, h->ao, h->M_max))) return fail(rc);
-        if ((rc = gemm_tc_plan(&ly.tc_1, ly.W1, f, d, h->a, h->M_max))) return fail(rc);
-        if ((rc = gemm_tc_plan(&ly.tc_2, ly.W2, d, f, h->hbuf, h->M_max))) return fail(rc);
+        if ((rc = gemm_sk_plan(&ly.tc_qkv, ly.Wqkv, 3 * d, d, h->a, h->M_max))) return fail(rc);
+        if ((rc = gemm_sk_plan(&ly.tc_o, ly.Wo, d, d, h->ao, h->M_max))) return fail(rc);
+        if ((rc = gemm_sk_plan(&ly.tc_1, ly.W1, f, d, h->a, h->M_max))) return fail(rc);
+        if ((rc = gemm_sk_plan(&ly.tc_2, ly.W2, d, f, h->hbuf, h->M_max))) return fail(rc);
       }
     }
   }
@@ -948,14 +974,14 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t
     return TSFM_OK;
   }
   if (Kd % 8) return TSFM_ERR_SHAPE;
-  if (int rc = gemm_tc_init()) return rc;
-  GemmTcPlan plan;
-  if (int rc = gemm_tc_plan(&plan, W, N, Kd, A, M)) return rc;
+  if (int rc = gemm_sk_init()) return rc;
+  GemmSkPlan plan;
+  if (int rc = gemm_sk_plan(&plan, W, N, Kd, A, M)) return rc;
   if (!plan.valid) return TSFM_ERR_SHAPE;
   int *status = nullptr;
   CU_TRY(cudaMalloc((void **)&status, sizeof(int)));
   CU_TRY(cudaMemsetAsync(status, 0, sizeof(int), s));
-  const bool ok = gemm_tc_launch(s, plan, A, C, M, EPI_F32, status);
+  const bool ok = gemm_sk_launch(s, plan, C, M, EPI_F32, status);
   if (ok) LAUNCHED();
   int hs = 0;
   cudaError_t e1 = cudaMemcpyAsync(&hs, status, sizeof(int), cudaMemcpyDeviceToHost, s);

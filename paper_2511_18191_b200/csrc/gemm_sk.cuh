@@ -1,0 +1,267 @@
+// bf16 x bf16 -> fp32 contraction on the sm_100a tensor cores, split along K across a
+// thread-block cluster.
+//
+//   C[t, f] (op)= sum_k A[t, k] * W[f, k]        A: [M, K] tokens, W: [N, K] weights
+//
+// Same swap-AB tiling as gemm_tc.cuh (128 weight rows = MMA M, BN tokens = MMA N, 64-wide K
+// stages fed by TMA into a 128-byte-swizzled ring, accumulator in tensor memory), with two
+// differences that matter when the token count is small and the call is latency-bound:
+//   * BN is a run-time value (any multiple of 16 up to 256), so M = 160 verification tokens
+//     are one tile, not a padded 256;
+//   * the K loop is split over the S CTAs of a cluster (grid.z = cluster.z = S <= 8).  Each CTA
+//     parks its partial tile in its own shared memory; after a cluster barrier CTA r sums rows
+//     r, r + S, ... of all S partial tiles through distributed shared memory and applies the
+//     epilogue once.  No atomics, no pre-zeroed accumulator, a fixed summation order, and every
+//     epilogue (GELU included) can be split.
+// Warp roles and bounded waits as in gemm_tc.cuh.
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace tsfm {
+
+constexpr int SK_MAX_SPLIT = 8;
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t local_addr, uint32_t rank) {
+  uint32_t remote;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+  return v;
+}
+__host__ __device__ constexpr uint32_t umma_idesc_rt(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+struct SkShape {
+  int BN, stages, tmem_cols, smem_bytes;
+};
+// Ring of `stages` x (W tile 16 KB + A tile BN x 128 B); the partial-sum tile (BN x 128 fp32)
+// reuses the ring once the accumulator is complete.
+static inline SkShape sk_shape(int BN, int kb_per_cta, bool split) {
+  SkShape s;
+  s.BN = BN;
+  const int stage = TC_W_BYTES + BN * TC_BK * 2;
+  int stages = BN > 160 ? 4 : BN > 64 ? 3 : 4;
+  if (stages > kb_per_cta) stages = kb_per_cta < 1 ? 1 : kb_per_cta;
+  int bytes = stages * stage;
+  if (split && bytes < BN * TC_BM * 4) bytes = BN * TC_BM * 4;
+  s.stages = stages;
+  s.tmem_cols = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
+  s.smem_bytes = bytes + 1024 + 256;
+  return s;
+}
+
+__device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi) {
+  if (epi == EPI_F32) ((float *)C)[o] = v;
+  else if (epi == EPI_T) ((bf16 *)C)[o] = __float2bfloat16_rn(v);
+  else if (epi == EPI_GELU_T) ((bf16 *)C)[o] = __float2bfloat16_rn(gelu_erf(v));
+  else ((float *)C)[o] += v;
+}
+
+// grid = (ceil(N / 128), ceil(M / BN), S), cluster = (1, 1, S), block = 192.
+// ring_bytes = size of the tile region (a multiple of 1024); barriers sit behind it.
+__global__ void __launch_bounds__(192, 1)
+gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
+               void *__restrict__ C, int M, int N, int K, int BN, int stages, int tmem_cols, int ring_bytes,
+               int epi, int *__restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = tiles + (uint32_t)ring_bytes;
+  const uint32_t full0 = bars, empty0 = bars + 64, accum = bars + 128, slot = bars + 136;
+  uint32_t *slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (slot - smem_u32(smem_raw)));
+  float *stage_f = reinterpret_cast<float *>(smem_raw + (tiles - smem_u32(smem_raw)));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int f0 = blockIdx.x * TC_BM, t0 = blockIdx.y * BN;
+  const int S = gridDim.z, rank = blockIdx.z;
+  const int KB_all = (K + TC_BK - 1) / TC_BK;
+  const int kb_lo = (int)(((long long)KB_all * rank) / S);
+  const int kb_hi = (int)(((long long)KB_all * (rank + 1)) / S);
+  const int KB = kb_hi - kb_lo;
+  const int a_bytes = BN * TC_BK * 2, stage_bytes = TC_W_BYTES + a_bytes;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    mbar_init(accum, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"((uint32_t)tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *slot_ptr;
+
+  if (warp == 4 && lane == 0) {
+    // ---------------- TMA producer
+    for (int kb = 0; kb < KB; ++kb) {
+      const int s = kb % stages;
+      const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+      if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { atomicExch(status, DEV_TIMEOUT_TMA); break; }
+      const uint32_t dst = tiles + s * stage_bytes;
+      mbar_expect_tx(full0 + 8 * s, (uint32_t)stage_bytes);
+      tma_load_2d(dst, &mapW, (kb_lo + kb) * TC_BK, f0, full0 + 8 * s);
+      tma_load_2d(dst + TC_W_BYTES, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * s);
+    }
+  } else if (warp == 5 && lane == 0) {
+    // ---------------- MMA issuer
+    const uint32_t idesc = umma_idesc_rt(BN);
+    bool ok = true;
+    for (int kb = 0; kb < KB && ok; ++kb) {
+      const int s = kb % stages;
+      const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+      if (!mbar_wait(full0 + 8 * s, ph)) { atomicExch(status, DEV_TIMEOUT_MMA); ok = false; break; }
+      tc_fence_after();
+      const uint32_t sw = tiles + s * stage_bytes;
+      const uint64_t dw = umma_smem_desc(sw), da = umma_smem_desc(sw + TC_W_BYTES);
+#pragma unroll
+      for (int k = 0; k < TC_BK / 16; ++k)
+        umma_bf16(tmem, dw + 2 * k, da + 2 * k, idesc, (kb | k) ? 1u : 0u);
+      umma_commit(empty0 + 8 * s);
+    }
+    if (ok) umma_commit(accum);
+  } else if (warp < 4) {
+    // ---------------- epilogue, part 1: drain the accumulator
+    if (KB > 0 && mbar_wait(accum, 0)) {
+      tc_fence_after();
+      const int fl = warp * 32 + lane, f = f0 + fl;
+      const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 16) {
+        if (t0 + c0 >= M) break;
+        float v[16];
+        tmem_ld16(tbase + c0, v);
+        if (S == 1) {
+          if (f < N) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (t0 + c0 + j < M) sk_store_rt(C, (size_t)(t0 + c0 + j) * N + f, v[j], epi);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * TC_BM + fl] = v[j];
+        }
+      }
+    } else if (KB > 0 && lane == 0) {
+      atomicExch(status, DEV_TIMEOUT_EPILOGUE);
+    }
+  }
+  __syncwarp();
+  if (S > 1) {
+    // ---------------- epilogue, part 2: reduce the S partial tiles through distributed shared memory
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp < 4) {
+      const int fl = warp * 32 + lane, f = f0 + fl;
+      uint32_t remote[SK_MAX_SPLIT];
+#pragma unroll
+      for (int r = 0; r < SK_MAX_SPLIT; ++r) {
+        uint32_t a = tiles + (uint32_t)fl * 4;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote[r]) : "r"(a), "r"((uint32_t)(r < S ? r : 0)));
+      }
+      for (int tl = rank; tl < BN; tl += S) {
+        const int t = t0 + tl;
+        if (t >= M) break;
+        float sum = 0.f;
+#pragma unroll
+        for (int r = 0; r < SK_MAX_SPLIT; ++r) {
+          if (r < S) {
+            float v;
+            asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote[r] + (uint32_t)tl * (TC_BM * 4)) : "memory");
+            sum += v;
+          }
+        }
+        if (f < N) sk_store_rt(C, (size_t)t * N + f, sum, epi);
+      }
+    }
+    cluster_sync_all();          // no CTA leaves while a peer may still read its tile
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)tmem_cols) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+struct GemmSkPlan {
+  bool valid = false;
+  int N = 0, K = 0, M_max = 0;
+  const void *A = nullptr;
+  CUtensorMap mapW;
+  CUtensorMap mapA[16];            // box (BN = 16 * (i + 1)) x 64, encoded on first use
+  bool haveA[16] = {false};
+};
+
+static int gemm_sk_init() {
+  if (int rc = gemm_tc_init()) return rc;
+  static bool done = false;
+  if (done) return 0;
+  if (cudaFuncSetAttribute(gemm_sk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    return -4;
+  done = true;
+  return 0;
+}
+
+static int gemm_sk_plan(GemmSkPlan *plan, const void *W, int N, int K, const void *A, int M_max) {
+  plan->valid = false;
+  plan->N = N; plan->K = K; plan->M_max = M_max; plan->A = A;
+  for (bool &b : plan->haveA) b = false;
+  if (K % 8 || K < 16 || N < 1 || M_max < 1) return 0;
+  if (((uintptr_t)W & 15) || ((uintptr_t)A & 15)) return 0;
+  if (!g_encode) return -4;
+  if (tc_encode(&plan->mapW, W, N, K, TC_BM)) return -4;
+  plan->valid = true;
+  return 0;
+}
+
+// Tile and split choice for M tokens: one token tile up to 256 rows (rounded up to 16), and
+// as many K splits (a power of two, at most 8, at most the number of K blocks) as it takes to
+// put the grid on most of the 148 SMs.
+static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S) {
+  int bn = M >= 256 ? 256 : ((M + 15) / 16) * 16;
+  const int tiles = ((N + TC_BM - 1) / TC_BM) * ((M + bn - 1) / bn);
+  const int KB = (K + TC_BK - 1) / TC_BK;
+  int s = 1;
+  while (s * 2 <= SK_MAX_SPLIT && s * 2 <= KB && tiles * s * 2 <= 160) s *= 2;
+  *BN = bn;
+  *S = s;
+}
+
+static bool gemm_sk_launch(cudaStream_t st, GemmSkPlan &p, void *C, int M, int epi, int *status) {
+  if (!p.valid || M < 1 || M > p.M_max) return false;
+  int BN, S;
+  gemm_sk_geometry(p.N, p.K, M, &BN, &S);
+  const int idx = BN / 16 - 1;
+  if (!p.haveA[idx]) {
+    if (tc_encode(&p.mapA[idx], p.A, p.M_max, p.K, BN)) return false;
+    p.haveA[idx] = true;
+  }
+  const int KB = (p.K + TC_BK - 1) / TC_BK;
+  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1);
+  const int ring_bytes = sh.smem_bytes - 1024 - 256;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((p.N + TC_BM - 1) / TC_BM, (M + BN - 1) / BN, S);
+  cfg.blockDim = dim3(192);
+  cfg.dynamicSmemBytes = sh.smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = S;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  int N = p.N, K = p.K, stages = sh.stages, cols = sh.tmem_cols, rb = ring_bytes;
+  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
+                            status) == cudaSuccess;
+}
+
+}  // namespace tsfm
