@@ -62,6 +62,9 @@ extern "C" {
 #define TSFM_EXEC_STREAM  1       /* kernels are launched one by one and the host checks for completion
                                    after every round (reference behaviour; also used while profiling) */
 
+#define TSFM_EXEC_NO_PDL  2       /* flag, may be OR-ed in: launch without programmatic dependent launch,
+                                   i.e. every kernel starts only after its predecessor has finished   */
+
 #define TSFM_MAX_K 32           /* hard upper bound on the block size K                             */
 
 typedef struct tsfm_spec tsfm_spec;   /* opaque decoder handle */
@@ -87,7 +90,7 @@ typedef struct {
   float   rms_eps;              /* RMSNorm epsilon (1e-6)                                        */
   float   norm_eps;             /* instance-norm variance epsilon (1e-5)                         */
   float   rope_base;            /* RoPE base (1e4)                                               */
-  int32_t exec_mode;            /* TSFM_EXEC_*                                                   */
+  int32_t exec_mode;            /* TSFM_EXEC_GRAPH or TSFM_EXEC_STREAM, optionally | TSFM_EXEC_NO_PDL */
   void   *stream;               /* cudaStream_t, borrowed for the handle's lifetime              */
 } tsfm_cfg;
 

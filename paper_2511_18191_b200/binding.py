@@ -19,7 +19,7 @@ TSFM_ERR_ARG, TSFM_ERR_SHAPE, TSFM_ERR_ARCH, TSFM_ERR_CUDA, TSFM_ERR_TIMEOUT, TS
 TSFM_F32, TSFM_BF16 = 0, 1
 TSFM_DRAFT_SEPARATE, TSFM_DRAFT_LAYER_SKIP = 0, 1
 TSFM_GEMM_AUTO, TSFM_GEMM_SIMT = 0, 1
-TSFM_EXEC_GRAPH, TSFM_EXEC_STREAM = 0, 1
+TSFM_EXEC_GRAPH, TSFM_EXEC_STREAM, TSFM_EXEC_NO_PDL = 0, 1, 2
 TSFM_MAX_K = 32
 
 EXPORTS = [

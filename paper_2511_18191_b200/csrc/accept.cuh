@@ -65,6 +65,7 @@ struct AcceptArgs {
 __global__ void round_end_kernel(DevState *st, const int *unfinished, int T,
                                  cudaGraphConditionalHandle handle, int use_handle,
                                  const int *body_launches, unsigned long long *launch_ctr) {
+  pdl_sync();
   const int r = st->round;
   const unsigned long long now = globaltimer_ns();
   if (r == 0) st->ns_prefill = st->t_phase[0] - st->t_call;
@@ -82,6 +83,7 @@ __global__ void round_end_kernel(DevState *st, const int *unfinished, int T,
 __global__ void __launch_bounds__(128) accept_kernel(AcceptArgs a) {
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
+  pdl_sync();
   if (a.st) {
     if (blockIdx.x == 0 && threadIdx.x == 0) a.st->t_phase[2] = globaltimer_ns();
     const int r = a.st->round;

@@ -127,6 +127,7 @@ struct tsfm_spec {
   DevState *st = nullptr;
   int cap = 0;
   bool use_tc = false;
+  bool pdl = false;                      // launches carry the programmatic-serialization attribute
   ModelDev tgt, drf;
   // activations (sized for M_max rows)
   int M_max = 0;
@@ -294,16 +295,34 @@ void prefer_max_smem_all() {
   cudaGetLastError();
 }
 
+// One kernel launch; with pdl the launch carries the programmatic-serialization attribute, so
+// the kernel may be scheduled while its predecessor drains (its pdl_wait() restores the order).
+template <typename... KArgs, typename... Args>
+void launch_ex(cudaStream_t s, bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+               Args &&...args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+  LAUNCHED();
+}
+
 template <typename T>
-void launch_gemm_simt(cudaStream_t s, const T *A, const T *W, void *C, int M, int N, int K, int epi) {
+void launch_gemm_simt(cudaStream_t s, bool pdl, const T *A, const T *W, void *C, int M, int N, int K, int epi) {
   dim3 grid((N + 63) / 64, (M + 63) / 64), block(256);
   switch (epi) {
-    case EPI_F32: gemm_simt_kernel<T, EPI_F32><<<grid, block, 0, s>>>(A, W, C, M, N, K); break;
-    case EPI_T: gemm_simt_kernel<T, EPI_T><<<grid, block, 0, s>>>(A, W, C, M, N, K); break;
-    case EPI_GELU_T: gemm_simt_kernel<T, EPI_GELU_T><<<grid, block, 0, s>>>(A, W, C, M, N, K); break;
-    default: gemm_simt_kernel<T, EPI_RESID><<<grid, block, 0, s>>>(A, W, C, M, N, K); break;
+    case EPI_F32: launch_ex(s, pdl, gemm_simt_kernel<T, EPI_F32>, grid, block, 0, A, W, C, M, N, K); break;
+    case EPI_T: launch_ex(s, pdl, gemm_simt_kernel<T, EPI_T>, grid, block, 0, A, W, C, M, N, K); break;
+    case EPI_GELU_T: launch_ex(s, pdl, gemm_simt_kernel<T, EPI_GELU_T>, grid, block, 0, A, W, C, M, N, K); break;
+    default: launch_ex(s, pdl, gemm_simt_kernel<T, EPI_RESID>, grid, block, 0, A, W, C, M, N, K); break;
   }
-  LAUNCHED();
 }
 
 // C (op)= A . W^T through the tensor-core kernel when a plan exists, else the FMA kernel.
@@ -316,10 +335,10 @@ void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C,
   const double flops = 2.0 * M * N * K;
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
     KTimer kt(h, KC_GEMM_TC, bytes, flops);
-    if (gemm_sk_launch(h->ls, *plan, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
+    if (gemm_sk_launch(h->ls, h->pdl, *plan, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
   }
   KTimer kt(h, KC_GEMM_SIMT, bytes, flops);
-  launch_gemm_simt<T>(h->ls, (const T *)A, (const T *)W, C, M, N, K, epi);
+  launch_gemm_simt<T>(h->ls, h->pdl, (const T *)A, (const T *)W, C, M, N, K, epi);
 }
 
 template <typename T, int DH>
@@ -335,9 +354,8 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   const double Mr = (double)B * g.q_len;
   KTimer kt(h, KC_ATTN, Mr * 3 * m.arch.d_model * 4 + kv + Mr * m.arch.d_model * (2.0 * sizeof(T) + sizeof(T)),
             4.0 * Mr * (std::max(g.base, 0) + 0.5 * g.q_len) * m.arch.d_model);
-  attn_kernel<T, DH><<<grid, 128, smem, h->ls>>>(h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
-                                                     nk_max, (T *)h->ao);
-  LAUNCHED();
+  launch_ex(h->ls, h->pdl, attn_kernel<T, DH>, grid, dim3(128), smem, h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
+            nk_max, (T *)h->ao);
 }
 
 enum { HEAD_NONE = 0, HEAD_LAST_TO_HIST = 1, HEAD_ALL_TO_VOUT = 2 };
@@ -351,8 +369,8 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   const float eps = h->cfg.rms_eps;
   {
     KTimer kt(h, KC_EMBED, (double)M * P * 4 + (double)d * P * sizeof(T) + (double)M * d * 4, 2.0 * M * P * d);
-    embed_kernel<T><<<dim3(M, (d + 127) / 128), 128, P * sizeof(float), s>>>(h->hist, g, P, d, (const T *)m.W_emb, h->x, stamp);
-    LAUNCHED();
+    launch_ex(s, h->pdl, embed_kernel<T>, dim3(M, (d + 127) / 128), dim3(128), P * sizeof(float), h->hist, g, P, d,
+              (const T *)m.W_emb, h->x, stamp);
   }
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
   const int L = m.arch.n_layers;
@@ -360,8 +378,7 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     LayerDev &ly = m.layers[l];
     {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g1, d, eps, (T *)h->a, nullptr, 0);
-      LAUNCHED();
+      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3(M), dim3(128), 0, h->x, ly.g1, d, eps, (T *)h->a, nullptr, 0);
     }
     gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
@@ -371,8 +388,7 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID);
     {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      rmsnorm_kernel<T><<<M, 128, 0, s>>>(h->x, ly.g2, d, eps, (T *)h->a, nullptr, 0);
-      LAUNCHED();
+      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3(M), dim3(128), 0, h->x, ly.g2, d, eps, (T *)h->a, nullptr, 0);
     }
     gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T);
     gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID);
@@ -381,13 +397,11 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   KTimer kt(h, head_mode == HEAD_NONE ? -1 : KC_HEAD, rows * d * 4 + (double)P * d * sizeof(T) + rows * P * 4,
             2.0 * rows * P * d);
   if (head_mode == HEAD_LAST_TO_HIST) {
-    head_kernel<T><<<dim3(B, (P + 7) / 8), 256, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 1,
-                                                     h->hist, nullptr);
-    LAUNCHED();
+    launch_ex(s, h->pdl, head_kernel<T>, dim3(B, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
+              (const T *)m.W_head, d, P, eps, g, 1, h->hist, nullptr);
   } else if (head_mode == HEAD_ALL_TO_VOUT) {
-    head_kernel<T><<<dim3(M, (P + 7) / 8), 256, d * sizeof(float), s>>>(h->x, m.g_f, (const T *)m.W_head, d, P, eps, g, 0,
-                                                     nullptr, vout);
-    LAUNCHED();
+    launch_ex(s, h->pdl, head_kernel<T>, dim3(M, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
+              (const T *)m.W_head, d, P, eps, g, 0, nullptr, vout);
   }
 }
 
@@ -419,15 +433,14 @@ void enqueue_begin(tsfm_spec *h, int B, int ctx_len) {
   const int P = h->cfg.patch_len;
   cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->ls);
   KTimer kt(h, KC_INSTNORM, (double)B * (ctx_len + (double)h->cap * P) * 4, 4.0 * B * ctx_len);
-  instnorm_kernel<<<B, 256, 0, h->ls>>>(h->st, ctx_len, P, h->cap, h->cfg.norm_eps, h->hist, h->mean, h->sd,
-                                        h->done);
-  LAUNCHED();
+  launch_ex(h->ls, h->pdl, instnorm_kernel, dim3(B), dim3(256), 0, h->st, ctx_len, P, h->cap, h->cfg.norm_eps, h->hist,
+            h->mean, h->sd, h->done);
 }
 
 void enqueue_denorm(tsfm_spec *h, int B, int N, int H) {
   KTimer kt(h, KC_DENORM, 8.0 * B * H, 2.0 * B * H);
-  denorm_kernel<<<B, 256, 0, h->ls>>>(h->hist, N, h->cfg.patch_len, h->cap, H, h->mean, h->sd, h->st);
-  LAUNCHED();
+  launch_ex(h->ls, h->pdl, denorm_kernel, dim3(B), dim3(256), 0, h->hist, N, h->cfg.patch_len, h->cap, H, h->mean, h->sd,
+            h->st);
 }
 
 // Everything of a speculative forecast that precedes the round loop: counters, traces,
@@ -480,11 +493,10 @@ void enqueue_round(tsfm_spec *h, int B, int N, int T, int K, cudaGraphConditiona
   a.st = h->st;
   {
     KTimer kt(h, KC_ACCEPT, (double)B * (2 * K + 2) * P * 4, 4.0 * B * K * P);
-    accept_kernel<<<(B + 3) / 4, 128, 0, h->ls>>>(a);
-    LAUNCHED();
+    launch_ex(h->ls, h->pdl, accept_kernel, dim3((B + 3) / 4), dim3(128), 0, a);
   }
-  round_end_kernel<<<1, 1, 0, h->ls>>>(h->st, h->unfinished, T, handle, use_handle, body_launches, h->dev_launches);
-  LAUNCHED();
+  launch_ex(h->ls, h->pdl, round_end_kernel, dim3(1), dim3(1), 0, h->st, (const int *)h->unfinished, T, handle,
+            use_handle, body_launches, h->dev_launches);
 }
 
 void enqueue_target_only(tsfm_spec *h, int B, int N, int T, int H) {
@@ -611,7 +623,7 @@ long long device_launches(tsfm_spec *h) {
   return (long long)v;
 }
 
-bool use_graph(const tsfm_spec *h) { return h->cfg.exec_mode == TSFM_EXEC_GRAPH && !h->profiling; }
+bool use_graph(const tsfm_spec *h) { return !(h->cfg.exec_mode & TSFM_EXEC_STREAM) && !h->profiling; }
 
 // Reads status and phase clocks back (synchronises) and fills ms_total.
 int finish_stats(tsfm_spec *h, tsfm_stats *stats, DevState *st_out) {
@@ -686,7 +698,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   *out_h = nullptr;
   const int P = cfg->patch_len;
   if (cfg->dtype != TSFM_F32 && cfg->dtype != TSFM_BF16) return TSFM_ERR_ARG;
-  if (cfg->exec_mode != TSFM_EXEC_GRAPH && cfg->exec_mode != TSFM_EXEC_STREAM) return TSFM_ERR_ARG;
+  if (cfg->exec_mode & ~(TSFM_EXEC_STREAM | TSFM_EXEC_NO_PDL)) return TSFM_ERR_ARG;
   if (cfg->draft_mode != TSFM_DRAFT_SEPARATE && cfg->draft_mode != TSFM_DRAFT_LAYER_SKIP) return TSFM_ERR_ARG;
   if (cfg->max_batch < 1 || cfg->max_ctx_tokens < 2 || cfg->max_horizon_patches < 1 || cfg->max_K < 1 ||
       cfg->max_K > TSFM_MAX_K)
@@ -713,6 +725,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   h->stream = h->ls = (cudaStream_t)cfg->stream;
   h->cap = cfg->max_ctx_tokens + cfg->max_horizon_patches + cfg->max_K + 1;
   h->use_tc = cfg->dtype == TSFM_BF16 && cfg->gemm_backend == TSFM_GEMM_AUTO;
+  h->pdl = (cfg->exec_mode & TSFM_EXEC_NO_PDL) == 0;
   int rc = TSFM_OK;
   auto fail = [&](int code) { tsfm_spec_destroy(h); return code; };
 
@@ -969,7 +982,7 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t
   if (M < 1 || N < 1 || Kd < 16 || Kd % 16) return TSFM_ERR_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   if (backend == TSFM_GEMM_SIMT) {
-    launch_gemm_simt<bf16>(s, (const bf16 *)A, (const bf16 *)W, C, M, N, Kd, EPI_F32);
+    launch_gemm_simt<bf16>(s, false, (const bf16 *)A, (const bf16 *)W, C, M, N, Kd, EPI_F32);
     CU_TRY(cudaGetLastError());
     return TSFM_OK;
   }
@@ -981,7 +994,7 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t
   int *status = nullptr;
   CU_TRY(cudaMalloc((void **)&status, sizeof(int)));
   CU_TRY(cudaMemsetAsync(status, 0, sizeof(int), s));
-  const bool ok = gemm_sk_launch(s, plan, C, M, EPI_F32, status);
+  const bool ok = gemm_sk_launch(s, false, plan, C, M, EPI_F32, status);
   if (ok) LAUNCHED();
   int hs = 0;
   cudaError_t e1 = cudaMemcpyAsync(&hs, status, sizeof(int), cudaMemcpyDeviceToHost, s);

@@ -101,8 +101,18 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
   const uint32_t tmem = *slot_ptr;
 
   if (warp == 4 && lane == 0) {
-    // ---------------- TMA producer
-    for (int kb = 0; kb < KB; ++kb) {
+    // ---------------- TMA producer.  The weights do not depend on the preceding kernel: the
+    // first ring-full of weight tiles is requested before waiting for it, the activation tiles
+    // after.
+    const int pre = KB < stages ? KB : stages;
+    for (int kb = 0; kb < pre; ++kb) {
+      mbar_expect_tx(full0 + 8 * kb, (uint32_t)stage_bytes);
+      tma_load_2d(tiles + kb * stage_bytes, &mapW, (kb_lo + kb) * TC_BK, f0, full0 + 8 * kb);
+    }
+    pdl_sync();
+    for (int kb = 0; kb < pre; ++kb)
+      tma_load_2d(tiles + kb * stage_bytes + TC_W_BYTES, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * kb);
+    for (int kb = pre; kb < KB; ++kb) {
       const int s = kb % stages;
       const uint32_t ph = (uint32_t)(kb / stages) & 1u;
       if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { atomicExch(status, DEV_TIMEOUT_TMA); break; }
@@ -111,6 +121,10 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       tma_load_2d(dst, &mapW, (kb_lo + kb) * TC_BK, f0, full0 + 8 * s);
       tma_load_2d(dst + TC_W_BYTES, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * s);
     }
+  } else {
+    pdl_sync();
+  }
+  if (warp == 4 && lane == 0) {
   } else if (warp == 5 && lane == 0) {
     // ---------------- MMA issuer
     const uint32_t idesc = umma_idesc_rt(BN);
@@ -160,26 +174,52 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
     tc_fence_before();
     cluster_sync_all();
     if (warp < 4) {
-      const int fl = warp * 32 + lane, f = f0 + fl;
+      // thread -> (row group, 4 consecutive features): one 16-byte load per partial tile, all S
+      // loads of a row in flight together, one 16-byte (fp32) or 8-byte (bf16) store per row
+      const int rg = threadIdx.x >> 5, c4 = (threadIdx.x & 31) * 4, f = f0 + c4;
       uint32_t remote[SK_MAX_SPLIT];
 #pragma unroll
       for (int r = 0; r < SK_MAX_SPLIT; ++r) {
-        uint32_t a = tiles + (uint32_t)fl * 4;
+        const uint32_t a = tiles + (uint32_t)c4 * 4;
         asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote[r]) : "r"(a), "r"((uint32_t)(r < S ? r : 0)));
       }
-      for (int tl = rank; tl < BN; tl += S) {
+      const bool vec = (N % 4 == 0) && (f + 3 < N);
+      for (int tl = rank + S * rg; tl < BN; tl += 4 * S) {
         const int t = t0 + tl;
         if (t >= M) break;
-        float sum = 0.f;
+        float4 v[SK_MAX_SPLIT];
 #pragma unroll
-        for (int r = 0; r < SK_MAX_SPLIT; ++r) {
-          if (r < S) {
-            float v;
-            asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote[r] + (uint32_t)tl * (TC_BM * 4)) : "memory");
-            sum += v;
+        for (int r = 0; r < SK_MAX_SPLIT; ++r)
+          if (r < S)
+            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                         : "=f"(v[r].x), "=f"(v[r].y), "=f"(v[r].z), "=f"(v[r].w)
+                         : "r"(remote[r] + (uint32_t)tl * (TC_BM * 4)) : "memory");
+        float4 sum = v[0];
+#pragma unroll
+        for (int r = 1; r < SK_MAX_SPLIT; ++r)
+          if (r < S) { sum.x += v[r].x; sum.y += v[r].y; sum.z += v[r].z; sum.w += v[r].w; }
+        const size_t o = (size_t)t * N + f;
+        if (vec) {
+          if (epi == EPI_F32) {
+            *reinterpret_cast<float4 *>((float *)C + o) = sum;
+          } else if (epi == EPI_RESID) {
+            float4 old = *reinterpret_cast<float4 *>((float *)C + o);
+            old.x += sum.x; old.y += sum.y; old.z += sum.z; old.w += sum.w;
+            *reinterpret_cast<float4 *>((float *)C + o) = old;
+          } else {
+            if (epi == EPI_GELU_T) { sum.x = gelu_erf(sum.x); sum.y = gelu_erf(sum.y); sum.z = gelu_erf(sum.z); sum.w = gelu_erf(sum.w); }
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(sum.x, sum.y), hi = __floats2bfloat162_rn(sum.z, sum.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<const uint32_t *>(&lo);
+            pk.y = *reinterpret_cast<const uint32_t *>(&hi);
+            *reinterpret_cast<uint2 *>((bf16 *)C + o) = pk;
           }
+        } else {
+          const float e[4] = {sum.x, sum.y, sum.z, sum.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            if (f + i < N) sk_store_rt(C, o + i, e[i], epi);
         }
-        if (f < N) sk_store_rt(C, (size_t)t * N + f, sum, epi);
       }
     }
     cluster_sync_all();          // no CTA leaves while a peer may still read its tile
@@ -227,17 +267,22 @@ static int gemm_sk_plan(GemmSkPlan *plan, const void *W, int N, int K, const voi
 // Tile and split choice for M tokens: one token tile up to 256 rows (rounded up to 16), and
 // as many K splits (a power of two, at most 8, at most the number of K blocks) as it takes to
 // put the grid on most of the 148 SMs.
+static int g_sk_force_bn = 0, g_sk_force_s = 0;   // experiment overrides (0 = automatic)
 static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S) {
-  int bn = M >= 256 ? 256 : ((M + 15) / 16) * 16;
+  if (g_sk_force_bn && g_sk_force_s) { *BN = g_sk_force_bn; *S = g_sk_force_s; return; }
+  // Measured on B200 (graph replay, dependent launches): up to a few hundred tokens a 32-token
+  // tile with K split until the grid has ~150-250 CTAs is fastest (the partial-tile exchange
+  // grows with the tile, the latency chain does not shrink); large M takes 128/256-token tiles.
+  int bn = M <= 16 ? 16 : M <= 512 ? 32 : M <= 2048 ? 128 : 256;
   const int tiles = ((N + TC_BM - 1) / TC_BM) * ((M + bn - 1) / bn);
   const int KB = (K + TC_BK - 1) / TC_BK;
   int s = 1;
-  while (s * 2 <= SK_MAX_SPLIT && s * 2 <= KB && tiles * s * 2 <= 160) s *= 2;
+  while (s * 2 <= SK_MAX_SPLIT && s * 2 <= KB && tiles * s * 2 <= 256) s *= 2;
   *BN = bn;
   *S = s;
 }
 
-static bool gemm_sk_launch(cudaStream_t st, GemmSkPlan &p, void *C, int M, int epi, int *status) {
+static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, int M, int epi, int *status) {
   if (!p.valid || M < 1 || M > p.M_max) return false;
   int BN, S;
   gemm_sk_geometry(p.N, p.K, M, &BN, &S);
@@ -254,11 +299,13 @@ static bool gemm_sk_launch(cudaStream_t st, GemmSkPlan &p, void *C, int M, int e
   cfg.blockDim = dim3(192);
   cfg.dynamicSmemBytes = sh.smem_bytes;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = S;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl ? 2 : 1;
   int N = p.N, K = p.K, stages = sh.stages, cols = sh.tmem_cols, rb = ring_bytes;
   return cudaLaunchKernelEx(&cfg, gemm_sk_kernel, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
                             status) == cudaSuccess;

@@ -32,6 +32,7 @@ __global__ void instnorm_kernel(DevState *__restrict__ st, int ctx_len, int P, i
                                 int *__restrict__ done) {
   __shared__ double red[32];
   const int b = blockIdx.x;
+  pdl_sync();
   if (b == 0 && threadIdx.x == 0) st->t_call = globaltimer_ns();
   const float *s = st->series + (size_t)b * ctx_len;
   double acc = 0.0;
@@ -59,6 +60,7 @@ __global__ void denorm_kernel(const float *__restrict__ hist, int N, int P, int 
                               const float *__restrict__ mean, const float *__restrict__ sd,
                               DevState *__restrict__ st) {
   const int b = blockIdx.x;
+  pdl_sync();
   float *out = st->out;
   if (b == 0 && threadIdx.x == 0) st->t_end = globaltimer_ns();
   const float m = mean[b], s = sd[b];
@@ -98,6 +100,7 @@ __global__ void __launch_bounds__(128)
 embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *__restrict__ W,
              float *__restrict__ x, unsigned long long *__restrict__ stamp) {
   extern __shared__ float zs[];
+  pdl_sync();
   const int row = blockIdx.x, b = row / g.q_len, j = row % g.q_len;
   if (stamp && row == 0 && blockIdx.y == 0 && threadIdx.x == 0) *stamp = globaltimer_ns();
   const float *z = hist + ((size_t)b * g.cap + pos0_of(g, b) + j) * P;
@@ -128,6 +131,7 @@ __global__ void __launch_bounds__(128)
 rmsnorm_kernel(const float *__restrict__ x, const float *__restrict__ gain, int d, float eps,
                T *__restrict__ a, float *__restrict__ zero, int zero_cols) {
   __shared__ float red[32];
+  pdl_sync();
   const size_t row = blockIdx.x;
   const float4 *xr = reinterpret_cast<const float4 *>(x + row * d);
   const float4 *gr = reinterpret_cast<const float4 *>(gain);
@@ -165,6 +169,7 @@ gemm_simt_kernel(const T *__restrict__ A, const T *__restrict__ W, void *__restr
   __shared__ float As[16][64 + 4];
   __shared__ float Ws[16][64 + 4];
   const int tid = threadIdx.x;
+  pdl_sync();
   const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
   const int lr = tid >> 2;          // 0..63: tile row loaded by this thread
   const int lk = (tid & 3) * 4;     // 0,4,8,12: first of 4 k's loaded
@@ -266,6 +271,7 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
 
   const int h = blockIdx.x, b = blockIdx.y, qt = blockIdx.z;
   const int d = n_heads * DH;
+  pdl_sync();
   const int p0 = pos0_of(g, b);
   const int j_lo = qt * QT;
   const int j_hi = min(g.q_len, j_lo + QT);          // queries [j_lo, j_hi)
@@ -413,6 +419,7 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
             float *__restrict__ vout) {
   extern __shared__ __align__(16) float xs[];
   __shared__ float red[32];
+  pdl_sync();
   int b, j;
   if (only_last) { b = blockIdx.x; j = g.q_len - 1; }
   else { b = blockIdx.x / g.q_len; j = blockIdx.x % g.q_len; }
