@@ -56,6 +56,11 @@ extern "C" {
 
 #define TSFM_GEMM_AUTO  0       /* bf16 contractions on tcgen05 tensor cores where shapes allow     */
 #define TSFM_GEMM_SIMT  1       /* force the plain FMA kernels everywhere (differential reference)  */
+#define TSFM_GEMM_FUSED_PASS 3  /* as AUTO, but a pass over at most 32 tokens per series group runs as
+                                   ONE cluster kernel (embedding to mean head) when the model has
+                                   head size 64 and at most 8 heads; measured slower than AUTO on
+                                   B200 (one CTA per head cannot stream its weight share fast
+                                   enough), kept as an alternative and a differential target        */
 
 #define TSFM_EXEC_GRAPH   0       /* a forecast is one CUDA-graph launch: prologue, a device-side WHILE
                                    over the rounds, de-normalisation; no host round trip             */

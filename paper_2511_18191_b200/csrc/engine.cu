@@ -20,6 +20,7 @@
 #include "accept.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_sk.cuh"
+#include "pass_cluster.cuh"
 
 using namespace tsfm;
 
@@ -101,6 +102,7 @@ struct ModelDev {
   void *Kc = nullptr, *Vc = nullptr;     // [L][B][heads][cap][dh]
   size_t kv_layer_elems = 0;
   float2 *rope = nullptr;                // [cap][dh/2] (cos, sin)
+  ClPlan cl;                             // whole-pass cluster kernel (small batches), if the shape allows
 };
 
 }  // namespace
@@ -127,6 +129,7 @@ struct tsfm_spec {
   DevState *st = nullptr;
   int cap = 0;
   bool use_tc = false;
+  bool use_cluster = false;              // whole-pass cluster kernel where eligible
   bool pdl = false;                      // launches carry the programmatic-serialization attribute
   ModelDev tgt, drf;
   // activations (sized for M_max rows)
@@ -158,9 +161,9 @@ namespace {
 
 // Kernel classes for per-launch timing.
 enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_TC, KC_GEMM_SIMT, KC_ATTN, KC_HEAD, KC_ACCEPT, KC_DENORM,
-       KC_COUNT };
+       KC_PASS, KC_COUNT };
 const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_tc", "gemm_simt", "attn",
-                                            "head", "accept", "denorm"};
+                                            "head", "accept", "denorm", "pass_cluster"};
 
 // Brackets one launch with two events when profiling is on (no-op otherwise).
 struct KTimer {
@@ -247,6 +250,40 @@ int make_rope(tsfm_spec *h, ModelDev &m) {
   return TSFM_OK;
 }
 
+// Device-resident descriptors of a model for the whole-pass cluster kernel (tensor maps of
+// every weight matrix, gains, cache pointers).  Leaves the plan invalid when the shape is
+// outside that kernel's domain.
+int make_cluster_plan(tsfm_spec *h, ModelDev &m) {
+  const int d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len, L = m.arch.n_layers;
+  m.cl.valid = false;
+  if (m.dh != 64 || !cl_model_ok(m.arch.n_heads, d, f, P)) return TSFM_OK;
+  std::vector<ClLayer> ls(L);
+  ClModel cm{};
+  for (int l = 0; l < L; ++l) {
+    const LayerDev &ly = m.layers[l];
+    if (tc_encode(&ls[l].qkv, ly.Wqkv, 3 * d, d, 64) || tc_encode(&ls[l].wo, ly.Wo, d, d, 128) ||
+        tc_encode(&ls[l].w1, ly.W1, f, d, 128) || tc_encode(&ls[l].w2, ly.W2, d, f, 128))
+      return TSFM_ERR_CUDA;
+    ls[l].g1 = ly.g1;
+    ls[l].g2 = ly.g2;
+    ls[l].Kc = (bf16 *)m.Kc + (size_t)l * m.kv_layer_elems;
+    ls[l].Vc = (bf16 *)m.Vc + (size_t)l * m.kv_layer_elems;
+  }
+  if (tc_encode(&cm.head, m.W_head, P, d, 128)) return TSFM_ERR_CUDA;
+  cm.W_emb = (const bf16 *)m.W_emb;
+  cm.g_f = m.g_f;
+  cm.rope = m.rope;
+  cm.n_layers = L; cm.d = d; cm.heads = m.arch.n_heads; cm.ff = f; cm.P = P;
+  if (int rc = dev_alloc(h, &m.cl.layers, (size_t)L)) return rc;
+  if (int rc = dev_alloc(h, &m.cl.model, 1)) return rc;
+  CU_TRY(cudaMemcpyAsync(m.cl.layers, ls.data(), sizeof(ClLayer) * L, cudaMemcpyHostToDevice, h->stream));
+  CU_TRY(cudaMemcpyAsync(m.cl.model, &cm, sizeof(ClModel), cudaMemcpyHostToDevice, h->stream));
+  CU_TRY(cudaStreamSynchronize(h->stream));
+  m.cl.R = m.arch.n_heads; m.cl.d = d; m.cl.ff = f; m.cl.P = P; m.cl.L = L;
+  m.cl.valid = true;
+  return TSFM_OK;
+}
+
 template <typename T> size_t attn_smem_bytes(int dh, int nk) {
   const int vw = AttnWords<T>::per_row(dh);
   return (size_t)nk * (2 * vw + 1) * 4 + (size_t)4 * nk * sizeof(float) + 4 * dh * sizeof(float);
@@ -292,6 +329,7 @@ void prefer_max_smem_all() {
   prefer_max_smem(accept_kernel);
   prefer_max_smem(round_end_kernel);
   prefer_max_smem(gemm_sk_kernel);
+  prefer_max_smem(pass_cluster_kernel);
   cudaGetLastError();
 }
 
@@ -405,9 +443,41 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   }
 }
 
+// The whole pass as one cluster kernel, when the model and the token count allow it.
+bool pass_fused(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout,
+                unsigned long long *stamp) {
+  if (!h->use_cluster || head_mode == HEAD_NONE) return false;
+  int Bg, BN, G, stages, smem;
+  if (!cl_geometry(m.cl, B, g.q_len, h->cap, &Bg, &BN, &G, &stages, &smem)) return false;
+  ClArgs a{};
+  a.model = m.cl.model;
+  a.layers = m.cl.layers;
+  a.hist_in = h->hist;
+  a.hist_out = h->hist;
+  a.vout = vout;
+  a.g = g;
+  a.B = B; a.Bg = Bg; a.BN = BN; a.stages = stages;
+  a.head_all = head_mode == HEAD_ALL_TO_VOUT;
+  a.eps = h->cfg.rms_eps;
+  a.status = h->dev_status;
+  a.stamp = stamp;
+  // algorithmic bytes: every weight once + the cached keys and values + tokens in, predictions out
+  const int d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len, L = m.arch.n_layers;
+  const double M = (double)B * g.q_len;
+  const double wbytes = 2.0 * ((double)d * P * 2 + (double)L * (4.0 * d * d + 2.0 * d * f));
+  const double kv = (double)L * B * (std::max(g.base, 0) + g.q_len) * 2.0 * d * 2;
+  const double flops = 2.0 * M * ((double)d * P * 2 + (double)L * (4.0 * d * d + 2.0 * d * f)) +
+                       4.0 * M * (std::max(g.base, 0) + 0.5 * g.q_len) * d * L;
+  KTimer kt(h, KC_PASS, wbytes + kv + 2.0 * M * P * 4, flops);
+  if (!cl_launch(h->ls, h->pdl, m.cl, a, G, smem)) return false;
+  LAUNCHED();
+  return true;
+}
+
 void pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout = nullptr,
           unsigned long long *stamp = nullptr) {
   if (g.q_len < 1) return;
+  if (pass_fused(h, m, B, g, head_mode, vout, stamp)) return;
   if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout, stamp);
   else run_pass<float>(h, m, B, g, head_mode, vout, stamp);
 }
@@ -699,6 +769,9 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   const int P = cfg->patch_len;
   if (cfg->dtype != TSFM_F32 && cfg->dtype != TSFM_BF16) return TSFM_ERR_ARG;
   if (cfg->exec_mode & ~(TSFM_EXEC_STREAM | TSFM_EXEC_NO_PDL)) return TSFM_ERR_ARG;
+  if (cfg->gemm_backend != TSFM_GEMM_AUTO && cfg->gemm_backend != TSFM_GEMM_SIMT &&
+      cfg->gemm_backend != TSFM_GEMM_FUSED_PASS)
+    return TSFM_ERR_ARG;
   if (cfg->draft_mode != TSFM_DRAFT_SEPARATE && cfg->draft_mode != TSFM_DRAFT_LAYER_SKIP) return TSFM_ERR_ARG;
   if (cfg->max_batch < 1 || cfg->max_ctx_tokens < 2 || cfg->max_horizon_patches < 1 || cfg->max_K < 1 ||
       cfg->max_K > TSFM_MAX_K)
@@ -724,7 +797,8 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   h->cfg = *cfg;
   h->stream = h->ls = (cudaStream_t)cfg->stream;
   h->cap = cfg->max_ctx_tokens + cfg->max_horizon_patches + cfg->max_K + 1;
-  h->use_tc = cfg->dtype == TSFM_BF16 && cfg->gemm_backend == TSFM_GEMM_AUTO;
+  h->use_tc = cfg->dtype == TSFM_BF16 && cfg->gemm_backend != TSFM_GEMM_SIMT;
+  h->use_cluster = cfg->dtype == TSFM_BF16 && cfg->gemm_backend == TSFM_GEMM_FUSED_PASS;
   h->pdl = (cfg->exec_mode & TSFM_EXEC_NO_PDL) == 0;
   int rc = TSFM_OK;
   auto fail = [&](int code) { tsfm_spec_destroy(h); return code; };
@@ -801,6 +875,11 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
         if ((rc = gemm_sk_plan(&ly.tc_2, ly.W2, d, f, h->hbuf, h->M_max))) return fail(rc);
       }
     }
+  }
+  if (h->use_cluster) {
+    if ((rc = cl_init())) return fail(rc);
+    for (ModelDev *m : {&h->tgt, &h->drf})
+      if ((rc = make_cluster_plan(h, *m))) return fail(rc);
   }
   if (cudaStreamSynchronize(h->stream) != cudaSuccess) return fail(TSFM_ERR_CUDA);
   {

@@ -35,6 +35,7 @@ __host__ __device__ constexpr uint32_t umma_idesc_rt(int bn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
+static int g_sk_force_stages = 0;   // experiment override
 struct SkShape {
   int BN, stages, tmem_cols, smem_bytes;
 };
@@ -45,11 +46,13 @@ static inline SkShape sk_shape(int BN, int kb_per_cta, bool split) {
   s.BN = BN;
   const int stage = TC_W_BYTES + BN * TC_BK * 2;
   int stages = BN > 160 ? 4 : BN > 64 ? 3 : 4;
+  if (g_sk_force_stages) stages = g_sk_force_stages;
   if (stages > kb_per_cta) stages = kb_per_cta < 1 ? 1 : kb_per_cta;
   int bytes = stages * stage;
   if (split && bytes < BN * TC_BM * 4) bytes = BN * TC_BM * 4;
   s.stages = stages;
-  s.tmem_cols = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
+  const int cols = BN;
+  s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : 256;
   s.smem_bytes = bytes + 1024 + 256;
   return s;
 }
@@ -82,6 +85,9 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
   const int kb_hi = (int)(((long long)KB_all * (rank + 1)) / S);
   const int KB = kb_hi - kb_lo;
   const int a_bytes = BN * TC_BK * 2, stage_bytes = TC_W_BYTES + a_bytes;
+  // (Measured: spreading the K steps of a stage over several accumulators does not help a narrow
+  // tile -- one MMA of 128 x BN x 16 takes ~90 ns whatever BN is -- so there is one accumulator.)
+  const int nacc = 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -137,8 +143,10 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       const uint32_t sw = tiles + s * stage_bytes;
       const uint64_t dw = umma_smem_desc(sw), da = umma_smem_desc(sw + TC_W_BYTES);
 #pragma unroll
-      for (int k = 0; k < TC_BK / 16; ++k)
-        umma_bf16(tmem, dw + 2 * k, da + 2 * k, idesc, (kb | k) ? 1u : 0u);
+      for (int k = 0; k < TC_BK / 16; ++k) {
+        if (nacc == 4) umma_bf16(tmem + k * BN, dw + 2 * k, da + 2 * k, idesc, kb ? 1u : 0u);
+        else umma_bf16(tmem, dw + 2 * k, da + 2 * k, idesc, (kb | k) ? 1u : 0u);
+      }
       umma_commit(empty0 + 8 * s);
     }
     if (ok) umma_commit(accum);
@@ -153,6 +161,12 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
         if (t0 + c0 >= M) break;
         float v[16];
         tmem_ld16(tbase + c0, v);
+        for (int q = 1; q < nacc; ++q) {
+          float w[16];
+          tmem_ld16(tbase + q * BN + c0, w);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] += w[j];
+        }
         if (S == 1) {
           if (f < N) {
 #pragma unroll

@@ -74,7 +74,8 @@ def test_c0_shape_ragged_batch_fp32(K, tau, H, exec_mode):
     run_and_compare(wl, K, tau, 7, range(6), exec_mode=exec_mode)
 
 
-@pytest.mark.parametrize("backend,exec_mode", [(1, 1), (0, 1), (0, 0)], ids=["simt-stream", "tcgen05-stream", "tcgen05-graph"])
+@pytest.mark.parametrize("backend,exec_mode", [(1, 1), (0, 1), (0, 0), (3, 0)],
+                         ids=["simt-stream", "tcgen05-stream", "tcgen05-graph", "fused_pass-graph"])
 @pytest.mark.parametrize("tau", [0.5, 1.0, 2.0])
 def test_c1_full(tau, backend, exec_mode):
     wl = workload("C1")

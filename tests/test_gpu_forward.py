@@ -45,10 +45,12 @@ def test_fp32_forward_matches_oracle(target, draft, P, n):
     assert np.abs(gd - wd).max() < 1e-4
 
 
-@pytest.mark.parametrize("backend", [1, 0], ids=["simt", "tcgen05"])
+@pytest.mark.parametrize("backend", [1, 0, 3], ids=["simt", "tcgen05", "fused_pass"])
 @pytest.mark.parametrize("target,draft,P,n,mode", [
-    (Arch(3, 256, 4, 1024), Arch(2, 128, 4, 256), 96, 9, "separate"),
-    (Arch(4, 512, 8, 2048), Arch(2, 512, 8, 2048), 32, 37, "layer_skip"),
+    (Arch(3, 256, 4, 1024), Arch(2, 128, 4, 256), 96, 9, "separate"),      # target: whole-pass cluster kernel
+    (Arch(4, 512, 8, 2048), Arch(2, 512, 8, 2048), 32, 37, "layer_skip"),  # too many tokens per cluster: per-op
+    (Arch(4, 512, 8, 2048), Arch(2, 512, 8, 2048), 32, 6, "layer_skip"),   # 8-CTA clusters, two token tiles of 16
+    (Arch(2, 384, 6, 1536), Arch(1, 128, 2, 256), 96, 3, "separate"),      # 6 heads: 3 feature tiles, ragged owners
 ])
 def test_bf16_forward_matches_oracle(backend, target, draft, P, n, mode):
     wl = small_workload("bf16", target, draft, P, mode)
