@@ -286,7 +286,8 @@ int make_cluster_plan(tsfm_spec *h, ModelDev &m) {
 
 template <typename T> size_t attn_smem_bytes(int dh, int nk) {
   const int vw = AttnWords<T>::per_row(dh);
-  return (size_t)nk * (2 * vw + 1) * 4 + (size_t)4 * nk * sizeof(float) + 4 * dh * sizeof(float);
+  return (size_t)nk * (2 * vw + 1) * 4 + (size_t)ATTN_QT * nk * sizeof(float) + (size_t)5 * ATTN_QT * dh * sizeof(float) +
+         ATTN_QT * sizeof(float);
 }
 
 template <typename T, int DH>
@@ -381,7 +382,7 @@ void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C,
 
 template <typename T, int DH>
 void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
-  const int QT = g.q_len <= 16 ? g.q_len : 16;
+  const int QT = g.q_len <= ATTN_QT ? g.q_len : ATTN_QT;
   dim3 grid(m.arch.n_heads, B, (g.q_len + QT - 1) / QT);
   const int nk_max = (h->cap + 3) & ~3;        // keeps every shared-memory region 16-byte aligned
   const size_t smem = attn_smem_bytes<T>(DH, nk_max);

@@ -235,10 +235,11 @@ gemm_simt_kernel(const T *__restrict__ A, const T *__restrict__ W, void *__restr
 // The CTA loads keys 0..pos0-1 from the cache (16-byte loads) and the keys of this pass
 // (rotated here) up to its last query into shared memory once; all queries of the tile share
 // that read.  The tile that owns a token writes its rotated key and its value to the cache.
-// grid = (heads, B, ceil(q_len / QT)), block = 128 (one query per warp at a time).
+// grid = (heads, B, ceil(q_len / QT)), block = 128; the queries of a tile are processed together.
 // Shared memory is addressed in 32-bit words: K rows are padded by one word so that lanes
 // reading different keys hit different banks.
-//   K tile [nk][KW] words, V tile [nk][VW] words, scores [4][nk] f32, q [4][DH] f32.
+//   K tile [nk][KW] words, V tile [nk][VW] words, scores [16][nk] f32, q [16][DH] f32,
+//   partial outputs [4][16][DH] f32, 1/sum [16] f32.
 // ----------------------------------------------------------------------------------
 template <typename T> struct AttnWords;                 // words per DH elements
 template <> struct AttnWords<float> {
@@ -252,6 +253,109 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t *>(&v);
 }
 
+constexpr int ATTN_QT = 16;                             // queries per tile (at most)
+
+// Scores, softmax and P.V of one query tile from shared memory.  All queries of the tile are
+// processed together, so that every key and value row is read once for the whole tile:
+// (1) scores, one key per thread, all queries; (2) softmax, one query per warp; (3) P.V with the
+// keys dealt out over the four warps and each lane owning DH/32 output dims; (4) sum of the four
+// partial outputs.  NQ = compile-time bound on the number of queries (loops are unrolled to it).
+template <typename T, int DH, int NQ>
+__device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs, float *sc, const float *qs, float *po,
+                                          float *inv_sum, int nq, int nk, int nk_max, int p0, int j_lo, size_t row0,
+                                          int d, int h, T *__restrict__ out) {
+  constexpr bool BF = sizeof(T) == 2;
+  constexpr int VW = AttnWords<T>::per_row(DH), KW = VW + 1, DPL = DH / 32;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, tid = threadIdx.x;
+  for (int t = tid; t < nk; t += blockDim.x) {
+    const uint32_t *kr = Ks + (size_t)t * KW;
+    float sacc[NQ];
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) sacc[i] = 0.f;
+    if (BF) {
+#pragma unroll 4
+      for (int c = 0; c < DH / 2; ++c) {
+        const uint32_t kk = kr[c];
+        const float k0 = __uint_as_float(kk << 16), k1 = __uint_as_float(kk & 0xffff0000u);
+#pragma unroll
+        for (int i = 0; i < NQ; ++i) {
+          const float2 qq = *reinterpret_cast<const float2 *>(qs + i * DH + 2 * c);
+          sacc[i] = fmaf(qq.x, k0, fmaf(qq.y, k1, sacc[i]));
+        }
+      }
+    } else {
+#pragma unroll 4
+      for (int c = 0; c < DH; ++c) {
+        const float kf = __uint_as_float(kr[c]);
+#pragma unroll
+        for (int i = 0; i < NQ; ++i) sacc[i] = fmaf(qs[i * DH + c], kf, sacc[i]);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < NQ; ++i)
+      if (i < nq) sc[(size_t)i * nk_max + t] = (t <= p0 + j_lo + i) ? sacc[i] : -INFINITY;   // causal mask
+  }
+  __syncthreads();
+  for (int i = w; i < nq; i += 4) {
+    float *row = sc + (size_t)i * nk_max;
+    float mx = -INFINITY;
+    for (int t = lane; t < nk; t += 32) mx = fmaxf(mx, row[t]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int t = lane; t < nk; t += 32) {
+      const float pv = expf(row[t] - mx);
+      row[t] = pv;
+      sum += pv;
+    }
+    sum = warp_sum(sum);
+    if (lane == 0) inv_sum[i] = 1.f / sum;
+  }
+  __syncthreads();
+  float acc[NQ][DPL];
+#pragma unroll
+  for (int i = 0; i < NQ; ++i)
+#pragma unroll
+    for (int c = 0; c < DPL; ++c) acc[i][c] = 0.f;
+#pragma unroll 2
+  for (int t = w; t < nk; t += 4) {
+    float v[DPL];
+    if (BF) {
+      if (DPL == 1) {                                // DH = 32: half a word per lane
+        const uint32_t vv = Vs[(size_t)t * VW + lane / 2];
+        v[0] = __uint_as_float((lane & 1) ? (vv & 0xffff0000u) : (vv << 16));
+      } else {
+#pragma unroll
+        for (int c = 0; c < DPL / 2; ++c) {
+          const uint32_t vv = Vs[(size_t)t * VW + lane * (DPL / 2) + c];
+          v[2 * c] = __uint_as_float(vv << 16);
+          v[2 * c + (DPL > 1 ? 1 : 0)] = __uint_as_float(vv & 0xffff0000u);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < DPL; ++c) v[c] = __uint_as_float(Vs[(size_t)t * VW + lane * DPL + c]);
+    }
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) {
+      const float pv = sc[(size_t)i * nk_max + t];     // rows >= nq hold stale but finite-or-not values: never stored
+#pragma unroll
+      for (int c = 0; c < DPL; ++c) acc[i][c] = fmaf(pv, v[c], acc[i][c]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < NQ; ++i)
+    if (i < nq)
+#pragma unroll
+      for (int c = 0; c < DPL; ++c) po[((size_t)w * ATTN_QT + i) * DH + lane * DPL + c] = acc[i][c];
+  __syncthreads();
+  for (int idx = tid; idx < nq * DH; idx += blockDim.x) {
+    const int i = idx / DH, c = idx % DH;
+    const float o = po[(size_t)(0 * ATTN_QT + i) * DH + c] + po[(size_t)(1 * ATTN_QT + i) * DH + c] +
+                    po[(size_t)(2 * ATTN_QT + i) * DH + c] + po[(size_t)(3 * ATTN_QT + i) * DH + c];
+    out[(row0 + j_lo + i) * d + h * DH + c] = from_f32<T>(o * inv_sum[i]);
+  }
+}
+
 template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
@@ -261,13 +365,14 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   constexpr int VW = AttnWords<T>::per_row(DH);   // words per value row
   constexpr int KW = VW + 1;                      // padded key row
   constexpr int HALF = DH / 2;
-  constexpr int DPL = DH / 32;                    // output dims per lane
   constexpr int EPV = 16 / sizeof(T);             // elements per 16-byte vector
   extern __shared__ __align__(16) uint32_t smem_w[];
   uint32_t *Vs = smem_w;                          // [nk_max][VW], 16-byte aligned rows
   uint32_t *Ks = Vs + (size_t)nk_max * VW;        // [nk_max][KW]
   float *sc = reinterpret_cast<float *>(Ks + (size_t)nk_max * KW);
-  float *qs = sc + 4 * nk_max;
+  float *qs = sc + (size_t)ATTN_QT * nk_max;        // [ATTN_QT][DH] rotated, scaled queries
+  float *po = qs + ATTN_QT * DH;                    // [4][ATTN_QT][DH] partial outputs per warp
+  float *inv_sum = po + 4 * ATTN_QT * DH;           // [ATTN_QT]
 
   const int h = blockIdx.x, b = blockIdx.y, qt = blockIdx.z;
   const int d = n_heads * DH;
@@ -279,14 +384,32 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   T *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
   T *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
 
-  // cached keys/values: p0 rows of DH elements, 16 bytes at a time
-  for (int i = threadIdx.x; i < p0 * (DH / EPV); i += blockDim.x) {
-    const int t = i / (DH / EPV), c = i % (DH / EPV);
-    const uint4 kv = *reinterpret_cast<const uint4 *>(Kb + (size_t)t * DH + c * EPV);
-    const uint4 vv = *reinterpret_cast<const uint4 *>(Vb + (size_t)t * DH + c * EPV);
-    uint32_t *kd = Ks + (size_t)t * KW + c * 4;
-    kd[0] = kv.x; kd[1] = kv.y; kd[2] = kv.z; kd[3] = kv.w;
-    *reinterpret_cast<uint4 *>(Vs + (size_t)t * VW + c * 4) = vv;
+  // cached keys/values: p0 rows of DH elements, 16 bytes at a time, eight independent loads in
+  // flight per thread (the cache comes from HBM: the copy is bound by bytes in flight)
+  {
+    constexpr int VPR = DH / EPV;                    // 16-byte vectors per row
+    const int nvec = p0 * VPR;
+    for (int i0 = 0; i0 < nvec; i0 += 4 * blockDim.x) {
+      uint4 kv[4], vv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * blockDim.x + threadIdx.x;
+        if (i < nvec) {
+          kv[u] = *reinterpret_cast<const uint4 *>(Kb + (size_t)i * EPV);
+          vv[u] = *reinterpret_cast<const uint4 *>(Vb + (size_t)i * EPV);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * blockDim.x + threadIdx.x;
+        if (i < nvec) {
+          const int t = i / VPR, c = i % VPR;
+          uint32_t *kd = Ks + (size_t)t * KW + c * 4;
+          kd[0] = kv[u].x; kd[1] = kv[u].y; kd[2] = kv[u].z; kd[3] = kv[u].w;
+          *reinterpret_cast<uint4 *>(Vs + (size_t)i * 4) = vv[u];
+        }
+      }
+    }
   }
   // keys/values of this pass (rotate keys; the owning tile appends to the cache).
   // One thread handles the element pair (c, c + 1) of the first half and its rotation partners.
@@ -329,79 +452,31 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   }
   __syncthreads();
 
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int tid = threadIdx.x;
   const float scale = rsqrtf((float)DH);
-  float *my_sc = sc + (size_t)w * nk_max;
-  float *my_q = qs + w * DH;
-  for (int j = j_lo + w; j < j_hi; j += 4) {
-    const float *src = qkv + (row0 + j) * 3 * d + h * DH;
-    for (int c = lane; c < HALF; c += 32) {
+  const int nq = j_hi - j_lo;                        // <= ATTN_QT
+  const int nk = p0 + j_hi;                          // keys visible to the tile's last query
+  for (int idx = tid; idx < ATTN_QT * HALF; idx += blockDim.x) {   // rotated, scaled queries (zero past nq)
+    const int i = idx / HALF, c = idx % HALF, j = j_lo + i;
+    float r1 = 0.f, r2 = 0.f;
+    if (i < nq) {
+      const float *src = qkv + (row0 + j) * 3 * d + h * DH;
       const float2 cs = rope[(size_t)(p0 + j) * HALF + c];
       const float q1 = src[c], q2 = src[c + HALF];
-      my_q[c] = (q1 * cs.x - q2 * cs.y) * scale;
-      my_q[c + HALF] = (q2 * cs.x + q1 * cs.y) * scale;
+      r1 = (q1 * cs.x - q2 * cs.y) * scale;
+      r2 = (q2 * cs.x + q1 * cs.y) * scale;
     }
-    __syncwarp();
-    const int nv = p0 + j + 1;                       // causal: keys 0..p0+j
-    float mx = -INFINITY;
-    for (int t = lane; t < nv; t += 32) {
-      const uint32_t *kr = Ks + (size_t)t * KW;
-      float s = 0.f;
-      if (BF) {
-#pragma unroll 8
-        for (int c = 0; c < DH / 2; ++c) {
-          const uint32_t kk = kr[c];
-          const float2 qq = *reinterpret_cast<const float2 *>(my_q + 2 * c);
-          s = fmaf(qq.x, __uint_as_float(kk << 16), s);
-          s = fmaf(qq.y, __uint_as_float(kk & 0xffff0000u), s);
-        }
-      } else {
-#pragma unroll 8
-        for (int c = 0; c < DH; ++c) s = fmaf(my_q[c], __uint_as_float(kr[c]), s);
-      }
-      my_sc[t] = s;
-      mx = fmaxf(mx, s);
-    }
-    mx = warp_max(mx);
-    float sum = 0.f;
-    for (int t = lane; t < nv; t += 32) {
-      const float p = expf(my_sc[t] - mx);
-      my_sc[t] = p;
-      sum += p;
-    }
-    sum = warp_sum(sum);
-    __syncwarp();
-    float acc[DPL];
-#pragma unroll
-    for (int c = 0; c < DPL; ++c) acc[c] = 0.f;
-    if (BF) {
-      // lane owns DPL consecutive dims = DPL / 2 words of each value row
-      for (int t = 0; t < nv; ++t) {
-        const float p = my_sc[t];
-#pragma unroll
-        for (int c = 0; c < DPL / 2; ++c) {
-          const uint32_t vv = Vs[(size_t)t * VW + lane * (DPL / 2) + c];
-          acc[2 * c] = fmaf(p, __uint_as_float(vv << 16), acc[2 * c]);
-          acc[2 * c + 1] = fmaf(p, __uint_as_float(vv & 0xffff0000u), acc[2 * c + 1]);
-        }
-        if (DPL == 1) {                              // DH = 32: half a word per lane
-          const uint32_t vv = Vs[(size_t)t * VW + lane / 2];
-          acc[0] = fmaf(p, __uint_as_float((lane & 1) ? (vv & 0xffff0000u) : (vv << 16)), acc[0]);
-        }
-      }
-    } else {
-      for (int t = 0; t < nv; ++t) {
-        const float p = my_sc[t];
-#pragma unroll
-        for (int c = 0; c < DPL; ++c) acc[c] = fmaf(p, __uint_as_float(Vs[(size_t)t * VW + lane * DPL + c]), acc[c]);
-      }
-    }
-    const float inv = 1.f / sum;
-#pragma unroll
-    for (int c = 0; c < DPL; ++c)
-      out[(row0 + j) * d + h * DH + lane * DPL + c] = from_f32<T>(acc[c] * inv);
-    __syncwarp();
+    qs[i * DH + c] = r1;
+    qs[i * DH + c + HALF] = r2;
   }
+  for (int idx = tid + nq * nk_max; idx < ATTN_QT * nk_max; idx += blockDim.x) sc[idx] = 0.f;   // unused score rows
+  __syncthreads();
+  if (nq == 1) attn_tile<T, DH, 1>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
+  else if (nq == 2) attn_tile<T, DH, 2>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
+  else if (nq <= 4) attn_tile<T, DH, 4>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
+  else if (nq <= 6) attn_tile<T, DH, 6>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
+  else if (nq <= 9) attn_tile<T, DH, 9>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
+  else attn_tile<T, DH, ATTN_QT>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
 }
 
 // ----------------------------------------------------------------------------------

@@ -52,7 +52,10 @@ def run_forecast(a):
         wl = wl.with_(**over)
     K = a.K or wl.K
     tw, dw = build_models(wl)
-    dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=K)
+    # kernels inside a graph with a conditional node cannot be profiled one by one: --exec stream
+    # launches the same kernels directly
+    mode = tsfm.TSFM_EXEC_STREAM if a.exec == "stream" else tsfm.TSFM_EXEC_GRAPH
+    dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=K, exec_mode=mode)
     s = make_series(wl)
     ctx = torch.from_numpy(np.ascontiguousarray(s[:, :wl.ctx_len])).cuda()
     out = torch.empty((wl.batch, wl.horizon), device="cuda")
@@ -86,6 +89,7 @@ def main(argv=None):
     f.add_argument("--K", type=int, default=0)
     f.add_argument("--tau", type=float, default=0.0)
     f.add_argument("--reps", type=int, default=2)
+    f.add_argument("--exec", default="graph", choices=["graph", "stream"])
     a = ap.parse_args(argv)
     (run_gemm if a.cmd == "gemm" else run_forecast)(a)
 
