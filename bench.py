@@ -143,6 +143,28 @@ def run_reference(args, wl, K, tau):
     }))
 
 
+# ------------------------------------------------------------------ multi-rank host logic
+def rank_workload(wl, rank: int):
+    """Every rank decodes its own batch: same shapes and weights, different series."""
+    return wl.with_(series_seed=wl.series_seed + 7919 * rank)
+
+
+def max_over_ranks(ms: float, world: int, device="cuda") -> float:
+    """The job's time is the slowest rank's: one scalar all-reduce(MAX) after the timed region."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, series_per_rank: int, patches: int, steps: int, ms: float) -> float:
+    """Committed patches per second of the whole job (all ranks), given the max-over-ranks time."""
+    return world * series_per_rank * patches * steps / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------ our arm
 def run_ours(args, wl, K, tau):
     import torch
@@ -175,7 +197,7 @@ def run_ours(args, wl, K, tau):
     tw, dw = build_models(wl)
     dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=K, device=f"cuda:{local}")
     # every rank decodes its own batch of B series (different series per rank)
-    s = make_series(wl.with_(series_seed=wl.series_seed + 7919 * rank))
+    s = make_series(rank_workload(wl, rank))
     ctx_host = torch.from_numpy(np.ascontiguousarray(s[:, :wl.ctx_len])).pin_memory()
     ctx = ctx_host.cuda()
     B, H, T = wl.batch, wl.horizon, wl.n_patches
@@ -193,12 +215,7 @@ def run_ours(args, wl, K, tau):
             fn(seeds0 + i)
             ev[i][1].record(stream)
         barrier()
-        ms = sum(a.elapsed_time(b) for a, b in ev)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), world)
 
     spec = lambda seed: tsfm.tsfm_spec_forecast(dec.h, ctx, B, wl.ctx_len, H, K, tau, seed, out, None)
     tonly = lambda seed: tsfm.tsfm_target_only_forecast(dec.h, ctx, B, wl.ctx_len, H, out, None)
@@ -231,7 +248,7 @@ def run_ours(args, wl, K, tau):
     tsfm.tsfm_spec_set_profiling(dec.h, False)
 
     units = world * B * T * args.steps
-    value = units / (ms_spec * 1e-3)
+    value = whole_job_value(world, B, T, args.steps, ms_spec)
     result = None
     if rank == 0:
         total_ms = sum(v["ms_total"] for v in prof.values())
