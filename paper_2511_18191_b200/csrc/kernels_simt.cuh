@@ -253,6 +253,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t *>(&v);
 }
 
+// Key rows in shared memory are dense (VW words) with their 16-byte chunks rotated by the row
+// index, so that 16-byte asynchronous copies land aligned and lanes that read the same logical
+// word of consecutive rows spread over the banks.  Physical word of logical word w of row t:
+template <int VW> __device__ __forceinline__ int attn_kword(int t, int w) {
+  return t * VW + ((((w >> 2) + t) & (VW / 4 - 1)) << 2) + (w & 3);
+}
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+
 constexpr int ATTN_QT = 16;                             // queries per tile (at most)
 
 // Scores, softmax and P.V of one query tile from shared memory.  All queries of the tile are
@@ -265,17 +275,16 @@ __device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs
                                           float *inv_sum, int nq, int nk, int nk_max, int p0, int j_lo, size_t row0,
                                           int d, int h, T *__restrict__ out) {
   constexpr bool BF = sizeof(T) == 2;
-  constexpr int VW = AttnWords<T>::per_row(DH), KW = VW + 1, DPL = DH / 32;
+  constexpr int VW = AttnWords<T>::per_row(DH), DPL = DH / 32;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, tid = threadIdx.x;
   for (int t = tid; t < nk; t += blockDim.x) {
-    const uint32_t *kr = Ks + (size_t)t * KW;
     float sacc[NQ];
 #pragma unroll
     for (int i = 0; i < NQ; ++i) sacc[i] = 0.f;
     if (BF) {
 #pragma unroll 4
       for (int c = 0; c < DH / 2; ++c) {
-        const uint32_t kk = kr[c];
+        const uint32_t kk = Ks[attn_kword<VW>(t, c)];
         const float k0 = __uint_as_float(kk << 16), k1 = __uint_as_float(kk & 0xffff0000u);
 #pragma unroll
         for (int i = 0; i < NQ; ++i) {
@@ -286,7 +295,7 @@ __device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs
     } else {
 #pragma unroll 4
       for (int c = 0; c < DH; ++c) {
-        const float kf = __uint_as_float(kr[c]);
+        const float kf = __uint_as_float(Ks[attn_kword<VW>(t, c)]);
 #pragma unroll
         for (int i = 0; i < NQ; ++i) sacc[i] = fmaf(qs[i * DH + c], kf, sacc[i]);
       }
@@ -363,7 +372,7 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
             T *__restrict__ out) {
   constexpr bool BF = sizeof(T) == 2;
   constexpr int VW = AttnWords<T>::per_row(DH);   // words per value row
-  constexpr int KW = VW + 1;                      // padded key row
+  constexpr int KW = VW;                          // dense key row, chunks rotated (attn_kword)
   constexpr int HALF = DH / 2;
   constexpr int EPV = 16 / sizeof(T);             // elements per 16-byte vector
   extern __shared__ __align__(16) uint32_t smem_w[];
@@ -384,31 +393,15 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   T *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
   T *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
 
-  // cached keys/values: p0 rows of DH elements, 16 bytes at a time, eight independent loads in
-  // flight per thread (the cache comes from HBM: the copy is bound by bytes in flight)
+  // cached keys/values: p0 rows of DH elements as 16-byte asynchronous copies, all issued up
+  // front (the cache comes from HBM: the copy is bound by the bytes in flight)
   {
-    constexpr int VPR = DH / EPV;                    // 16-byte vectors per row
+    constexpr int VPR = DH / EPV;                    // 16-byte chunks per row
     const int nvec = p0 * VPR;
-    for (int i0 = 0; i0 < nvec; i0 += 4 * blockDim.x) {
-      uint4 kv[4], vv[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * blockDim.x + threadIdx.x;
-        if (i < nvec) {
-          kv[u] = *reinterpret_cast<const uint4 *>(Kb + (size_t)i * EPV);
-          vv[u] = *reinterpret_cast<const uint4 *>(Vb + (size_t)i * EPV);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = i0 + u * blockDim.x + threadIdx.x;
-        if (i < nvec) {
-          const int t = i / VPR, c = i % VPR;
-          uint32_t *kd = Ks + (size_t)t * KW + c * 4;
-          kd[0] = kv[u].x; kd[1] = kv[u].y; kd[2] = kv[u].z; kd[3] = kv[u].w;
-          *reinterpret_cast<uint4 *>(Vs + (size_t)i * 4) = vv[u];
-        }
-      }
+    for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+      const int t = i / VPR, c = i % VPR;
+      cp_async16(Ks + (size_t)t * VW + (((c + t) & (VPR - 1)) << 2), Kb + (size_t)i * EPV);
+      cp_async16(Vs + (size_t)i * 4, Vb + (size_t)i * EPV);
     }
   }
   // keys/values of this pass (rotate keys; the owning tile appends to the cache).
@@ -427,8 +420,8 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
     if (BF) {
       const uint32_t k1 = pack_bf16x2(r1a, r1b), k2 = pack_bf16x2(r2a, r2b);
       const uint32_t v1 = pack_bf16x2(va.x, va.y), v2 = pack_bf16x2(vb.x, vb.y);
-      Ks[(size_t)t * KW + c / 2] = k1;
-      Ks[(size_t)t * KW + (c + HALF) / 2] = k2;
+      Ks[attn_kword<VW>(t, c / 2)] = k1;
+      Ks[attn_kword<VW>(t, (c + HALF) / 2)] = k2;
       Vs[(size_t)t * VW + c / 2] = v1;
       Vs[(size_t)t * VW + (c + HALF) / 2] = v2;
       if (j >= j_lo) {
@@ -438,9 +431,10 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
         vg[c / 2] = v1; vg[(c + HALF) / 2] = v2;
       }
     } else {
-      float *kf = reinterpret_cast<float *>(Ks + (size_t)t * KW);
+      float *kf = reinterpret_cast<float *>(Ks);
       float *vf = reinterpret_cast<float *>(Vs + (size_t)t * VW);
-      kf[c] = r1a; kf[c + 1] = r1b; kf[c + HALF] = r2a; kf[c + HALF + 1] = r2b;
+      kf[attn_kword<VW>(t, c)] = r1a; kf[attn_kword<VW>(t, c + 1)] = r1b;
+      kf[attn_kword<VW>(t, c + HALF)] = r2a; kf[attn_kword<VW>(t, c + HALF + 1)] = r2b;
       vf[c] = va.x; vf[c + 1] = va.y; vf[c + HALF] = vb.x; vf[c + HALF + 1] = vb.y;
       if (j >= j_lo) {
         float *kg = reinterpret_cast<float *>(Kb + (size_t)t * DH);
@@ -450,7 +444,6 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
       }
     }
   }
-  __syncthreads();
 
   const int tid = threadIdx.x;
   const float scale = rsqrtf((float)DH);
@@ -470,6 +463,7 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
     qs[i * DH + c + HALF] = r2;
   }
   for (int idx = tid + nq * nk_max; idx < ATTN_QT * nk_max; idx += blockDim.x) sc[idx] = 0.f;   // unused score rows
+  asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
   if (nq == 1) attn_tile<T, DH, 1>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
   else if (nq == 2) attn_tile<T, DH, 2>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
