@@ -41,18 +41,18 @@ struct SkShape {
 };
 // Ring of `stages` x (W tile 16 KB + A tile BN x 128 B); the partial-sum tile (BN x 128 fp32)
 // reuses the ring once the accumulator is complete.
-static inline SkShape sk_shape(int BN, int kb_per_cta, bool split) {
+static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1) {
   SkShape s;
   s.BN = BN;
-  const int stage = TC_W_BYTES + BN * TC_BK * 2;
-  int stages = BN > 160 ? 4 : BN > 64 ? 3 : 4;
+  const int stage = TC_W_BYTES * wt + BN * TC_BK * 2;
+  int stages = wt == 2 ? 3 : BN > 160 ? 4 : BN > 64 ? 3 : 4;
   if (g_sk_force_stages) stages = g_sk_force_stages;
   if (stages > kb_per_cta) stages = kb_per_cta < 1 ? 1 : kb_per_cta;
   int bytes = stages * stage;
   if (split && bytes < BN * TC_BM * 4) bytes = BN * TC_BM * 4;
   s.stages = stages;
-  const int cols = BN;
-  s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : 256;
+  const int cols = BN * wt;
+  s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
   s.smem_bytes = bytes + 1024 + 256;
   return s;
 }
@@ -66,10 +66,12 @@ __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi)
 
 // grid = (ceil(N / 128), ceil(M / BN), S), cluster = (1, 1, S), block = 192.
 // ring_bytes = size of the tile region (a multiple of 1024); barriers sit behind it.
+template <int WT>
 __global__ void __launch_bounds__(192, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
                void *__restrict__ C, int M, int N, int K, int BN, int stages, int tmem_cols, int ring_bytes,
                int epi, int *__restrict__ status) {
+  constexpr int wt = WT;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = tiles + (uint32_t)ring_bytes;
@@ -78,16 +80,18 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
   float *stage_f = reinterpret_cast<float *>(smem_raw + (tiles - smem_u32(smem_raw)));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int f0 = blockIdx.x * TC_BM, t0 = blockIdx.y * BN;
+  // wt = weight tiles (of 128 output features) per CTA, 1 or 2.  Two tiles share each token tile
+  // in shared memory: per K block a 256 x 256 output tile loads 64 KB instead of 2 x 48 KB, which
+  // is what lets one CTA's TMA stream (~120 GB/s) keep up with its tensor core.
+  const int f0 = blockIdx.x * TC_BM * wt, t0 = blockIdx.y * BN;
   const int S = gridDim.z, rank = blockIdx.z;
   const int KB_all = (K + TC_BK - 1) / TC_BK;
   const int kb_lo = (int)(((long long)KB_all * rank) / S);
   const int kb_hi = (int)(((long long)KB_all * (rank + 1)) / S);
   const int KB = kb_hi - kb_lo;
-  const int a_bytes = BN * TC_BK * 2, stage_bytes = TC_W_BYTES + a_bytes;
+  const int a_bytes = BN * TC_BK * 2, w_bytes = TC_W_BYTES * wt, stage_bytes = w_bytes + a_bytes;
   // (Measured: spreading the K steps of a stage over several accumulators does not help a narrow
-  // tile -- one MMA of 128 x BN x 16 takes ~90 ns whatever BN is -- so there is one accumulator.)
-  const int nacc = 1;
+  // tile -- one MMA of 128 x BN x 16 takes ~90 ns whatever BN is -- so one accumulator per tile.)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -113,19 +117,21 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
     const int pre = KB < stages ? KB : stages;
     for (int kb = 0; kb < pre; ++kb) {
       mbar_expect_tx(full0 + 8 * kb, (uint32_t)stage_bytes);
-      tma_load_2d(tiles + kb * stage_bytes, &mapW, (kb_lo + kb) * TC_BK, f0, full0 + 8 * kb);
+      for (int q = 0; q < wt; ++q)
+        tma_load_2d(tiles + kb * stage_bytes + q * TC_W_BYTES, &mapW, (kb_lo + kb) * TC_BK, f0 + q * TC_BM, full0 + 8 * kb);
     }
     pdl_sync();
     for (int kb = 0; kb < pre; ++kb)
-      tma_load_2d(tiles + kb * stage_bytes + TC_W_BYTES, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * kb);
+      tma_load_2d(tiles + kb * stage_bytes + w_bytes, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * kb);
     for (int kb = pre; kb < KB; ++kb) {
       const int s = kb % stages;
       const uint32_t ph = (uint32_t)(kb / stages) & 1u;
       if (!mbar_wait(empty0 + 8 * s, ph ^ 1u)) { atomicExch(status, DEV_TIMEOUT_TMA); break; }
       const uint32_t dst = tiles + s * stage_bytes;
       mbar_expect_tx(full0 + 8 * s, (uint32_t)stage_bytes);
-      tma_load_2d(dst, &mapW, (kb_lo + kb) * TC_BK, f0, full0 + 8 * s);
-      tma_load_2d(dst + TC_W_BYTES, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * s);
+      for (int q = 0; q < wt; ++q)
+        tma_load_2d(dst + q * TC_W_BYTES, &mapW, (kb_lo + kb) * TC_BK, f0 + q * TC_BM, full0 + 8 * s);
+      tma_load_2d(dst + w_bytes, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * s);
     }
   } else {
     pdl_sync();
@@ -141,11 +147,11 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       if (!mbar_wait(full0 + 8 * s, ph)) { atomicExch(status, DEV_TIMEOUT_MMA); ok = false; break; }
       tc_fence_after();
       const uint32_t sw = tiles + s * stage_bytes;
-      const uint64_t dw = umma_smem_desc(sw), da = umma_smem_desc(sw + TC_W_BYTES);
+      const uint64_t dw = umma_smem_desc(sw), dw2 = umma_smem_desc(sw + TC_W_BYTES), da = umma_smem_desc(sw + w_bytes);
 #pragma unroll
       for (int k = 0; k < TC_BK / 16; ++k) {
-        if (nacc == 4) umma_bf16(tmem + k * BN, dw + 2 * k, da + 2 * k, idesc, kb ? 1u : 0u);
-        else umma_bf16(tmem, dw + 2 * k, da + 2 * k, idesc, (kb | k) ? 1u : 0u);
+        umma_bf16(tmem, dw + 2 * k, da + 2 * k, idesc, (kb | k) ? 1u : 0u);
+        if (wt == 2) umma_bf16(tmem + BN, dw2 + 2 * k, da + 2 * k, idesc, (kb | k) ? 1u : 0u);
       }
       umma_commit(empty0 + 8 * s);
     }
@@ -154,28 +160,24 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
     // ---------------- epilogue, part 1: drain the accumulator
     if (KB > 0 && mbar_wait(accum, 0)) {
       tc_fence_after();
-      const int fl = warp * 32 + lane, f = f0 + fl;
+      const int fl = warp * 32 + lane;
       const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16);
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 16) {
-        if (t0 + c0 >= M) break;
+      for (int c0 = 0; c0 < BN * wt; c0 += 16) {
+        const int q = c0 >= BN ? 1 : 0, cc = c0 - q * BN;      // weight tile, column inside it
+        const int f = f0 + q * TC_BM + fl;
+        if (t0 + cc >= M) { if (q + 1 < wt) { c0 = BN - 16; continue; } break; }
         float v[16];
         tmem_ld16(tbase + c0, v);
-        for (int q = 1; q < nacc; ++q) {
-          float w[16];
-          tmem_ld16(tbase + q * BN + c0, w);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] += w[j];
-        }
         if (S == 1) {
           if (f < N) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              if (t0 + c0 + j < M) sk_store_rt(C, (size_t)(t0 + c0 + j) * N + f, v[j], epi);
+              if (t0 + cc + j < M) sk_store_rt(C, (size_t)(t0 + cc + j) * N + f, v[j], epi);
           }
         } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * TC_BM + fl] = v[j];
+          for (int j = 0; j < 16; ++j) stage_f[(cc + j) * TC_BM + fl] = v[j];
         }
       }
     } else if (KB > 0 && lane == 0) {
@@ -260,7 +262,8 @@ static int gemm_sk_init() {
   if (int rc = gemm_tc_init()) return rc;
   static bool done = false;
   if (done) return 0;
-  if (cudaFuncSetAttribute(gemm_sk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+  if (cudaFuncSetAttribute(gemm_sk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_sk_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
     return -4;
   done = true;
   return 0;
@@ -281,15 +284,33 @@ static int gemm_sk_plan(GemmSkPlan *plan, const void *W, int N, int K, const voi
 // Tile and split choice for M tokens: one token tile up to 256 rows (rounded up to 16), and
 // as many K splits (a power of two, at most 8, at most the number of K blocks) as it takes to
 // put the grid on most of the 148 SMs.
+static int g_sk_force_wt = 0;
 static int g_sk_force_bn = 0, g_sk_force_s = 0;   // experiment overrides (0 = automatic)
-static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S) {
-  if (g_sk_force_bn && g_sk_force_s) { *BN = g_sk_force_bn; *S = g_sk_force_s; return; }
+static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
+  *WT = 1;
+  if (g_sk_force_bn && g_sk_force_s) {
+    *BN = g_sk_force_bn; *S = g_sk_force_s;
+    if (g_sk_force_wt) *WT = g_sk_force_wt;
+    return;
+  }
   // Measured on B200 (graph replay, dependent launches): up to a few hundred tokens a 32-token
   // tile with K split until the grid has ~150-250 CTAs is fastest (the partial-tile exchange
   // grows with the tile, the latency chain does not shrink); large M takes 128/256-token tiles.
-  int bn = M <= 16 ? 16 : M <= 512 ? 32 : M <= 2048 ? 128 : 256;
-  const int tiles = ((N + TC_BM - 1) / TC_BM) * ((M + bn - 1) / bn);
-  const int KB = (K + TC_BK - 1) / TC_BK;
+  const int FT = (N + TC_BM - 1) / TC_BM, KB = (K + TC_BK - 1) / TC_BK;
+  if (M >= 4096) {
+    // Very large M (prefill, wide verification), no split.  Two candidates, chosen by a two-line
+    // cost model fitted to graph-replay timings on B200 (us per K block of a CTA, epilogue, CTAs
+    // resident per SM):
+    //   (a) 128 x 128 tiles, two CTAs per SM sharing the SM's TMA stream, epilogues overlapped
+    //   (b) 256 x 256 tiles (two weight tiles per CTA), one CTA per SM, loads and MMAs balanced
+    const int ctas_a = FT * ((M + 127) / 128), ctas_b = ((FT + 1) / 2) * ((M + 255) / 256);
+    const double ta = ((ctas_a + 295) / 296) * (KB * 0.53 + 1.5), tb = ((ctas_b + 147) / 148) * (KB * 0.55 + 5.0);
+    *S = 1;
+    if (tb < ta && ctas_b >= 64) { *BN = 256; *WT = 2; } else { *BN = 128; }
+    return;
+  }
+  int bn = M <= 16 ? 16 : M <= 512 ? 32 : 128;
+  const int tiles = FT * ((M + bn - 1) / bn);
   int s = 1;
   while (s * 2 <= SK_MAX_SPLIT && s * 2 <= KB && tiles * s * 2 <= 256) s *= 2;
   *BN = bn;
@@ -298,18 +319,19 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S) {
 
 static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, int M, int epi, int *status) {
   if (!p.valid || M < 1 || M > p.M_max) return false;
-  int BN, S;
-  gemm_sk_geometry(p.N, p.K, M, &BN, &S);
+  int BN, S, wt;
+  gemm_sk_geometry(p.N, p.K, M, &BN, &S, &wt);
   const int idx = BN / 16 - 1;
   if (!p.haveA[idx]) {
     if (tc_encode(&p.mapA[idx], p.A, p.M_max, p.K, BN)) return false;
     p.haveA[idx] = true;
   }
   const int KB = (p.K + TC_BK - 1) / TC_BK;
-  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1);
+  const int FT = (p.N + TC_BM - 1) / TC_BM, TT = (M + BN - 1) / BN;
+  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1, wt);
   const int ring_bytes = sh.smem_bytes - 1024 - 256;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((p.N + TC_BM - 1) / TC_BM, (M + BN - 1) / BN, S);
+  cfg.gridDim = dim3((FT + wt - 1) / wt, TT, S);
   cfg.blockDim = dim3(192);
   cfg.dynamicSmemBytes = sh.smem_bytes;
   cfg.stream = st;
@@ -321,7 +343,10 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 2 : 1;
   int N = p.N, K = p.K, stages = sh.stages, cols = sh.tmem_cols, rb = ring_bytes;
-  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
+  if (wt == 2)
+    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<2>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
+                              status) == cudaSuccess;
+  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
                             status) == cudaSuccess;
 }
 
