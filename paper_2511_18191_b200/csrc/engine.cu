@@ -329,8 +329,8 @@ void prefer_max_smem_all() {
   prefer_max_smem(denorm_kernel);
   prefer_max_smem(accept_kernel);
   prefer_max_smem(round_end_kernel);
-  prefer_max_smem(gemm_sk_kernel<1>);
-  prefer_max_smem(gemm_sk_kernel<2>);
+  prefer_max_smem(gemm_sk_kernel<1, false>);
+  prefer_max_smem(gemm_sk_kernel<2, true>);
   prefer_max_smem(pass_cluster_kernel);
   cudaGetLastError();
 }

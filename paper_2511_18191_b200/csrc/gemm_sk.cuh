@@ -66,7 +66,9 @@ __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi)
 
 // grid = (ceil(N / 128), ceil(M / BN), S), cluster = (1, 1, S), block = 192.
 // ring_bytes = size of the tile region (a multiple of 1024); barriers sit behind it.
-template <int WT>
+// WT = weight tiles per CTA; WIDE = compile the 64-token residual epilogue (only with two weight
+// tiles, one CTA per SM: it costs registers that launches with several CTAs per SM cannot spare).
+template <int WT, bool WIDE>
 __global__ void __launch_bounds__(192, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
                void *__restrict__ C, int M, int N, int K, int BN, int stages, int tmem_cols, int ring_bytes,
@@ -167,6 +169,20 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
         const int q = c0 >= BN ? 1 : 0, cc = c0 - q * BN;      // weight tile, column inside it
         const int f = f0 + q * TC_BM + fl;
         if (t0 + cc >= M) { if (q + 1 < wt) { c0 = BN - 16; continue; } break; }
+        if (WIDE && S == 1 && epi == EPI_RESID && f < N && cc + 64 <= BN && t0 + cc + 64 <= M) {
+          // residual epilogue, 64 tokens at a time: the 64 old values are requested before the
+          // accumulator is read, so one L2 round trip covers them all
+          float r[64], v[64];
+          float *cp = (float *)C + (size_t)(t0 + cc) * N + f;
+#pragma unroll
+          for (int j = 0; j < 64; ++j) r[j] = cp[(size_t)j * N];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) tmem_ld16(tbase + c0 + 16 * u, v + 16 * u);
+#pragma unroll
+          for (int j = 0; j < 64; ++j) cp[(size_t)j * N] = r[j] + v[j];
+          c0 += 48;
+          continue;
+        }
         float v[16];
         tmem_ld16(tbase + c0, v);
         if (S == 1) {
@@ -262,8 +278,8 @@ static int gemm_sk_init() {
   if (int rc = gemm_tc_init()) return rc;
   static bool done = false;
   if (done) return 0;
-  if (cudaFuncSetAttribute(gemm_sk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_sk_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+  if (cudaFuncSetAttribute(gemm_sk_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_sk_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
     return -4;
   done = true;
   return 0;
@@ -344,9 +360,9 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   cfg.numAttrs = pdl ? 2 : 1;
   int N = p.N, K = p.K, stages = sh.stages, cols = sh.tmem_cols, rb = ring_bytes;
   if (wt == 2)
-    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<2>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
+    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<2, true>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
                               status) == cudaSuccess;
-  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
+  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, false>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
                             status) == cudaSuccess;
 }
 
