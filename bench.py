@@ -165,6 +165,21 @@ def whole_job_value(world: int, series_per_rank: int, patches: int, steps: int, 
     return world * series_per_rank * patches * steps / (ms * 1e-3)
 
 
+def throughput_law(stats, to_stats, K, T):
+    """Predicted speedup S(K) = E[L] / (c K + v) of the paper's Eq. 8 from this run's own measurements:
+    acceptance rate alpha = accepted / tested, c = draft step time / target step time, v = verification
+    pass time / target step time (phase clocks of the decoder), E[L] of Eq. 7."""
+    rounds = max(stats["rounds"], 1)
+    step = to_stats["ms_verify"] / T
+    if step <= 0:
+        return None
+    alpha = stats["proposals_accepted"] / max(stats["proposals_tested"], 1)
+    c = stats["ms_draft"] / (rounds * K) / step
+    v = stats["ms_verify"] / rounds / step
+    e_l = float(K + 1) if alpha >= 1.0 else (1.0 - alpha ** (K + 1)) / (1.0 - alpha)
+    return {"alpha": alpha, "c": c, "v": v, "E_L": e_l, "predicted_speedup": e_l / (c * K + v)}
+
+
 # ------------------------------------------------------------------ our arm
 def run_ours(args, wl, K, tau):
     import torch
@@ -219,12 +234,14 @@ def run_ours(args, wl, K, tau):
 
     spec = lambda seed: tsfm.tsfm_spec_forecast(dec.h, ctx, B, wl.ctx_len, H, K, tau, seed, out, None)
     tonly = lambda seed: tsfm.tsfm_target_only_forecast(dec.h, ctx, B, wl.ctx_len, H, out, None)
+    donly = lambda seed: tsfm.tsfm_draft_only_forecast(dec.h, ctx, B, wl.ctx_len, H, out, None)
     spec_host = lambda seed: tsfm.tsfm_spec_forecast_host(dec.h, ctx_host, B, wl.ctx_len, H, K, tau, seed, out_host, None)
 
     seed0 = wl.forecast_seed
     for i in range(args.warmup):
         spec(seed0 + i)
         tonly(0)
+        donly(0)
         spec_host(seed0 + i)
     sampler = ClockSampler(local)
     if rank == 0:
@@ -234,11 +251,20 @@ def run_ours(args, wl, K, tau):
     launches = tsfm.tsfm_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     ms_tonly = timed(tonly, args.steps, 0)
+    ms_donly = timed(donly, args.steps, 0)
+    # accuracy of the three arms against the synthetic ground-truth tail (normalised series: plain MSE)
+    truth = torch.from_numpy(np.ascontiguousarray(s[:, wl.ctx_len:wl.ctx_len + H])).cuda()
+    mse = {}
+    for name, fn in (("target_only", tonly), ("draft_only", donly), ("speculative", spec)):
+        fn(seed0)
+        mse[name] = float(((out - truth) ** 2).mean().item())
     ms_e2e = timed(spec_host, args.steps, seed0)
 
     # one forecast for the acceptance counters, then one profiled forecast for per-kernel times
     _, st = dec.forecast(ctx, H, K, tau, seed0)
     stats = st.as_dict()
+    _, st_t = dec.target_only(ctx, H)
+    to_stats = st_t.as_dict()
     tsfm.tsfm_spec_set_profiling(dec.h, True)
     flush.fill_(1)
     n_prof = 3
@@ -276,7 +302,10 @@ def run_ours(args, wl, K, tau):
             "clocks": clocks,
             "roofline": roofline,
             "target_only": {"value": units / (ms_tonly * 1e-3), "unit": UNIT, "ms_per_step": ms_tonly / args.steps},
+            "draft_only": {"value": units / (ms_donly * 1e-3), "unit": UNIT, "ms_per_step": ms_donly / args.steps},
             "speedup_vs_target_only": ms_tonly / ms_spec,
+            "mse_vs_truth": mse,
+            "throughput_law": throughput_law(stats, to_stats, K, T),
             "acceptance": {"accepted_over_tested": acc / max(tested, 1), "rounds": stats["rounds"],
                            "mean_yield": (sum(l * c for l, c in enumerate(stats["L_hist"])) /
                                           max(sum(stats["L_hist"]), 1))},

@@ -169,6 +169,12 @@ int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx
 int tsfm_target_only_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len,
                               int32_t H, float *out, tsfm_stats *stats);
 
+/* Draft-only decoding: the same loop as tsfm_target_only_forecast run with the draft model alone
+ * (the third arm of the paper's matched three-way protocol, Sec. 4.1 "Evaluation Protocol").
+ * Timing goes to ms_prefill / ms_draft. */
+int tsfm_draft_only_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len,
+                             int32_t H, float *out, tsfm_stats *stats);
+
 /* The two forecasts with HOST buffers: series host [B, ctx_len], out host [B, H] (pinned
  * memory makes the copies asynchronous; pageable memory works too).  The input is copied to
  * a device staging buffer owned by the handle, the forecast runs as above, the result is

@@ -24,7 +24,7 @@ TSFM_MAX_K = 32
 
 EXPORTS = [
     "tsfm_weights_bytes", "tsfm_weights_offset", "tsfm_spec_create", "tsfm_spec_forecast",
-    "tsfm_target_only_forecast", "tsfm_spec_forecast_host", "tsfm_target_only_forecast_host",
+    "tsfm_target_only_forecast", "tsfm_draft_only_forecast", "tsfm_spec_forecast_host", "tsfm_target_only_forecast_host",
     "tsfm_spec_last_trace", "tsfm_accept_round", "tsfm_model_forward", "tsfm_gemm_bf16", "tsfm_gemm_bf16_static",
     "tsfm_spec_set_profiling", "tsfm_spec_kernel_profile", "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
 ]
@@ -87,7 +87,7 @@ def _load() -> C.CDLL:
         fn = getattr(lib, name)
         fn.restype = C.c_int
         fn.argtypes = [vp, vp, i32, i32, i32, i32, f32, u64, vp, C.POINTER(tsfm_stats)]
-    for name in ("tsfm_target_only_forecast", "tsfm_target_only_forecast_host"):
+    for name in ("tsfm_target_only_forecast", "tsfm_draft_only_forecast", "tsfm_target_only_forecast_host"):
         fn = getattr(lib, name)
         fn.restype = C.c_int
         fn.argtypes = [vp, vp, i32, i32, i32, vp, C.POINTER(tsfm_stats)]
@@ -210,6 +210,11 @@ def tsfm_spec_forecast(h, series, B, ctx_len, H, K, tau, seed, out, stats: Optio
 def tsfm_target_only_forecast(h, series, B, ctx_len, H, out, stats: Optional[tsfm_stats] = None) -> None:
     _check(lib.tsfm_target_only_forecast(h, _ptr(series), B, ctx_len, H, _ptr(out),
                                          C.byref(stats) if stats is not None else None), "tsfm_target_only_forecast")
+
+
+def tsfm_draft_only_forecast(h, series, B, ctx_len, H, out, stats: Optional[tsfm_stats] = None) -> None:
+    _check(lib.tsfm_draft_only_forecast(h, _ptr(series), B, ctx_len, H, _ptr(out),
+                                        C.byref(stats) if stats is not None else None), "tsfm_draft_only_forecast")
 
 
 def tsfm_spec_forecast_host(h, series, B, ctx_len, H, K, tau, seed, out, stats: Optional[tsfm_stats] = None) -> None:
@@ -342,6 +347,14 @@ class SpecDecoder:
             out = self.torch.empty((B, H), dtype=self.torch.float32, device=series.device)
         st = tsfm_stats() if stats else None
         tsfm_target_only_forecast(self.h, series, B, ctx_len, H, out, st)
+        return out, st
+
+    def draft_only(self, series, H: int, out=None, stats: bool = True):
+        B, ctx_len = series.shape
+        if out is None:
+            out = self.torch.empty((B, H), dtype=self.torch.float32, device=series.device)
+        st = tsfm_stats() if stats else None
+        tsfm_draft_only_forecast(self.h, series, B, ctx_len, H, out, st)
         return out, st
 
     def last_trace(self, B: int, K: int):

@@ -162,7 +162,7 @@ namespace {
 // Kernel classes for per-launch timing.
 enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_TC, KC_GEMM_SIMT, KC_ATTN, KC_HEAD, KC_ACCEPT, KC_DENORM,
        KC_PASS, KC_COUNT };
-const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_tc", "gemm_simt", "attn",
+const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_sk", "gemm_simt", "attn",
                                             "head", "accept", "denorm", "pass_cluster"};
 
 // Brackets one launch with two events when profiling is on (no-op otherwise).
@@ -571,11 +571,12 @@ void enqueue_round(tsfm_spec *h, int B, int N, int T, int K, cudaGraphConditiona
             use_handle, body_launches, h->dev_launches);
 }
 
-void enqueue_target_only(tsfm_spec *h, int B, int N, int T, int H) {
+// Plain patch-autoregressive decoding with one model (the target, or the draft on its own).
+void enqueue_single_model(tsfm_spec *h, ModelDev &m, int B, int N, int T, int H) {
   enqueue_begin(h, B, N * h->cfg.patch_len);
-  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
-  for (int t = 0; t < T; ++t)       // Eq. 1: one target pass per committed patch
-    pass(h, h->tgt, B, PassGeom{nullptr, N - 1 + t, 1, h->cap}, HEAD_LAST_TO_HIST, nullptr,
+  pass(h, m, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
+  for (int t = 0; t < T; ++t)       // Eq. 1: one pass per committed patch
+    pass(h, m, B, PassGeom{nullptr, N - 1 + t, 1, h->cap}, HEAD_LAST_TO_HIST, nullptr,
          t == 0 ? &h->st->t_phase[0] : nullptr);
   enqueue_denorm(h, B, N, H);
 }
@@ -603,8 +604,8 @@ int capture_graph(tsfm_spec *h, const GraphKey &k, int slot, GraphInfo *out) {
     return rc == TSFM_OK;
   };
   h->ls = cs;
-  if (k.mode == 1) {
-    enqueue_target_only(h, k.B, k.N, T, k.H);
+  if (k.mode != 0) {
+    enqueue_single_model(h, k.mode == 1 ? h->tgt : h->drf, k.B, k.N, T, k.H);
   } else {
     enqueue_spec_prologue(h, k.B, k.N, T, k.K);
     cudaStreamCaptureStatus status;
@@ -892,8 +893,8 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   return TSFM_OK;
 }
 
-int tsfm_target_only_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H,
-                              float *out, tsfm_stats *stats) {
+static int single_model_forecast(tsfm_spec *h, int mode, const float *series, int32_t B, int32_t ctx_len, int32_t H,
+                                 float *out, tsfm_stats *stats) {
   if (int rc = check_call(h, series, B, ctx_len, H, out, 1)) return rc;
   const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
   cudaStream_t s = h->stream;
@@ -901,12 +902,12 @@ int tsfm_target_only_forecast(tsfm_spec *h, const float *series, int32_t B, int3
   if (int rc = write_call_state(h, series, out, 1.f, 0)) return rc;
   if (use_graph(h)) {
     GraphInfo gi;
-    if (int rc = get_graph(h, GraphKey{1, B, N, H, 0}, &gi)) return rc;
+    if (int rc = get_graph(h, GraphKey{mode, B, N, H, 0}, &gi)) return rc;
     CU_TRY(cudaGraphLaunch(gi.exec, s));
     g_launches.fetch_add(gi.n_fixed, std::memory_order_relaxed);
   } else {
     h->ls = s;
-    enqueue_target_only(h, B, N, T, H);
+    enqueue_single_model(h, mode == 1 ? h->tgt : h->drf, B, N, T, H);
   }
   CU_TRY(cudaGetLastError());
   if (stats) {
@@ -914,12 +915,22 @@ int tsfm_target_only_forecast(tsfm_spec *h, const float *series, int32_t B, int3
     DevState st;
     if (int rc = finish_stats(h, stats, &st)) return rc;
     stats->ms_prefill = (float)((st.t_phase[0] - st.t_call) * 1e-6);
-    stats->ms_verify = (float)((st.t_end - st.t_phase[0]) * 1e-6);
+    (mode == 1 ? stats->ms_verify : stats->ms_draft) = (float)((st.t_end - st.t_phase[0]) * 1e-6);
     stats->rounds = T;
     stats->patches_committed = (int64_t)B * T;
     if (stats->device_status) return TSFM_ERR_TIMEOUT;
   }
   return TSFM_OK;
+}
+
+int tsfm_target_only_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H,
+                              float *out, tsfm_stats *stats) {
+  return single_model_forecast(h, 1, series, B, ctx_len, H, out, stats);
+}
+
+int tsfm_draft_only_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H,
+                             float *out, tsfm_stats *stats) {
+  return single_model_forecast(h, 2, series, B, ctx_len, H, out, stats);
 }
 
 int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H, int32_t K,

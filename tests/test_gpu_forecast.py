@@ -144,6 +144,22 @@ def test_c4_subset():
     run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, [0, 63])
 
 
+@pytest.mark.parametrize("name,ids", [("C0", [0]), ("C1", [0, 7, 31]), ("C2", [3, 200])])
+def test_draft_only_forecast_matches_oracle(name, ids):
+    """Third arm of the matched three-way protocol: the draft model decoding on its own (Eq. 1)."""
+    wl = workload(name)
+    dec, tw, dw = make_decoder(wl)
+    s, ctx = series_on_device(wl)
+    out, st = dec.draft_only(ctx, wl.horizon)
+    d = st.as_dict()
+    assert d["device_status"] == 0 and d["rounds"] == wl.n_patches and d["patches_committed"] == wl.batch * wl.n_patches
+    dec.close()
+    tm, dm = parity.oracle_models(wl, tw, dw)
+    want = orc.forecast_target_only(dm, s[list(ids)], wl.ctx_len, wl.horizon)
+    kind, tol = parity.VALUE_TOL[wl.dtype]
+    assert parity.value_error(kind, out.cpu().numpy()[list(ids)], want) <= tol
+
+
 def test_tiny_tau_recovers_target_only_and_result_is_independent_of_batch_composition():
     wl = workload("C1")
     dec, tw, dw = make_decoder(wl)
