@@ -134,7 +134,7 @@ struct tsfm_spec {
   ModelDev tgt, drf;
   // activations (sized for M_max rows)
   int M_max = 0;
-  float *x = nullptr, *qkv = nullptr;
+  float *x = nullptr, *qkv = nullptr, *ssq = nullptr;   // ssq: [M_max][d / 32] slice sums of squares
   void *a = nullptr, *ao = nullptr, *hbuf = nullptr;
   // decoding state
   float *hist = nullptr, *vout = nullptr, *mean = nullptr, *sd = nullptr;
@@ -329,8 +329,9 @@ void prefer_max_smem_all() {
   prefer_max_smem(denorm_kernel);
   prefer_max_smem(accept_kernel);
   prefer_max_smem(round_end_kernel);
-  prefer_max_smem(gemm_sk_kernel<1, false>);
-  prefer_max_smem(gemm_sk_kernel<2, true>);
+  prefer_max_smem(gemm_sk_kernel<1, false, false>);
+  prefer_max_smem(gemm_sk_kernel<1, false, true>);
+  prefer_max_smem(gemm_sk_kernel<2, true, false>);
   prefer_max_smem(pass_cluster_kernel);
   cudaGetLastError();
 }
@@ -368,14 +369,14 @@ void launch_gemm_simt(cudaStream_t s, bool pdl, const T *A, const T *W, void *C,
 // C (op)= A . W^T through the tensor-core kernel when a plan exists, else the FMA kernel.
 template <typename T>
 void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C, int M, int N,
-          int K, int epi) {
+          int K, int epi, const SkNorm *norm = nullptr) {
   const double e = sizeof(T);
   const double out_b = (epi == EPI_F32 || epi == EPI_ATOMIC) ? 4.0 : epi == EPI_RESID ? 8.0 : e;
   const double bytes = ((double)N * K + (double)M * K) * e + (double)M * N * out_b;
   const double flops = 2.0 * M * N * K;
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
     KTimer kt(h, KC_GEMM_TC, bytes, flops);
-    if (gemm_sk_launch(h->ls, h->pdl, *plan, C, M, epi, h->dev_status)) { LAUNCHED(); return; }
+    if (gemm_sk_launch(h->ls, h->pdl, *plan, C, M, epi, h->dev_status, norm)) { LAUNCHED(); return; }
   }
   KTimer kt(h, KC_GEMM_SIMT, bytes, flops);
   launch_gemm_simt<T>(h->ls, h->pdl, (const T *)A, (const T *)W, C, M, N, K, epi);
@@ -407,31 +408,49 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   const int M = B * g.q_len, d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len;
   cudaStream_t s = h->ls;
   const float eps = h->cfg.rms_eps;
+  // On the tensor-core path the RMSNorms are folded into the contractions around them (SkNorm):
+  // whoever produces the residual stream also writes the next operand a' = bf16(gain * x) and the
+  // rows' slice sums of squares; whoever consumes a' scales its result rows by rstd.
+  // (Only for passes of few tokens, where a launch costs more than the extra epilogue work: with
+  // large tiles the epilogue is the bottleneck and the separate RMSNorm kernel is the cheaper way.)
+  const bool fold = sizeof(T) == 2 && h->use_tc && m.layers[0].tc_qkv.valid && M <= 512;
+  const int L = m.arch.n_layers;
   {
     KTimer kt(h, KC_EMBED, (double)M * P * 4 + (double)d * P * sizeof(T) + (double)M * d * 4, 2.0 * M * P * d);
     launch_ex(s, h->pdl, embed_kernel<T>, dim3(M, (d + 127) / 128), dim3(128), P * sizeof(float), h->hist, g, P, d,
-              (const T *)m.W_emb, h->x, stamp);
+              (const T *)m.W_emb, h->x, stamp, fold ? m.layers[0].g1 : (const float *)nullptr,
+              fold ? (T *)h->a : (T *)nullptr, fold ? h->ssq : (float *)nullptr);
   }
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
-  const int L = m.arch.n_layers;
+  SkNorm consume{};                 // scale the result rows by rstd of the input rows
+  consume.ssq_in = h->ssq;
+  consume.n_part = d / 32;
+  consume.inv_d = 1.f / d;
+  consume.eps = eps;
   for (int l = 0; l < L; ++l) {
     LayerDev &ly = m.layers[l];
-    {
+    if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
       launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3(M), dim3(128), 0, h->x, ly.g1, d, eps, (T *)h->a, nullptr, 0);
     }
-    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32);
+    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
     else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
     else launch_attn<T, 128>(h, m, l, B, g);
     if (l == L - 1 && head_mode == HEAD_NONE) break;   // prefill: only the cache is needed
-    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID);
-    {
+    SkNorm produce{};               // residual epilogue also emits the next operand and its statistics
+    produce.ssq_out = h->ssq;
+    produce.a_out = (bf16 *)h->a;
+    produce.gain = ly.g2;
+    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, fold ? &produce : nullptr);
+    if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
       launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3(M), dim3(128), 0, h->x, ly.g2, d, eps, (T *)h->a, nullptr, 0);
     }
-    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T);
-    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID);
+    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, fold ? &consume : nullptr);
+    produce.gain = l + 1 < L ? m.layers[l + 1].g1 : nullptr;
+    if (l + 1 == L) produce.a_out = nullptr, produce.ssq_out = nullptr;   // the head kernel norms the final rows itself
+    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID, fold && l + 1 < L ? &produce : nullptr);
   }
   const double rows = head_mode == HEAD_LAST_TO_HIST ? B : M;
   KTimer kt(h, head_mode == HEAD_NONE ? -1 : KC_HEAD, rows * d * 4 + (double)P * d * sizeof(T) + rows * P * 4,
@@ -834,6 +853,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   const size_t Mx = h->M_max;
   if ((rc = dev_alloc(h, &h->x, Mx * dmax))) return fail(rc);
   if ((rc = dev_alloc(h, &h->qkv, Mx * 3 * dmax))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->ssq, Mx * (dmax / 32 + 1)))) return fail(rc);
   if ((rc = dev_alloc(h, (char **)&h->a, Mx * dmax * e))) return fail(rc);
   if ((rc = dev_alloc(h, (char **)&h->ao, Mx * dmax * e))) return fail(rc);
   if ((rc = dev_alloc(h, (char **)&h->hbuf, Mx * fmax * e))) return fail(rc);

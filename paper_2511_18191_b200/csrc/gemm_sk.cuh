@@ -35,6 +35,20 @@ __host__ __device__ constexpr uint32_t umma_idesc_rt(int bn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
+// RMSNorm folded into the contractions around it.  The norm of a row is a scalar factor, so it
+// commutes with the contraction that consumes the row: the kernel that PRODUCES the residual
+// stream (residual epilogue) also writes a' = bf16(gain * x) -- the next contraction's operand,
+// not yet normalised -- and the sum of squares of every 32-feature slice of the row; the kernel
+// that CONSUMES a' multiplies its result rows by rstd = rsqrt(sum of the slices / d + eps).
+struct SkNorm {
+  const float *ssq_in;      // [M][n_part] slice sums of squares of this contraction's input rows, or NULL
+  float *ssq_out;           // [M][N / 32] written by a residual epilogue, or NULL
+  const float *gain;        // [N] gain of the norm that follows the residual epilogue
+  bf16 *a_out;              // [M][N] bf16(gain * x_new), or NULL
+  int n_part;               // slices per input row (d / 32)
+  float inv_d, eps;
+};
+
 static int g_sk_force_stages = 0;   // experiment override
 struct SkShape {
   int BN, stages, tmem_cols, smem_bytes;
@@ -53,7 +67,7 @@ static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1) {
   s.stages = stages;
   const int cols = BN * wt;
   s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
-  s.smem_bytes = bytes + 1024 + 256;
+  s.smem_bytes = bytes + 1024 + 256 + 1024;        // + alignment slack, barriers, rstd of the tile's rows
   return s;
 }
 
@@ -68,17 +82,19 @@ __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi)
 // ring_bytes = size of the tile region (a multiple of 1024); barriers sit behind it.
 // WT = weight tiles per CTA; WIDE = compile the 64-token residual epilogue (only with two weight
 // tiles, one CTA per SM: it costs registers that launches with several CTAs per SM cannot spare).
-template <int WT, bool WIDE>
+// NORM = compile the folded-RMSNorm epilogues (SkNorm); the plain instantiations carry none of it.
+template <int WT, bool WIDE, bool NORM>
 __global__ void __launch_bounds__(192, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
                void *__restrict__ C, int M, int N, int K, int BN, int stages, int tmem_cols, int ring_bytes,
-               int epi, int *__restrict__ status) {
+               int epi, const SkNorm nm, int *__restrict__ status) {
   constexpr int wt = WT;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = tiles + (uint32_t)ring_bytes;
   const uint32_t full0 = bars, empty0 = bars + 64, accum = bars + 128, slot = bars + 136;
   uint32_t *slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (slot - smem_u32(smem_raw)));
+  float *rs = reinterpret_cast<float *>(smem_raw + (bars + 256 - smem_u32(smem_raw)));   // [BN] rstd of the tile's rows
   float *stage_f = reinterpret_cast<float *>(smem_raw + (tiles - smem_u32(smem_raw)));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -137,6 +153,17 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
     }
   } else {
     pdl_sync();
+    if (warp < 4) {
+      if (NORM && nm.ssq_in) {                                // overlaps the main loop
+        for (int i = threadIdx.x; i < BN; i += 128) {
+          float acc = 0.f;
+          if (t0 + i < M)
+            for (int j = 0; j < nm.n_part; ++j) acc += nm.ssq_in[(size_t)(t0 + i) * nm.n_part + j];
+          rs[i] = rsqrtf(acc * nm.inv_d + nm.eps);
+        }
+      }
+      if (NORM) asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
   }
   if (warp == 4 && lane == 0) {
   } else if (warp == 5 && lane == 0) {
@@ -179,7 +206,15 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
 #pragma unroll
           for (int u = 0; u < 4; ++u) tmem_ld16(tbase + c0 + 16 * u, v + 16 * u);
 #pragma unroll
-          for (int j = 0; j < 64; ++j) cp[(size_t)j * N] = r[j] + v[j];
+          for (int j = 0; j < 64; ++j) {
+            const float xn = r[j] + v[j];
+            cp[(size_t)j * N] = xn;
+            if (NORM && nm.a_out) {
+              nm.a_out[(size_t)(t0 + cc + j) * N + f] = __float2bfloat16_rn(nm.gain[f] * xn);
+              const float sq = warp_sum(xn * xn);
+              if (lane == 0) nm.ssq_out[(size_t)(t0 + cc + j) * (N >> 5) + (f >> 5)] = sq;
+            }
+          }
           c0 += 48;
           continue;
         }
@@ -189,7 +224,25 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
           if (f < N) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              if (t0 + cc + j < M) sk_store_rt(C, (size_t)(t0 + cc + j) * N + f, v[j], epi);
+              if (t0 + cc + j < M) {
+                const size_t o = (size_t)(t0 + cc + j) * N + f;
+                if (NORM && nm.ssq_in) v[j] *= rs[cc + j];
+                if (NORM && epi == EPI_RESID && nm.a_out) {
+                  const float xn = ((float *)C)[o] + v[j];
+                  ((float *)C)[o] = xn;
+                  nm.a_out[o] = __float2bfloat16_rn(nm.gain[f] * xn);
+                  v[j] = xn * xn;
+                } else {
+                  sk_store_rt(C, o, v[j], epi);
+                }
+              }
+          }
+          if (NORM && epi == EPI_RESID && nm.a_out) {          // slice sums of squares (N is a multiple of 32 here)
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float sq = warp_sum(v[j]);
+              if (lane == 0 && t0 + cc + j < M) nm.ssq_out[(size_t)(t0 + cc + j) * (N >> 5) + (f >> 5)] = sq;
+            }
           }
         } else {
 #pragma unroll
@@ -231,6 +284,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
         for (int r = 1; r < SK_MAX_SPLIT; ++r)
           if (r < S) { sum.x += v[r].x; sum.y += v[r].y; sum.z += v[r].z; sum.w += v[r].w; }
         const size_t o = (size_t)t * N + f;
+        if (NORM && nm.ssq_in) { const float k = rs[tl]; sum.x *= k; sum.y *= k; sum.z *= k; sum.w *= k; }
         if (vec) {
           if (epi == EPI_F32) {
             *reinterpret_cast<float4 *>((float *)C + o) = sum;
@@ -238,6 +292,19 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
             float4 old = *reinterpret_cast<float4 *>((float *)C + o);
             old.x += sum.x; old.y += sum.y; old.z += sum.z; old.w += sum.w;
             *reinterpret_cast<float4 *>((float *)C + o) = old;
+            if (NORM && nm.a_out) {
+              const float4 gg = *reinterpret_cast<const float4 *>(nm.gain + f);
+              const __nv_bfloat162 lo = __floats2bfloat162_rn(gg.x * old.x, gg.y * old.y), hi = __floats2bfloat162_rn(gg.z * old.z, gg.w * old.w);
+              uint2 pk;
+              pk.x = *reinterpret_cast<const uint32_t *>(&lo);
+              pk.y = *reinterpret_cast<const uint32_t *>(&hi);
+              *reinterpret_cast<uint2 *>(nm.a_out + o) = pk;
+              float sq = old.x * old.x + old.y * old.y + old.z * old.z + old.w * old.w;   // 8 lanes = one 32-feature slice
+              sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+              sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+              sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+              if ((threadIdx.x & 7) == 0) nm.ssq_out[(size_t)t * (N >> 5) + (f >> 5)] = sq;
+            }
           } else {
             if (epi == EPI_GELU_T) { sum.x = gelu_erf(sum.x); sum.y = gelu_erf(sum.y); sum.z = gelu_erf(sum.z); sum.w = gelu_erf(sum.w); }
             const __nv_bfloat162 lo = __floats2bfloat162_rn(sum.x, sum.y), hi = __floats2bfloat162_rn(sum.z, sum.w);
@@ -278,8 +345,9 @@ static int gemm_sk_init() {
   if (int rc = gemm_tc_init()) return rc;
   static bool done = false;
   if (done) return 0;
-  if (cudaFuncSetAttribute(gemm_sk_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_sk_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+  if (cudaFuncSetAttribute(gemm_sk_kernel<1, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_sk_kernel<1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_sk_kernel<2, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
     return -4;
   done = true;
   return 0;
@@ -322,7 +390,8 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
     const int ctas_a = FT * ((M + 127) / 128), ctas_b = ((FT + 1) / 2) * ((M + 255) / 256);
     const double ta = ((ctas_a + 295) / 296) * (KB * 0.53 + 1.5), tb = ((ctas_b + 147) / 148) * (KB * 0.55 + 5.0);
     *S = 1;
-    if (tb < ta && ctas_b >= 64) { *BN = 256; *WT = 2; } else { *BN = 128; }
+    // (with fewer than 16 K blocks the unoverlapped epilogue of the big tile eats the gain: measured)
+    if (tb < ta && ctas_b >= 64 && KB >= 16) { *BN = 256; *WT = 2; } else { *BN = 128; }
     return;
   }
   int bn = M <= 16 ? 16 : M <= 512 ? 32 : 128;
@@ -333,7 +402,8 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
   *S = s;
 }
 
-static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, int M, int epi, int *status) {
+static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, int M, int epi, int *status,
+                           const SkNorm *norm = nullptr) {
   if (!p.valid || M < 1 || M > p.M_max) return false;
   int BN, S, wt;
   gemm_sk_geometry(p.N, p.K, M, &BN, &S, &wt);
@@ -345,7 +415,8 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   const int KB = (p.K + TC_BK - 1) / TC_BK;
   const int FT = (p.N + TC_BM - 1) / TC_BM, TT = (M + BN - 1) / BN;
   const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1, wt);
-  const int ring_bytes = sh.smem_bytes - 1024 - 256;
+  const int ring_bytes = sh.smem_bytes - 1024 - 256 - 1024;
+  const SkNorm nm = norm ? *norm : SkNorm{};
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((FT + wt - 1) / wt, TT, S);
   cfg.blockDim = dim3(192);
@@ -360,10 +431,13 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   cfg.numAttrs = pdl ? 2 : 1;
   int N = p.N, K = p.K, stages = sh.stages, cols = sh.tmem_cols, rb = ring_bytes;
   if (wt == 2)
-    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<2, true>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
-                              status) == cudaSuccess;
-  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, false>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
-                            status) == cudaSuccess;
+    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<2, true, false>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
+                              nm, status) == cudaSuccess;
+  if (norm)
+    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, false, true>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb,
+                              epi, nm, status) == cudaSuccess;
+  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, false, false>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
+                            nm, status) == cudaSuccess;
 }
 
 }  // namespace tsfm

@@ -98,7 +98,8 @@ template <> struct Vec16<bf16> {
 template <typename T>
 __global__ void __launch_bounds__(128)
 embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *__restrict__ W,
-             float *__restrict__ x, unsigned long long *__restrict__ stamp) {
+             float *__restrict__ x, unsigned long long *__restrict__ stamp,
+             const float *__restrict__ gain, T *__restrict__ a_out, float *__restrict__ ssq_out) {
   extern __shared__ float zs[];
   pdl_sync();
   const int row = blockIdx.x, b = row / g.q_len, j = row % g.q_len;
@@ -119,6 +120,11 @@ embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *
     for (int c = 0; c < V; ++c) acc = fmaf(w[c], zs[i + c], acc);
   }
   x[(size_t)row * d + f] = acc;
+  if (a_out) {            // operand of the first contraction, normalised later (see SkNorm); d % 32 == 0
+    a_out[(size_t)row * d + f] = from_f32<T>(gain[f] * acc);
+    const float sq = warp_sum(acc * acc);
+    if ((threadIdx.x & 31) == 0) ssq_out[(size_t)row * (d >> 5) + (f >> 5)] = sq;
+  }
 }
 
 // ----------------------------------------------------------------------------------
