@@ -297,7 +297,7 @@ int attn_set_attr(size_t bytes) {
 }
 template <typename T>
 int attn_prepare(int dh, int cap) {
-  const size_t bytes = attn_smem_bytes<T>(dh, (cap + 3) & ~3);
+  const size_t bytes = attn_smem_bytes<T>(dh, (cap + 15) & ~15);
   if (bytes > 227 * 1024) return TSFM_ERR_SHAPE;
   const size_t optin = 227 * 1024;        // opt in once to the per-CTA maximum; launches size themselves
   if (dh == 32) return attn_set_attr<T, 32>(optin);
@@ -386,7 +386,7 @@ template <typename T, int DH>
 void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   const int QT = g.q_len <= ATTN_QT ? g.q_len : ATTN_QT;
   dim3 grid(m.arch.n_heads, B, (g.q_len + QT - 1) / QT);
-  const int nk_max = (h->cap + 3) & ~3;        // keeps every shared-memory region 16-byte aligned
+  const int nk_max = (h->cap + 15) & ~15;      // keys padded to whole MMA blocks; regions stay 16-byte aligned
   const size_t smem = attn_smem_bytes<T>(DH, nk_max);
   T *Kc = (T *)m.Kc + (size_t)l * m.kv_layer_elems;
   T *Vc = (T *)m.Vc + (size_t)l * m.kv_layer_elems;

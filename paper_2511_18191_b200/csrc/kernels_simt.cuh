@@ -371,6 +371,130 @@ __device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs
   }
 }
 
+// ----------------------------------------------------------------------------------
+// The same tile computation on the warp-level tensor-core path (mma.sync m16n8k16, bf16 operands,
+// fp32 accumulate) for bf16 caches: the query tile (at most 16 rows) is the M side of both
+// products.  S = Q K^T: each warp takes every fourth block of 8 keys; the rotated fp32 queries
+// are split into a bf16 high and low part (two MMAs) so that the scores keep fp32-like accuracy.
+// O = P V: each warp takes every fourth block of 16 keys, P rounded to bf16, V fragments by
+// ldmatrix.trans; the four partial outputs are summed as in attn_tile.  sc rows >= nq are zero,
+// key columns in [nk, round_up(nk, 16)) get probability 0 and V rows there are zero.
+// ----------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_bf16_16816(float *c, const uint32_t *a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void split_bf16x2(float x, float y, uint32_t &hi, uint32_t &lo) {
+  const float xh = __bfloat162float(__float2bfloat16_rn(x)), yh = __bfloat162float(__float2bfloat16_rn(y));
+  hi = pack_bf16x2(xh, yh);
+  lo = pack_bf16x2(x - xh, y - yh);
+}
+
+template <int DH>
+__device__ __forceinline__ void attn_tile_mma(const uint32_t *Ks, const uint32_t *Vs, float *sc, const float *qs, float *po,
+                                              float *inv_sum, int nq, int nk, int nk_max, int p0, int j_lo, size_t row0,
+                                              int d, int h, bf16 *__restrict__ out) {
+  constexpr int VW = DH / 2, KS = DH / 16;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, tid = threadIdx.x;
+  const int g = lane >> 2, q4 = lane & 3;            // fragment row group, column pair
+  const int nk16 = (nk + 15) & ~15;
+  {
+    // ---- scores
+    uint32_t qhi[KS][4], qlo[KS][4];
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const int c = ks * 16 + q4 * 2;
+      const float2 a = *reinterpret_cast<const float2 *>(qs + g * DH + c);
+      const float2 b = *reinterpret_cast<const float2 *>(qs + (g + 8) * DH + c);
+      const float2 a8 = *reinterpret_cast<const float2 *>(qs + g * DH + c + 8);
+      const float2 b8 = *reinterpret_cast<const float2 *>(qs + (g + 8) * DH + c + 8);
+      split_bf16x2(a.x, a.y, qhi[ks][0], qlo[ks][0]);
+      split_bf16x2(b.x, b.y, qhi[ks][1], qlo[ks][1]);
+      split_bf16x2(a8.x, a8.y, qhi[ks][2], qlo[ks][2]);
+      split_bf16x2(b8.x, b8.y, qhi[ks][3], qlo[ks][3]);
+    }
+    for (int nt = w; nt < nk16 / 8; nt += 4) {
+      const int key = nt * 8 + g;                    // B fragment: this lane's key row
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const uint32_t b0 = Ks[attn_kword<VW>(key, ks * 8 + q4)], b1 = Ks[attn_kword<VW>(key, ks * 8 + 4 + q4)];
+        mma_bf16_16816(c, qhi[ks], b0, b1);
+        mma_bf16_16816(c, qlo[ks], b0, b1);
+      }
+      const int t = nt * 8 + q4 * 2;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int r = g + (e >> 1) * 8, tt = t + (e & 1);
+        if (r < nq) sc[(size_t)r * nk_max + tt] = (tt <= p0 + j_lo + r && tt < nk) ? c[e] : -INFINITY;
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = w; i < nq; i += 4) {
+    float *row = sc + (size_t)i * nk_max;
+    float mx = -INFINITY;
+    for (int t = lane; t < nk16; t += 32) mx = fmaxf(mx, row[t]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int t = lane; t < nk16; t += 32) {
+      const float pv = expf(row[t] - mx);
+      row[t] = pv;
+      sum += pv;
+    }
+    sum = warp_sum(sum);
+    if (lane == 0) inv_sum[i] = 1.f / sum;
+  }
+  __syncthreads();
+  {
+    // ---- P . V
+    float acc[DH / 8][4];
+#pragma unroll
+    for (int n = 0; n < DH / 8; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[n][e] = 0.f;
+    const uint32_t vbase = (uint32_t)__cvta_generic_to_shared(Vs);
+    for (int kb = w; kb < nk16 / 16; kb += 4) {
+      const int t = kb * 16 + q4 * 2;
+      uint32_t a[4];
+      {
+        const float2 p0v = *reinterpret_cast<const float2 *>(sc + (size_t)g * nk_max + t);
+        const float2 p1v = *reinterpret_cast<const float2 *>(sc + (size_t)(g + 8) * nk_max + t);
+        const float2 p2v = *reinterpret_cast<const float2 *>(sc + (size_t)g * nk_max + t + 8);
+        const float2 p3v = *reinterpret_cast<const float2 *>(sc + (size_t)(g + 8) * nk_max + t + 8);
+        a[0] = pack_bf16x2(p0v.x, p0v.y); a[1] = pack_bf16x2(p1v.x, p1v.y);
+        a[2] = pack_bf16x2(p2v.x, p2v.y); a[3] = pack_bf16x2(p3v.x, p3v.y);
+      }
+      // ldmatrix.x4.trans: matrices (keys 0-7 | 8-15) x (dims n0..n0+7 | n0+8..n0+15)
+      const int mrow = kb * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+#pragma unroll
+      for (int n0 = 0; n0 < DH; n0 += 16) {
+        uint32_t b[4];
+        const uint32_t addr = vbase + (uint32_t)(mrow * VW * 4 + (n0 + mcol) * 2);
+        asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]) : "r"(addr));
+        mma_bf16_16816(acc[n0 / 8], a, b[0], b[1]);
+        mma_bf16_16816(acc[n0 / 8 + 1], a, b[2], b[3]);
+      }
+    }
+#pragma unroll
+    for (int n = 0; n < DH / 8; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int r = g + (e >> 1) * 8, c = n * 8 + q4 * 2 + (e & 1);
+        if (r < nq) po[((size_t)w * ATTN_QT + r) * DH + c] = acc[n][e];
+      }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < nq * DH; idx += blockDim.x) {
+    const int i = idx / DH, c = idx % DH;
+    const float o = po[(size_t)(0 * ATTN_QT + i) * DH + c] + po[(size_t)(1 * ATTN_QT + i) * DH + c] +
+                    po[(size_t)(2 * ATTN_QT + i) * DH + c] + po[(size_t)(3 * ATTN_QT + i) * DH + c];
+    out[(row0 + j_lo + i) * d + h * DH + c] = __float2bfloat16_rn(o * inv_sum[i]);
+  }
+}
+
 template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
@@ -471,6 +595,14 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   for (int idx = tid + nq * nk_max; idx < ATTN_QT * nk_max; idx += blockDim.x) sc[idx] = 0.f;   // unused score rows
   asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
+  if (BF && nq >= 3 && nk >= 96) {                   // tensor-core tile routine (bf16 caches, long rows: measured)
+    const int nk16 = (nk + 15) & ~15;
+    for (int idx = tid + nk * VW; idx < nk16 * VW; idx += blockDim.x) Vs[idx] = 0u;   // value rows of the padding keys
+    __syncthreads();
+    if constexpr (BF)
+      attn_tile_mma<DH>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, reinterpret_cast<bf16 *>(out));
+    return;
+  }
   if (nq == 1) attn_tile<T, DH, 1>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
   else if (nq == 2) attn_tile<T, DH, 2>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
   else if (nq <= 4) attn_tile<T, DH, 4>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
