@@ -579,7 +579,10 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   const float scale = rsqrtf((float)DH);
   const int nq = j_hi - j_lo;                        // <= ATTN_QT
   const int nk = p0 + j_hi;                          // keys visible to the tile's last query
-  for (int idx = tid; idx < ATTN_QT * HALF; idx += blockDim.x) {   // rotated, scaled queries (zero past nq)
+  // rows the tile routine will touch: its compile-time query bound (16 on the tensor-core path)
+  const bool use_mma = BF && nq >= 3 && nk >= 96;
+  const int nqb = use_mma ? ATTN_QT : nq <= 2 ? nq : nq <= 4 ? 4 : nq <= 6 ? 6 : nq <= 9 ? 9 : ATTN_QT;
+  for (int idx = tid; idx < nqb * HALF; idx += blockDim.x) {       // rotated, scaled queries (zero past nq)
     const int i = idx / HALF, c = idx % HALF, j = j_lo + i;
     float r1 = 0.f, r2 = 0.f;
     if (i < nq) {
@@ -592,10 +595,10 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
     qs[i * DH + c] = r1;
     qs[i * DH + c + HALF] = r2;
   }
-  for (int idx = tid + nq * nk_max; idx < ATTN_QT * nk_max; idx += blockDim.x) sc[idx] = 0.f;   // unused score rows
+  for (int idx = tid + nq * nk_max; idx < nqb * nk_max; idx += blockDim.x) sc[idx] = 0.f;       // unused score rows
   asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
-  if (BF && nq >= 3 && nk >= 96) {                   // tensor-core tile routine (bf16 caches, long rows: measured)
+  if (use_mma) {                                     // tensor-core tile routine (bf16 caches, long rows: measured)
     const int nk16 = (nk + 15) & ~15;
     for (int idx = tid + nk * VW; idx < nk16 * VW; idx += blockDim.x) Vs[idx] = 0u;   // value rows of the padding keys
     __syncthreads();

@@ -51,6 +51,7 @@ def test_fp32_forward_matches_oracle(target, draft, P, n):
     (Arch(4, 512, 8, 2048), Arch(2, 512, 8, 2048), 32, 37, "layer_skip"),  # too many tokens per cluster: per-op
     (Arch(4, 512, 8, 2048), Arch(2, 512, 8, 2048), 32, 6, "layer_skip"),   # 8-CTA clusters, two token tiles of 16
     (Arch(2, 384, 6, 1536), Arch(1, 128, 2, 256), 96, 3, "separate"),      # 6 heads: 3 feature tiles, ragged owners
+    (Arch(2, 256, 4, 1024), Arch(1, 128, 2, 256), 32, 120, "separate"),    # 120 keys: tensor-core attention tiles
 ])
 def test_bf16_forward_matches_oracle(backend, target, draft, P, n, mode):
     wl = small_workload("bf16", target, draft, P, mode)
