@@ -45,6 +45,7 @@ def parse_args():
     ap.add_argument("--K", type=int, default=None)
     ap.add_argument("--cpu-series", type=int, default=None, help="series per oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--others", default="C2,C4", help="comma list of further workloads to profile briefly ('' = none)")
     return ap.parse_args()
 
 
@@ -141,6 +142,42 @@ def run_reference(args, wl, K, tau):
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+# ------------------------------------------------------------------ other workloads (informational)
+def profile_workload(name, hbm_peak, tf_peak):
+    """One warm speculative and target-only forecast of another workload plus one profiled forecast:
+    where the tensor-bound verification GEMMs (C2) and the KV-bound attention (C4) stand against the
+    measured peaks.  Not part of the headline metric."""
+    import torch
+    import paper_2511_18191_b200 as tsfm
+    from tsfm_inputs import build_models, make_series, workload
+    wl = workload(name)
+    tw, dw = build_models(wl)
+    dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=wl.K)
+    s = make_series(wl)
+    ctx = torch.from_numpy(np.ascontiguousarray(s[:, :wl.ctx_len])).cuda()
+    for _ in range(2):
+        _, st = dec.forecast(ctx, wl.horizon, wl.K, wl.tau, wl.forecast_seed)
+        _, st_t = dec.target_only(ctx, wl.horizon)
+    d, dt = st.as_dict(), st_t.as_dict()
+    tsfm.tsfm_spec_set_profiling(dec.h, True)
+    dec.forecast(ctx, wl.horizon, wl.K, wl.tau, wl.forecast_seed, stats=False)
+    prof = tsfm.tsfm_spec_kernel_profile(dec.h)
+    tsfm.tsfm_spec_set_profiling(dec.h, False)
+    dec.close()
+    tot = sum(v["ms_total"] for v in prof.values())
+    kernels = {}
+    for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms_total"])[:3]:
+        gbs, tfs = v["bytes"] / v["ms_total"] / 1e6, v["flops"] / v["ms_total"] / 1e9
+        kernels[k] = {"share": round(v["ms_total"] / tot, 3), "avg_launch_us": round(v["ms_total"] * 1e3 / v["launches"], 2),
+                      "GB/s": round(gbs, 1), "frac_hbm": round(gbs / hbm_peak, 4),
+                      "TFLOP/s": round(tfs, 1), "frac_tensor": round(tfs / tf_peak, 4)}
+    return {"ms_per_forecast": d["ms_total"], "ms_target_only": dt["ms_total"],
+            "phases_ms": {k: d[k] for k in ("ms_prefill", "ms_draft", "ms_verify", "ms_accept")},
+            "rounds": d["rounds"], "accepted_over_tested": d["proposals_accepted"] / max(d["proposals_tested"], 1),
+            "B": wl.batch, "patches_per_s": wl.batch * wl.n_patches / (d["ms_total"] * 1e-3),
+            "kernels_event_timed": kernels}
 
 
 # ------------------------------------------------------------------ multi-rank host logic
@@ -317,6 +354,14 @@ def run_ours(args, wl, K, tau):
                                       "sample": f"{n_series} of {B} series of {wl.name}, full forecast, 3 repeats, "
                                                 f"{total:.1f} s"}
     dec.close()
+    if result is not None and world == 1 and args.others:
+        tf_peak = float(peaks.get("bf16_tflops_sustained", 1400.0))
+        result["other_workloads"] = {"peaks": {"hbm_gbs": hbm_peak, "bf16_tflops_sustained": tf_peak, "source": peak_src}}
+        for name in [n for n in args.others.split(",") if n]:
+            try:
+                result["other_workloads"][name] = profile_workload(name, hbm_peak, tf_peak)
+            except Exception as e:          # informational: never lose the headline line
+                result["other_workloads"][name] = {"error": repr(e)}
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
