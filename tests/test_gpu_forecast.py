@@ -160,6 +160,17 @@ def test_draft_only_forecast_matches_oracle(name, ids):
     assert parity.value_error(kind, out.cpu().numpy()[list(ids)], want) <= tol
 
 
+@pytest.mark.parametrize("K,H,ctx_patches,B", [(32, 96 * 3, 2, 2), (1, 50, 2, 1), (5, 96, 3, 7), (8, 96 * 9 + 1, 7, 3)])
+def test_edge_geometries_fp32(K, H, ctx_patches, B):
+    """Degenerate and extreme geometries on the fp32 path: the largest block size the ABI allows (far
+    more proposals than patches to commit), a horizon shorter than one patch, the shortest legal
+    context (two patches), a single-patch horizon with K > T, a ragged last patch."""
+    wl = workload("C0", batch=B, series_recipe="c1", horizon=H, ctx_len=96 * ctx_patches)
+    for mode in (1, 0):
+        res = run_and_compare(wl, K, 2.0, 11, range(B), exec_mode=mode)
+        assert res["stats"]["rounds"] <= -(-H // 96)
+
+
 def test_tiny_tau_recovers_target_only_and_result_is_independent_of_batch_composition():
     wl = workload("C1")
     dec, tw, dw = make_decoder(wl)
