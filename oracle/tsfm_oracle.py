@@ -85,6 +85,42 @@ def acceptance_uniform(seed: int, series: int, rnd: int, pos: int) -> float:
     return uniform_from_word(philox4x32_10((series, rnd, pos, 0), key)[0])
 
 
+NOISE_PROPOSAL = 0x10000000      # counter word 3 of the proposal-noise stream
+NOISE_FALLBACK = 0x20000000      # ... of the fallback / bonus noise stream
+
+
+def standard_normals(seed: int, series: int, rnd: int, pos: int, stream: int, n: int) -> np.ndarray:
+    """n standard normal draws for the sampled variants of Section 3.3 (proposal noise, fallback
+    noise).  Box-Muller on Philox words: element pair (2j, 2j+1) takes the counter
+    (series, round, position, stream | j), u1, u2 from output words 0 and 1 on the same 23-bit grid
+    as the acceptance uniforms, z = sqrt(-2 ln u1) * (cos, sin)(2 pi u2)."""
+    key = (seed & _MASK32, (seed >> 32) & _MASK32)
+    out = np.empty(n)
+    for j in range((n + 1) // 2):
+        w = philox4x32_10((series, rnd, pos, stream | j), key)
+        u1, u2 = uniform_from_word(w[0]), uniform_from_word(w[1])
+        rad = math.sqrt(-2.0 * math.log(u1))
+        out[2 * j] = rad * math.cos(2.0 * math.pi * u2)
+        if 2 * j + 1 < n:
+            out[2 * j + 1] = rad * math.sin(2.0 * math.pi * u2)
+    return out
+
+
+@dataclass
+class Variant:
+    """Knobs of the general rule (Sections 3.2-3.3, Algorithm 1); the deployed scheme is the default.
+
+    sigma_q:           draft surrogate scale (None = sigma_p: the determinant term vanishes)
+    sample_proposals:  x_i = mu_q^(i) + sigma_q * eps instead of the mean
+    fallback_noise:    r in t = mu_p + r * eps for the correction and the bonus patch
+    tempering:         False drops the 1/d factor of Eq. 5 (component ablation)
+    """
+    sigma_q: Optional[float] = None
+    sample_proposals: bool = False
+    fallback_noise: float = 0.0
+    tempering: bool = True
+
+
 # ----------------------------------------------------------------------------
 # The network (this build's reading; see the header)
 # ----------------------------------------------------------------------------
@@ -238,8 +274,13 @@ class RoundRecord:
 def speculative_round(hist: np.ndarray, target: Model, draft: Model, K: int, sigma: float,
                       uniforms: Sequence[float],
                       forced: Optional[Sequence[bool]] = None,
-                      caches=None) -> RoundRecord:
-    """Algorithm 1 for one series with mean proposals and r = 0.
+                      caches=None, variant: Optional[Variant] = None,
+                      proposal_eps: Optional[np.ndarray] = None,
+                      fallback_eps: Optional[np.ndarray] = None) -> RoundRecord:
+    """Algorithm 1 for one series; mean proposals and r = 0 unless ``variant`` says otherwise.
+
+    With a variant the standard-normal draws are inputs: ``proposal_eps`` [K, P] for the sampled
+    proposals, ``fallback_eps`` [K+1, P] (row i for a correction at position i, row K for the bonus).
 
     hist: [n, P] context + committed patches (normalised space).  ``uniforms``
     supplies u_1..u_K.  ``forced`` (optional) overrides the decisions, used to
@@ -256,17 +297,28 @@ def speculative_round(hist: np.ndarray, target: Model, draft: Model, K: int, sig
         out = forward(model, tokens[cache.length:], cache)
         return np.concatenate([np.zeros((tokens.shape[0] - out.shape[0], out.shape[1])), out], axis=0)
 
+    var = variant or Variant()
+    sigma_q = sigma if var.sigma_q is None else var.sigma_q
     props: List[np.ndarray] = []
+    means: List[np.ndarray] = []
     for i in range(K):                                    # draft rollout
         toks = np.concatenate([hist] + [p[None, :] for p in props], axis=0)
-        props.append(run(draft, dc, toks)[-1])
-    x = np.stack(props, axis=0)                           # x_i = mu_q^(i)
+        mu = run(draft, dc, toks)[-1]
+        means.append(mu)
+        props.append(mu + sigma_q * proposal_eps[i] if var.sample_proposals else mu)
+    x = np.stack(props, axis=0)                           # x_i = mu_q^(i) (+ sigma_q eps)
+    mu_q = np.stack(means, axis=0)
     o = run(target, tc, np.concatenate([hist, x], axis=0))
     mu_p = o[n - 1: n + K]                                # boundaries N-1+i, i = 0..K
+    if var.fallback_noise != 0.0:
+        mu_p = mu_p + var.fallback_noise * np.asarray(fallback_eps, dtype=np.float64)
     ell, log_u, dec = [], [], []
     n_acc = 0
     for i in range(K):
-        l_i = log_ratio(x[i], mu_p[i], x[i], sigma, sigma)
+        mp_i = o[n - 1 + i]                               # the statistic uses the noise-free target mean
+        l_i = log_ratio(x[i], mp_i, mu_q[i], sigma, sigma_q)
+        if not var.tempering:
+            l_i *= x.shape[1]                             # l_i is (1/d) log p/q: undo the 1/d
         ok = accept(l_i, uniforms[i]) if forced is None else bool(forced[i])
         ell.append(l_i)
         log_u.append(math.log(uniforms[i]))
@@ -331,7 +383,8 @@ class ForecastTrace:
 def forecast_speculative(target: Model, draft: Model, series: np.ndarray, ctx_len: int, H: int,
                          K: int, tau: float, seed: int,
                          forced: Optional[List[List[Sequence[bool]]]] = None,
-                         use_cache: bool = True, series_index0: int = 0):
+                         use_cache: bool = True, series_index0: int = 0,
+                         variant: Optional[Variant] = None):
     """Algorithm 1 looped until T = ceil(H/P) patches are committed, per series.
 
     Every round drafts K and verifies K+1; the committed list of the last round
@@ -351,7 +404,13 @@ def forecast_speculative(target: Model, draft: Model, series: np.ndarray, ctx_le
         while done < T:
             us = [acceptance_uniform(seed, series_index0 + b, rnd, i) for i in range(K)]
             f = None if forced is None else forced[b][rnd]
-            rec = speculative_round(hist, target, draft, K, tau, us, forced=f, caches=caches)
+            pe = fe = None
+            if variant is not None and variant.sample_proposals:
+                pe = np.stack([standard_normals(seed, series_index0 + b, rnd, i, NOISE_PROPOSAL, P) for i in range(K)])
+            if variant is not None and variant.fallback_noise != 0.0:
+                fe = np.stack([standard_normals(seed, series_index0 + b, rnd, i, NOISE_FALLBACK, P) for i in range(K + 1)])
+            rec = speculative_round(hist, target, draft, K, tau, us, forced=f, caches=caches, variant=variant,
+                                    proposal_eps=pe, fallback_eps=fe)
             new = committed_patches(rec)[: T - done]
             rec.committed = new.shape[0]
             hist = np.concatenate([hist, new], axis=0)

@@ -313,3 +313,102 @@ def test_simulated_rounds_match_the_pmf():
             L += 1
         counts[L] += 1
     np.testing.assert_allclose(counts[1:] / n, orc.capped_geometric_pmf(alpha, K), atol=0.01)
+
+
+# ----------------------------------------------------------------------------
+# Sampled variants (Sec. 3.3 "Fallback Correction and Sampled Variants"; Algorithm 1 with r > 0)
+# ----------------------------------------------------------------------------
+def test_standard_normals_are_standard_and_streams_differ():
+    z = np.concatenate([orc.standard_normals(7, s, 0, 0, orc.NOISE_PROPOSAL, 96) for s in range(400)])
+    assert abs(z.mean()) < 0.02 and abs(z.var() - 1.0) < 0.03
+    assert abs(np.mean(z ** 4) - 3.0) < 0.15                        # Gaussian kurtosis
+    assert abs(np.mean(np.abs(z) > 1.959964) - 0.05) < 0.005        # two-sided 5 % tail
+    a = orc.standard_normals(7, 1, 2, 3, orc.NOISE_PROPOSAL, 8)
+    b = orc.standard_normals(7, 1, 2, 3, orc.NOISE_FALLBACK, 8)
+    assert not np.allclose(a, b)
+    np.testing.assert_array_equal(a[:5], orc.standard_normals(7, 1, 2, 3, orc.NOISE_PROPOSAL, 5))   # prefix-stable
+
+
+def test_sampled_proposals_accept_at_the_equal_covariance_rate_in_one_dimension():
+    """Equal-covariance acceptance (appendix proposition): with x ~ q = N(mu_q, s^2) and the
+    untempered ratio, the mean acceptance is 2 Phi(-Delta / 2), Delta = |mu_p - mu_q| / s.  In one
+    dimension the 1/d tempering is the identity, so the rule as implemented must reproduce it."""
+    from scipy.stats import norm
+    rng = np.random.default_rng(5)
+    s, mu_q = 0.7, np.array([0.3])
+    for delta in (0.5, 1.0, 2.0):
+        mu_p = mu_q + delta * s
+        x = mu_q + s * rng.standard_normal((200000, 1))
+        ell = np.array([orc.log_ratio(xi, mu_p, mu_q, s, s) for xi in x[:20000]])
+        alpha = np.minimum(1.0, np.exp(ell)).mean()
+        assert alpha == pytest.approx(2 * norm.cdf(-delta / 2), abs=0.01)
+
+
+def test_round_with_sampled_proposals_fallback_noise_and_unequal_scales():
+    """Algorithm 1 in its general form, step by step against its definition: x_i = mu_q^(i) + sigma_q eps_i
+    where mu_q^(i) is the draft's mean given the SAMPLED x_1..x_{i-1}; the statistic is Eq. 5 with both
+    energies and the determinant term; a rejection commits mu_p^(i) + r eps, full acceptance the bonus
+    mu_p^(K+1) + r eps."""
+    tgt, drf = tiny_models(P=8)
+    P, K, sp, sq, r = 8, 3, 0.9, 0.5, 0.25
+    hist = toy_series(1, 5 * P, seed=2)[0].reshape(5, P)
+    rng = np.random.default_rng(9)
+    pe, fe = rng.standard_normal((K, P)), rng.standard_normal((K + 1, P))
+    var = orc.Variant(sigma_q=sq, sample_proposals=True, fallback_noise=r)
+    for script in ([True, True, True], [True, False], [False]):
+        rec = orc.speculative_round(hist, tgt, drf, K, sp, [0.5] * K, forced=script, variant=var,
+                                    proposal_eps=pe, fallback_eps=fe)
+        # proposals: rebuilt by per-prefix draft forwards on the sampled tokens
+        toks = hist.copy()
+        for i in range(K):
+            mu = orc.forward(drf, toks)[-1]
+            np.testing.assert_allclose(rec.mu_q[i], mu + sq * pe[i], rtol=0, atol=1e-12)
+            toks = np.concatenate([toks, rec.mu_q[i][None, :]], axis=0)
+        # statistic of the first tested position, written out from Eq. 5
+        mu_q1 = orc.forward(drf, hist)[-1]
+        mu_p1 = orc.forward(tgt, hist)[-1]
+        x1 = rec.mu_q[0]
+        want = (-np.sum((x1 - mu_p1) ** 2) / P / (2 * sp ** 2) + np.sum((x1 - mu_q1) ** 2) / P / (2 * sq ** 2)
+                + 0.5 * math.log(sq ** 2 / sp ** 2))
+        assert rec.ell[0] == pytest.approx(want, rel=1e-12)
+        n = rec.n_accept
+        assert n == sum(script[:script.index(False)] if False in script else script)
+        commit = orc.committed_patches(rec)
+        np.testing.assert_array_equal(commit[:n], rec.mu_q[:n])
+        clean = orc.forward(tgt, np.concatenate([hist, rec.mu_q[:n]], axis=0))[-1]
+        np.testing.assert_allclose(commit[n], clean + r * fe[n], rtol=0, atol=1e-12)
+
+
+def test_dropping_the_tempering_multiplies_the_statistic_by_d_and_kills_acceptance():
+    """Component ablation (Table 2, row "w/o 1/d tempering"): the untempered log ratio is d times
+    the tempered one, and at patch dimensions acceptance collapses."""
+    tgt, drf = tiny_models(P=8)
+    P, K = 8, 2
+    hist = toy_series(1, 4 * P, seed=4)[0].reshape(4, P)
+    a = orc.speculative_round(hist, tgt, drf, K, 1.0, [0.999] * K, forced=[True, True])
+    b = orc.speculative_round(hist, tgt, drf, K, 1.0, [0.999] * K, forced=[True, True],
+                              variant=orc.Variant(tempering=False))
+    np.testing.assert_allclose(np.array(b.ell), P * np.array(a.ell), rtol=1e-12)
+    s = toy_series(6, 4 * P + 6 * P, seed=5)
+    _, tr_t = orc.forecast_speculative(tgt, drf, s, 4 * P, 6 * P, K, 1.0, 3)
+    _, tr_u = orc.forecast_speculative(tgt, drf, s, 4 * P, 6 * P, K, 1.0, 3, variant=orc.Variant(tempering=False))
+    acc = lambda tr: sum(sum(r.decisions) for sr in tr.rounds for r in sr)
+    assert acc(tr_u) <= acc(tr_t)
+
+
+def test_variant_defaults_reproduce_the_deployed_scheme_and_noise_is_seeded():
+    tgt, drf = tiny_models(P=8)
+    P = 8
+    s = toy_series(3, 4 * P + 5 * P, seed=6)
+    base, _ = orc.forecast_speculative(tgt, drf, s, 4 * P, 5 * P, 2, 1.0, 11)
+    same, _ = orc.forecast_speculative(tgt, drf, s, 4 * P, 5 * P, 2, 1.0, 11, variant=orc.Variant())
+    np.testing.assert_array_equal(base, same)
+    v = orc.Variant(sample_proposals=True, fallback_noise=0.3)
+    n1, _ = orc.forecast_speculative(tgt, drf, s, 4 * P, 5 * P, 2, 1.0, 11, variant=v)
+    n2, _ = orc.forecast_speculative(tgt, drf, s, 4 * P, 5 * P, 2, 1.0, 11, variant=v)
+    n3, _ = orc.forecast_speculative(tgt, drf, s, 4 * P, 5 * P, 2, 1.0, 12, variant=v)
+    np.testing.assert_array_equal(n1, n2)
+    assert not np.allclose(n1, base) and not np.allclose(n1, n3)
+    # a series decoded alone (same series id) sees the same noise as inside the batch
+    solo, _ = orc.forecast_speculative(tgt, drf, s[1:2], 4 * P, 5 * P, 2, 1.0, 11, variant=v, series_index0=1)
+    np.testing.assert_array_equal(solo[0], n1[1])
