@@ -163,6 +163,27 @@ int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx
                        int32_t H, int32_t K, float tau, uint64_t seed,
                        float *out, tsfm_stats *stats);
 
+/* The general form of the rule (Sec. 3.3 "Fallback Correction and Sampled Variants", Algorithm 1
+ * with r > 0; component ablation of Table 2).  The deployed scheme is tsfm_spec_forecast: mean
+ * proposals, r = 0, sigma_q = sigma_p = tau, 1/d tempering.
+ *   sigma_q           draft surrogate scale of Eq. 5; 0 = same as tau (determinant term vanishes)
+ *   fallback_noise    r >= 0: correction and bonus patches are mu_p + r eps
+ *   sample_proposals  nonzero: x_i = mu_q^(i) + sigma_q eps, the draft continues from the sampled x_i
+ *   no_tempering      nonzero: drop the 1/d factor of the statistic
+ * eps are standard normals from the same Philox key: Box-Muller on the words of counter
+ * (series, round, position, stream | element / 2), stream 0x10000000 for proposals and 0x20000000
+ * for the fallback, cosine branch for even elements, sine for odd.  variant == NULL is the deployed
+ * scheme.  Noise is not available with TSFM_GEMM_FUSED_PASS (TSFM_ERR_ARG). */
+typedef struct {
+  float   sigma_q;
+  float   fallback_noise;
+  int32_t sample_proposals;
+  int32_t no_tempering;
+} tsfm_variant;
+int tsfm_spec_forecast_variant(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len,
+                               int32_t H, int32_t K, float tau, uint64_t seed,
+                               const tsfm_variant *variant, float *out, tsfm_stats *stats);
+
 /* Target-only decoding (Eq. 1): T sequential one-token target passes.  Same argument
  * meaning as above; only the timing fields, rounds (= T) and patches_committed of `stats`
  * are filled. */

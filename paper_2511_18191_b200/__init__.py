@@ -5,5 +5,5 @@ marshals arguments.  Importing it without the built library raises ImportError.
 """
 from .binding import *  # noqa: F401,F403
 from .binding import (  # noqa: F401
-    SpecDecoder, TsfmError, EXPORTS, lib, pack_weights, tsfm_arch, tsfm_cfg, tsfm_stats, tsfm_weights,
+    SpecDecoder, TsfmError, EXPORTS, lib, pack_weights, tsfm_arch, tsfm_cfg, tsfm_stats, tsfm_variant, tsfm_weights,
 )

@@ -23,7 +23,7 @@ TSFM_EXEC_GRAPH, TSFM_EXEC_STREAM, TSFM_EXEC_NO_PDL = 0, 1, 2
 TSFM_MAX_K = 32
 
 EXPORTS = [
-    "tsfm_weights_bytes", "tsfm_weights_offset", "tsfm_spec_create", "tsfm_spec_forecast",
+    "tsfm_weights_bytes", "tsfm_weights_offset", "tsfm_spec_create", "tsfm_spec_forecast", "tsfm_spec_forecast_variant",
     "tsfm_target_only_forecast", "tsfm_draft_only_forecast", "tsfm_spec_forecast_host", "tsfm_target_only_forecast_host",
     "tsfm_spec_last_trace", "tsfm_accept_round", "tsfm_model_forward", "tsfm_gemm_bf16", "tsfm_gemm_bf16_static",
     "tsfm_spec_set_profiling", "tsfm_spec_kernel_profile", "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
@@ -65,6 +65,11 @@ class tsfm_stats(C.Structure):
         return d
 
 
+class tsfm_variant(C.Structure):
+    _fields_ = [("sigma_q", C.c_float), ("fallback_noise", C.c_float), ("sample_proposals", C.c_int32),
+                ("no_tempering", C.c_int32)]
+
+
 class tsfm_kernel_stat(C.Structure):
     _fields_ = [("name", C.c_char * 24), ("launches", C.c_int64), ("ms_total", C.c_double),
                 ("bytes", C.c_double), ("flops", C.c_double)]
@@ -87,6 +92,9 @@ def _load() -> C.CDLL:
         fn = getattr(lib, name)
         fn.restype = C.c_int
         fn.argtypes = [vp, vp, i32, i32, i32, i32, f32, u64, vp, C.POINTER(tsfm_stats)]
+    lib.tsfm_spec_forecast_variant.restype = C.c_int
+    lib.tsfm_spec_forecast_variant.argtypes = [vp, vp, i32, i32, i32, i32, f32, u64, C.POINTER(tsfm_variant), vp,
+                                               C.POINTER(tsfm_stats)]
     for name in ("tsfm_target_only_forecast", "tsfm_draft_only_forecast", "tsfm_target_only_forecast_host"):
         fn = getattr(lib, name)
         fn.restype = C.c_int
@@ -205,6 +213,13 @@ def tsfm_spec_destroy(h: int) -> None:
 def tsfm_spec_forecast(h, series, B, ctx_len, H, K, tau, seed, out, stats: Optional[tsfm_stats] = None) -> None:
     _check(lib.tsfm_spec_forecast(h, _ptr(series), B, ctx_len, H, K, tau, seed, _ptr(out),
                                   C.byref(stats) if stats is not None else None), "tsfm_spec_forecast")
+
+
+def tsfm_spec_forecast_variant(h, series, B, ctx_len, H, K, tau, seed, variant: Optional[tsfm_variant], out,
+                               stats: Optional[tsfm_stats] = None) -> None:
+    _check(lib.tsfm_spec_forecast_variant(h, _ptr(series), B, ctx_len, H, K, tau, seed,
+                                          C.byref(variant) if variant is not None else None, _ptr(out),
+                                          C.byref(stats) if stats is not None else None), "tsfm_spec_forecast_variant")
 
 
 def tsfm_target_only_forecast(h, series, B, ctx_len, H, out, stats: Optional[tsfm_stats] = None) -> None:
@@ -332,13 +347,17 @@ class SpecDecoder:
         except Exception:
             pass
 
-    def forecast(self, series, H: int, K: int, tau: float, seed: int, out=None, stats: bool = True):
+    def forecast(self, series, H: int, K: int, tau: float, seed: int, out=None, stats: bool = True,
+                 variant: Optional[tsfm_variant] = None):
         """series: CUDA float32 [B, ctx_len]. Returns (out [B, H] CUDA, tsfm_stats | None)."""
         B, ctx_len = series.shape
         if out is None:
             out = self.torch.empty((B, H), dtype=self.torch.float32, device=series.device)
         st = tsfm_stats() if stats else None
-        tsfm_spec_forecast(self.h, series, B, ctx_len, H, K, tau, seed, out, st)
+        if variant is None:
+            tsfm_spec_forecast(self.h, series, B, ctx_len, H, K, tau, seed, out, st)
+        else:
+            tsfm_spec_forecast_variant(self.h, series, B, ctx_len, H, K, tau, seed, variant, out, st)
         return out, st
 
     def target_only(self, series, H: int, out=None, stats: bool = True):

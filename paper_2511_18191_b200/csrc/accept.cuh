@@ -25,6 +25,23 @@ __device__ __forceinline__ float uniform_from_word(uint32_t w) {
   return ((float)(w >> 9) + 0.5f) * 1.1920928955078125e-07f;
 }
 
+// Standard normal draw for element e of a patch, for the sampled variants of Sec. 3.3: Box-Muller
+// on the Philox words of counter (series, round, position, stream | e / 2); the even element takes
+// the cosine branch, the odd one the sine branch.
+constexpr uint32_t NOISE_PROPOSAL = 0x10000000u, NOISE_FALLBACK = 0x20000000u;
+__device__ __forceinline__ float standard_normal(uint2 key, uint32_t series, uint32_t round, uint32_t pos,
+                                                 uint32_t stream, int e) {
+  const uint4 w = philox4x32_10(make_uint4(series, round, pos, stream | (uint32_t)(e >> 1)), key);
+  const float rad = sqrtf(-2.f * logf(uniform_from_word(w.x)));
+  float sn, cs;
+  sincospif(2.f * uniform_from_word(w.y), &sn, &cs);
+  return rad * ((e & 1) ? sn : cs);
+}
+
+__device__ float head_normal(const DevState *st, int series, int k_pos, int e) {
+  return standard_normal(make_uint2(st->key0, st->key1), (uint32_t)series, (uint32_t)st->round, (uint32_t)k_pos, NOISE_PROPOSAL, e);
+}
+
 struct AcceptCounters {            // device mirror of the integer part of tsfm_stats
   unsigned long long drafted, tested, accepted, committed, near_margin;
   unsigned long long tested_by_pos[32], accepted_by_pos[32], L_hist[34];
@@ -35,6 +52,9 @@ struct AcceptArgs {
   // element (b, i, :) at x + b * x_stride_b + i * P   (i = 0..K-1)
   const float *x, *mu_q;
   long long x_stride_b;
+  // where the draft means live when they are not the proposals themselves (sampled proposals):
+  // element (b, i, :) at mu_q_alt + (b * K + i) * P; NULL = use mu_q as above
+  const float *mu_q_alt;
   const float *mu_p;               // [B, K+1, P] boundary predictions
   // where committed patches go: patch c of this round (c = 0..n) at
   // commit + b * commit_stride_b + c * P.  When commit_accepted == 0 the accepted
@@ -87,7 +107,8 @@ __global__ void __launch_bounds__(128) accept_kernel(AcceptArgs a) {
   if (a.st) {
     if (blockIdx.x == 0 && threadIdx.x == 0) a.st->t_phase[2] = globaltimer_ns();
     const int r = a.st->round;
-    a.sigma_p = a.sigma_q = a.st->tau;
+    a.sigma_p = a.st->tau;
+    a.sigma_q = a.st->sigma_q;
     a.key = make_uint2(a.st->key0, a.st->key1);
     a.round_idx = r;
     if (a.n_accept) a.n_accept += (size_t)r * a.B;
@@ -104,7 +125,10 @@ __global__ void __launch_bounds__(128) accept_kernel(AcceptArgs a) {
   const int K = a.K, P = a.P;
   const long long hist_adv = a.commit_follows_done ? (long long)m * P : 0;
   const float *xb = a.x + b * a.x_stride_b + hist_adv;
-  const float *qb = a.mu_q + b * a.x_stride_b + hist_adv;
+  const int flags = a.st ? a.st->flags : 0;
+  const float fallback_r = a.st ? a.st->fallback_r : 0.f;
+  const float *qb = (a.mu_q_alt && (flags & VAR_SAMPLE_PROPOSALS)) ? a.mu_q_alt + (size_t)b * a.K * a.P
+                                                                     : a.mu_q + b * a.x_stride_b + hist_adv;
   const float *pb = a.mu_p + (size_t)b * (K + 1) * P;
 
   // energies ||x - mu_p||_d^2 and ||x - mu_q||_d^2 of every position; lane i keeps position i
@@ -128,6 +152,7 @@ __global__ void __launch_bounds__(128) accept_kernel(AcceptArgs a) {
   if (lane < K) {
     l = -my_ep / (2.f * a.sigma_p * a.sigma_p) + my_eq / (2.f * a.sigma_q * a.sigma_q)
         + 0.5f * logf((a.sigma_q * a.sigma_q) / (a.sigma_p * a.sigma_p));
+    if (flags & VAR_NO_TEMPERING) l *= (float)P;     // l is (1/d) log p/q: undo the 1/d (component ablation)
     float u;
     if (a.forced_u) u = a.forced_u[(size_t)b * K + lane];
     else u = uniform_from_word(philox4x32_10(
@@ -146,7 +171,12 @@ __global__ void __launch_bounds__(128) accept_kernel(AcceptArgs a) {
   float *cb = a.commit + b * a.commit_stride_b + hist_adv;
   if (a.commit_accepted)
     for (int c = lane; c < n * P; c += 32) cb[c] = xb[c];
-  for (int c = lane; c < P; c += 32) cb[(size_t)n * P + c] = pb[(size_t)n * P + c];
+  for (int c = lane; c < P; c += 32) {
+    float t = pb[(size_t)n * P + c];
+    if (fallback_r != 0.f)                          // t = mu_p + r eps (Algorithm 1, correction and bonus)
+      t += fallback_r * standard_normal(a.key, (uint32_t)(a.series0 + b), (uint32_t)a.round_idx, (uint32_t)n, NOISE_FALLBACK, c);
+    cb[(size_t)n * P + c] = t;
+  }
 
   const bool tested = lane < min(n + 1, K);
   const bool near = tested && fabsf(l - lu) < a.margin;

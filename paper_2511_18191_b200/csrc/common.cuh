@@ -17,7 +17,10 @@ enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_E
 struct DevState {
   const float *series;            // [B, ctx_len] raw context values
   float *out;                     // [B, H] forecast
-  float tau;                      // acceptance temperature (the paper's sigma)
+  float tau;                      // acceptance temperature (the paper's sigma; sigma_p of Eq. 5)
+  float sigma_q;                  // draft surrogate scale (= tau in the deployed scheme)
+  float fallback_r;               // r of t = mu_p + r eps (0 in the deployed scheme)
+  int flags;                      // VAR_* bits
   uint32_t key0, key1;            // Philox key = forecast seed
   int round;                      // index of the round in flight
   unsigned long long t_call;      // %globaltimer stamps: call start, ...
@@ -25,6 +28,8 @@ struct DevState {
   unsigned long long t_end;
   unsigned long long ns_prefill, ns_draft, ns_verify, ns_accept;   // accumulated phase times
 };
+
+enum : int { VAR_SAMPLE_PROPOSALS = 1, VAR_NO_TEMPERING = 2 };
 
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
   unsigned long long t;

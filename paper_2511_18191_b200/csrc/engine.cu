@@ -138,6 +138,7 @@ struct tsfm_spec {
   void *a = nullptr, *ao = nullptr, *hbuf = nullptr;
   // decoding state
   float *hist = nullptr, *vout = nullptr, *mean = nullptr, *sd = nullptr;
+  float *muq = nullptr;                  // [B][max_K][P] draft means of the round (sampled proposals)
   int *done = nullptr;
   AcceptCounters *ctr = nullptr;
   int *unfinished = nullptr;             // [max_T + 1]
@@ -401,10 +402,14 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
 
 enum { HEAD_NONE = 0, HEAD_LAST_TO_HIST = 1, HEAD_ALL_TO_VOUT = 2 };
 
+// Draft step i of a round (k_pos = i - 1): lets the head kernel turn its mean into a sampled
+// proposal when the call asks for one (Sec. 3.3); target and prefill passes carry none.
+struct DraftStep { int k_pos = -1, K = 0; };
+
 // One causal pass of a model over q_len new tokens per series (appends to its KV cache).
 template <typename T>
 void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout,
-              unsigned long long *stamp) {
+              unsigned long long *stamp, DraftStep ds) {
   const int M = B * g.q_len, d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len;
   cudaStream_t s = h->ls;
   const float eps = h->cfg.rms_eps;
@@ -457,10 +462,11 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
             2.0 * rows * P * d);
   if (head_mode == HEAD_LAST_TO_HIST) {
     launch_ex(s, h->pdl, head_kernel<T>, dim3(B, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
-              (const T *)m.W_head, d, P, eps, g, 1, h->hist, nullptr);
+              (const T *)m.W_head, d, P, eps, g, 1, h->hist, (float *)nullptr,
+              ds.k_pos >= 0 ? (const DevState *)h->st : (const DevState *)nullptr, h->muq, ds.k_pos, ds.K);
   } else if (head_mode == HEAD_ALL_TO_VOUT) {
     launch_ex(s, h->pdl, head_kernel<T>, dim3(M, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
-              (const T *)m.W_head, d, P, eps, g, 0, nullptr, vout);
+              (const T *)m.W_head, d, P, eps, g, 0, (float *)nullptr, vout, (const DevState *)nullptr, (float *)nullptr, 0, 0);
   }
 }
 
@@ -496,11 +502,11 @@ bool pass_fused(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mo
 }
 
 void pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout = nullptr,
-          unsigned long long *stamp = nullptr) {
+          unsigned long long *stamp = nullptr, DraftStep ds = DraftStep{}) {
   if (g.q_len < 1) return;
   if (pass_fused(h, m, B, g, head_mode, vout, stamp)) return;
-  if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout, stamp);
-  else run_pass<float>(h, m, B, g, head_mode, vout, stamp);
+  if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout, stamp, ds);
+  else run_pass<float>(h, m, B, g, head_mode, vout, stamp, ds);
 }
 
 int check_call(tsfm_spec *h, const float *series, int B, int ctx_len, int H, float *out, int K) {
@@ -557,15 +563,17 @@ void enqueue_round(tsfm_spec *h, int B, int N, int T, int K, cudaGraphConditiona
   const int P = h->cfg.patch_len;
   // step 1 re-ingests the last two committed patches (the draft cache may lack the last
   // accepted proposal), steps 2..K ingest the previous proposal
-  pass(h, h->drf, B, PassGeom{h->done, N - 2, 2, h->cap}, HEAD_LAST_TO_HIST, nullptr, &h->st->t_phase[0]);
+  pass(h, h->drf, B, PassGeom{h->done, N - 2, 2, h->cap}, HEAD_LAST_TO_HIST, nullptr, &h->st->t_phase[0], DraftStep{0, K});
   for (int i = 2; i <= K; ++i)
-    pass(h, h->drf, B, PassGeom{h->done, N - 1 + (i - 1), 1, h->cap}, HEAD_LAST_TO_HIST);
+    pass(h, h->drf, B, PassGeom{h->done, N - 1 + (i - 1), 1, h->cap}, HEAD_LAST_TO_HIST, nullptr, nullptr,
+         DraftStep{i - 1, K});
   // single-pass verification over [pending, x_1..x_K]
   pass(h, h->tgt, B, PassGeom{h->done, N - 1, K + 1, h->cap}, HEAD_ALL_TO_VOUT, h->vout, &h->st->t_phase[1]);
 
   AcceptArgs a{};
   a.x = a.mu_q = h->hist + (size_t)N * P;       // slot N + done[b] holds x_1
   a.x_stride_b = (long long)h->cap * P;
+  a.mu_q_alt = h->muq;                          // used only when the call samples its proposals
   a.mu_p = h->vout;
   a.commit = h->hist + (size_t)N * P;
   a.commit_stride_b = a.x_stride_b;
@@ -694,11 +702,15 @@ int get_graph(tsfm_spec *h, const GraphKey &k, GraphInfo *info) {
 
 // Writes the call parameters and clears the loop state.  The source is an ordinary host
 // struct: for pageable memory the copy is staged before the call returns.
-int write_call_state(tsfm_spec *h, const float *series, float *out, float tau, uint64_t seed) {
+int write_call_state(tsfm_spec *h, const float *series, float *out, float tau, uint64_t seed,
+                     const tsfm_variant *v = nullptr) {
   DevState st{};
   st.series = series;
   st.out = out;
   st.tau = tau;
+  st.sigma_q = v && v->sigma_q > 0.f ? v->sigma_q : tau;
+  st.fallback_r = v ? v->fallback_noise : 0.f;
+  st.flags = v ? (v->sample_proposals ? VAR_SAMPLE_PROPOSALS : 0) | (v->no_tempering ? VAR_NO_TEMPERING : 0) : 0;
   st.key0 = (uint32_t)(seed & 0xffffffffu);
   st.key1 = (uint32_t)(seed >> 32);
   CU_TRY(cudaMemcpyAsync(h->st, &st, sizeof(st), cudaMemcpyHostToDevice, h->stream));
@@ -859,6 +871,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   if ((rc = dev_alloc(h, (char **)&h->hbuf, Mx * fmax * e))) return fail(rc);
   if ((rc = dev_alloc(h, &h->hist, (size_t)Bm * h->cap * P))) return fail(rc);
   if ((rc = dev_alloc(h, &h->vout, (size_t)Bm * (cfg->max_K + 1) * P))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->muq, (size_t)Bm * cfg->max_K * P))) return fail(rc);
   if ((rc = dev_alloc(h, &h->mean, Bm))) return fail(rc);
   if ((rc = dev_alloc(h, &h->sd, Bm))) return fail(rc);
   if ((rc = dev_alloc(h, &h->done, Bm))) return fail(rc);
@@ -955,13 +968,26 @@ int tsfm_draft_only_forecast(tsfm_spec *h, const float *series, int32_t B, int32
 
 int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H, int32_t K,
                        float tau, uint64_t seed, float *out, tsfm_stats *stats) {
+  return tsfm_spec_forecast_variant(h, series, B, ctx_len, H, K, tau, seed, nullptr, out, stats);
+}
+
+int tsfm_spec_forecast_variant(tsfm_spec *h, const float *series, int32_t B, int32_t ctx_len, int32_t H, int32_t K,
+                               float tau, uint64_t seed, const tsfm_variant *variant, float *out,
+                               tsfm_stats *stats) {
   if (K < 1) return TSFM_ERR_ARG;
   if (!(tau > 0.f) || !std::isfinite(tau)) return TSFM_ERR_ARG;
+  if (variant) {
+    if (!std::isfinite(variant->sigma_q) || variant->sigma_q < 0.f || !std::isfinite(variant->fallback_noise) ||
+        variant->fallback_noise < 0.f)
+      return TSFM_ERR_ARG;
+    if (h && h->use_cluster && (variant->sample_proposals || variant->fallback_noise != 0.f))
+      return TSFM_ERR_ARG;             // the whole-pass cluster kernel has no noise path
+  }
   if (int rc = check_call(h, series, B, ctx_len, H, out, K)) return rc;
   const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
   cudaStream_t s = h->stream;
   if (stats) CU_TRY(cudaEventRecord(h->ev[0], s));
-  if (int rc = write_call_state(h, series, out, tau, seed)) return rc;
+  if (int rc = write_call_state(h, series, out, tau, seed, variant)) return rc;
   if (use_graph(h)) {
     // one launch: prologue, WHILE(rounds), de-normalisation; no host round trip
     GraphInfo gi;

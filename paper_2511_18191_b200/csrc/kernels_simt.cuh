@@ -622,11 +622,13 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
 //   history slot hist[b, pos0 + q_len, :]  (draft steps, target-only steps);
 // only_last = 0: every token, written to vout[b, j, :]  (verification; vout [B, q_len, P]).
 // ----------------------------------------------------------------------------------
+__device__ float head_normal(const DevState *st, int series, int k_pos, int e);   // accept.cuh
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T *__restrict__ Wh, int d,
             int P, float eps, PassGeom g, int only_last, float *__restrict__ hist,
-            float *__restrict__ vout) {
+            float *__restrict__ vout, const DevState *__restrict__ st, float *__restrict__ muq, int k_pos, int K) {
   extern __shared__ __align__(16) float xs[];
   __shared__ float red[32];
   pdl_sync();
@@ -658,7 +660,14 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
     for (int c = 0; c < V; ++c) acc = fmaf(wv[c], xs[i + c], acc);
   }
   acc = warp_sum(acc);
-  if (lane == 0) dst[p] = acc;
+  if (lane == 0) {
+    if (only_last && st && (st->flags & VAR_SAMPLE_PROPOSALS)) {
+      // sampled proposal x = mu_q + sigma_q eps (Sec. 3.3); the mean is kept for the statistic
+      muq[((size_t)b * K + k_pos) * P + p] = acc;
+      acc += st->sigma_q * head_normal(st, b, k_pos, p);
+    }
+    dst[p] = acc;
+  }
 }
 
 }  // namespace tsfm

@@ -40,7 +40,8 @@ def gpu_decisions(n_accept: np.ndarray, K: int, b: int):
     return rounds
 
 
-def compare_forecast(wl, target, draft, series, H, K, tau, seed, gpu_out, gpu_nacc, series_ids, dtype=None):
+def compare_forecast(wl, target, draft, series, H, K, tau, seed, gpu_out, gpu_nacc, series_ids, dtype=None,
+                     variant=None):
     """Compare GPU results for the series in `series_ids` with the oracle.
 
     Returns a dict with the value error, the number of decisions compared, the number of
@@ -60,7 +61,8 @@ def compare_forecast(wl, target, draft, series, H, K, tau, seed, gpu_out, gpu_na
         # the GPU's rounds must cover the horizon exactly
         L = [sum(f) + 1 for f in forced[0]]
         assert sum(L[:-1]) < T <= sum(L), f"series {b}: GPU rounds {L} do not cover T={T}"
-        out, tr = orc.forecast_speculative(target, draft, s, ctx, H, K, tau, seed, forced=forced, series_index0=b)
+        out, tr = orc.forecast_speculative(target, draft, s, ctx, H, K, tau, seed, forced=forced, series_index0=b,
+                                           variant=variant)
         for r, rec in enumerate(tr.rounds[0]):
             for i, (ell, lu, dec) in enumerate(zip(rec.ell, rec.log_u, rec.decisions)):
                 natural = lu <= min(ell, 0.0)

@@ -171,6 +171,43 @@ def test_edge_geometries_fp32(K, H, ctx_patches, B):
         assert res["stats"]["rounds"] <= -(-H // 96)
 
 
+@pytest.mark.parametrize("name,kw", [
+    ("unequal_scales", dict(sigma_q=0.6)),
+    ("sampled_proposals", dict(sample_proposals=1)),
+    ("fallback_noise", dict(fallback_noise=0.3)),
+    ("all_knobs", dict(sigma_q=0.8, fallback_noise=0.2, sample_proposals=1)),
+    ("no_tempering", dict(no_tempering=1)),
+])
+@pytest.mark.parametrize("wl_name", ["C0", "C1"])
+def test_general_rule_variants_match_oracle(wl_name, name, kw):
+    """Sec. 3.3's sampled variants and Table 2's tempering ablation through the forecast call: sampled
+    proposals (the draft continues from the sampled patch), fallback / bonus noise, sigma_q != sigma_p."""
+    import paper_2511_18191_b200 as tsfm
+    wl = workload("C0", batch=5, series_recipe="c1") if wl_name == "C0" else workload("C1", batch=6)
+    K, tau, seed = wl.K, 1.5, 17
+    dec, tw, dw = make_decoder(wl, batch=wl.batch)
+    s, ctx = series_on_device(wl, wl.batch)
+    v = tsfm.tsfm_variant(kw.get("sigma_q", 0.0), kw.get("fallback_noise", 0.0), kw.get("sample_proposals", 0),
+                          kw.get("no_tempering", 0))
+    base, _ = dec.forecast(ctx, wl.horizon, K, tau, seed)
+    out, st = dec.forecast(ctx, wl.horizon, K, tau, seed, variant=v)
+    d = check_stats(st, wl.batch, wl.n_patches, K)
+    nacc, ell, logu = dec.last_trace(wl.batch, K)
+    # replaying the default scheme afterwards on the same handle is unaffected by the variant call
+    again, _ = dec.forecast(ctx, wl.horizon, K, tau, seed)
+    np.testing.assert_array_equal(base.cpu().numpy(), again.cpu().numpy())
+    dec.close()
+    tm, dm = parity.oracle_models(wl, tw, dw)
+    var = orc.Variant(sigma_q=kw.get("sigma_q") or None, sample_proposals=bool(kw.get("sample_proposals", 0)),
+                      fallback_noise=kw.get("fallback_noise", 0.0), tempering=not kw.get("no_tempering", 0))
+    res = parity.compare_forecast(wl, tm, dm, s, wl.horizon, K, tau, seed, out.cpu().numpy(), nacc, range(wl.batch),
+                                  variant=var)
+    if name != "unequal_scales":
+        assert not np.allclose(out.cpu().numpy(), base.cpu().numpy())
+    if name == "no_tempering":
+        assert d["proposals_accepted"] == 0                     # acceptance collapses without the 1/d
+
+
 def test_tiny_tau_recovers_target_only_and_result_is_independent_of_batch_composition():
     wl = workload("C1")
     dec, tw, dw = make_decoder(wl)
