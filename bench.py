@@ -214,7 +214,10 @@ def throughput_law(stats, to_stats, K, T):
     c = stats["ms_draft"] / (rounds * K) / step
     v = stats["ms_verify"] / rounds / step
     e_l = float(K + 1) if alpha >= 1.0 else (1.0 - alpha ** (K + 1)) / (1.0 - alpha)
-    return {"alpha": alpha, "c": c, "v": v, "E_L": e_l, "predicted_speedup": e_l / (c * K + v)}
+    import paper_2511_18191_b200 as tsfm
+    k_star, s_star = tsfm.tsfm_advise_block_size(alpha, c, v, 32)
+    return {"alpha": alpha, "c": c, "v": v, "E_L": e_l, "predicted_speedup": e_l / (c * K + v),
+            "advised_K": k_star, "predicted_speedup_at_advised_K": s_star}
 
 
 # ------------------------------------------------------------------ our arm

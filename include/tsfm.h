@@ -284,6 +284,15 @@ typedef struct {
 int tsfm_spec_set_profiling(tsfm_spec *h, int32_t enable);
 int tsfm_spec_kernel_profile(tsfm_spec *h, int32_t cap, int32_t *n, tsfm_kernel_stat *out);
 
+/* Block-size advice from measured quantities (host arithmetic only).  alpha = conditional
+ * acceptance rate, c = draft step cost and v = verification pass cost in units of one target step.
+ * Expected yield E[L_K] = sum_{j=0..K} alpha^j (Eq. 7), predicted speedup S(K) = E[L_K] / (c K + v)
+ * (Eq. 8).  Steps K up from 1 while the marginal-gain condition alpha^(K+1) (c K + v) >= c E[L_K]
+ * of the block-size proposition holds (it is equivalent to S(K+1) >= S(K)) and returns the K reached,
+ * at most max_K; *speedup (nullable) receives S at that K.  Returns 0 on invalid arguments
+ * (alpha outside [0, 1], c <= 0, v <= 0, max_K < 1). */
+int32_t tsfm_advise_block_size(double alpha, double c, double v, int32_t max_K, double *speedup);
+
 int tsfm_spec_destroy(tsfm_spec *h);
 
 /* Number of kernels this library has launched in this process (all handles, all streams).  The

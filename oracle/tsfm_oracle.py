@@ -443,3 +443,19 @@ def capped_geometric_mean(alpha: float, K: int) -> float:
 def predicted_speedup(alpha: float, K: int, c: float, v: float) -> float:
     """S(K) = E[L] / (c K + v)."""
     return capped_geometric_mean(alpha, K) / (c * K + v)
+
+
+def marginal_gain_holds(alpha: float, K: int, c: float, v: float) -> bool:
+    """Marginal-gain condition (appendix proposition on block-size selection):
+    S(K+1) >= S(K)  iff  alpha^(K+1) (c K + v) >= c E[L_K]."""
+    return alpha ** (K + 1) * (c * K + v) >= c * capped_geometric_mean(alpha, K)
+
+
+def best_block_size(alpha: float, c: float, v: float, max_K: int) -> int:
+    """argmax over K = 1..max_K of S(K) = E[L_K] / (c K + v), by brute force (smallest K on ties)."""
+    best, best_s = 1, -1.0
+    for K in range(1, max_K + 1):
+        s_k = predicted_speedup(alpha, K, c, v)
+        if s_k > best_s * (1.0 + 1e-15):
+            best, best_s = K, s_k
+    return best

@@ -26,7 +26,7 @@ EXPORTS = [
     "tsfm_weights_bytes", "tsfm_weights_offset", "tsfm_spec_create", "tsfm_spec_forecast", "tsfm_spec_forecast_variant",
     "tsfm_target_only_forecast", "tsfm_draft_only_forecast", "tsfm_spec_forecast_host", "tsfm_target_only_forecast_host",
     "tsfm_spec_last_trace", "tsfm_accept_round", "tsfm_model_forward", "tsfm_gemm_bf16", "tsfm_gemm_bf16_static",
-    "tsfm_spec_set_profiling", "tsfm_spec_kernel_profile", "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
+    "tsfm_spec_set_profiling", "tsfm_spec_kernel_profile", "tsfm_advise_block_size", "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
 ]
 
 
@@ -113,6 +113,8 @@ def _load() -> C.CDLL:
     lib.tsfm_spec_set_profiling.argtypes = [vp, i32]
     lib.tsfm_spec_kernel_profile.restype = C.c_int
     lib.tsfm_spec_kernel_profile.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(tsfm_kernel_stat)]
+    lib.tsfm_advise_block_size.restype = C.c_int32
+    lib.tsfm_advise_block_size.argtypes = [C.c_double, C.c_double, C.c_double, i32, C.POINTER(C.c_double)]
     lib.tsfm_spec_destroy.restype = C.c_int
     lib.tsfm_spec_destroy.argtypes = [vp]
     lib.tsfm_launch_count.restype = C.c_int64
@@ -293,6 +295,13 @@ def tsfm_spec_kernel_profile(h):
     _check(lib.tsfm_spec_kernel_profile(h, 32, C.byref(n), arr), "tsfm_spec_kernel_profile")
     return {arr[i].name.decode(): dict(launches=arr[i].launches, ms_total=arr[i].ms_total, bytes=arr[i].bytes,
                                        flops=arr[i].flops) for i in range(n.value)}
+
+
+def tsfm_advise_block_size(alpha: float, c: float, v: float, max_K: int):
+    """(K, predicted speedup) by the marginal-gain rule; K == 0 on invalid arguments."""
+    s = C.c_double(0.0)
+    k = int(lib.tsfm_advise_block_size(alpha, c, v, max_K, C.byref(s)))
+    return k, s.value
 
 
 def tsfm_launch_count() -> int:

@@ -1239,6 +1239,19 @@ int tsfm_spec_kernel_profile(tsfm_spec *h, int32_t cap, int32_t *n, tsfm_kernel_
   return k <= cap ? TSFM_OK : TSFM_ERR_ARG;
 }
 
+int32_t tsfm_advise_block_size(double alpha, double c, double v, int32_t max_K, double *speedup) {
+  if (!(alpha >= 0.0 && alpha <= 1.0) || !(c > 0.0) || !(v > 0.0) || max_K < 1) return 0;
+  int K = 1;
+  double EL = 1.0 + alpha, pw = alpha * alpha;      // E[L_1], alpha^(K+1) at K = 1
+  while (K < max_K && pw * (c * K + v) >= c * EL) {
+    EL += pw;                                        // E[L_{K+1}] = E[L_K] + alpha^(K+1)
+    pw *= alpha;
+    ++K;
+  }
+  if (speedup) *speedup = EL / (c * K + v);
+  return K;
+}
+
 int64_t tsfm_launch_count(void) {
   long long n = g_launches.load();
   std::lock_guard<std::mutex> lock(g_handles_mu);

@@ -79,6 +79,21 @@ def test_argument_validation_needs_no_device_and_never_falls_back():
         assert rc in (tsfm.TSFM_ERR_CUDA, tsfm.TSFM_ERR_ARCH) and not h.value
 
 
+def test_block_size_advice_agrees_with_the_oracle_rule():
+    import paper_2511_18191_b200 as tsfm
+    from oracle import tsfm_oracle as orc
+    for alpha in (0.0, 0.2, 0.6, 0.9, 0.99, 1.0):
+        for c in (0.04, 0.25, 1.0):
+            for v in (1.0, 1.44, 2.5):
+                k, s = tsfm.tsfm_advise_block_size(alpha, c, v, 32)
+                best = orc.best_block_size(alpha, c, v, 32)
+                assert s == pytest.approx(orc.predicted_speedup(alpha, k, c, v), rel=1e-12)
+                assert s == pytest.approx(orc.predicted_speedup(alpha, best, c, v), rel=1e-9)
+    assert tsfm.tsfm_advise_block_size(1.5, 0.1, 1.0, 8)[0] == 0
+    assert tsfm.tsfm_advise_block_size(0.5, 0.0, 1.0, 8)[0] == 0
+    assert tsfm.tsfm_advise_block_size(0.5, 0.1, 1.0, 0)[0] == 0
+
+
 def test_product_never_imports_the_oracle():
     pkg = os.path.join(ROOT, "paper_2511_18191_b200")
     for dirpath, _, files in os.walk(pkg):

@@ -412,3 +412,20 @@ def test_variant_defaults_reproduce_the_deployed_scheme_and_noise_is_seeded():
     # a series decoded alone (same series id) sees the same noise as inside the batch
     solo, _ = orc.forecast_speculative(tgt, drf, s[1:2], 4 * P, 5 * P, 2, 1.0, 11, variant=v, series_index0=1)
     np.testing.assert_array_equal(solo[0], n1[1])
+
+
+def test_marginal_gain_condition_is_equivalent_to_a_speedup_gain_and_finds_the_best_block():
+    """Prop. (marginal-gain condition for K): S(K+1) >= S(K) iff alpha^(K+1)(cK+v) >= c E[L_K];
+    stepping K up while it holds lands on the brute-force argmax of Eq. 8."""
+    for alpha in (0.05, 0.3, 0.6, 0.8, 0.95, 0.999):
+        for c in (0.02, 0.1, 0.25, 0.5, 1.0):
+            for v in (1.0, 1.4, 2.5):
+                K = 1
+                while K < 32 and orc.marginal_gain_holds(alpha, K, c, v):
+                    K += 1
+                for k in range(1, 12):
+                    lhs = orc.predicted_speedup(alpha, k + 1, c, v) >= orc.predicted_speedup(alpha, k, c, v) * (1 - 1e-12)
+                    assert lhs == orc.marginal_gain_holds(alpha, k, c, v) or \
+                        abs(orc.predicted_speedup(alpha, k + 1, c, v) - orc.predicted_speedup(alpha, k, c, v)) < 1e-12
+                best = orc.best_block_size(alpha, c, v, 32)
+                assert orc.predicted_speedup(alpha, K, c, v) == pytest.approx(orc.predicted_speedup(alpha, best, c, v), rel=1e-12)
