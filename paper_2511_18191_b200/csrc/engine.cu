@@ -17,6 +17,7 @@
 
 #include "common.cuh"
 #include "kernels_simt.cuh"
+#include "attn_flash.cuh"
 #include "accept.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_sk.cuh"
@@ -288,17 +289,38 @@ int make_cluster_plan(tsfm_spec *h, ModelDev &m) {
 template <typename T> size_t attn_smem_bytes(int dh, int nk) {
   const int vw = AttnWords<T>::per_row(dh);
   return (size_t)nk * (2 * vw + 1) * 4 + (size_t)ATTN_QT * nk * sizeof(float) + (size_t)5 * ATTN_QT * dh * sizeof(float) +
-         ATTN_QT * sizeof(float);
+         2 * ATTN_QT * sizeof(float);
 }
+
+// Number of CTAs (one cluster) that share the keys of one (series, head, query tile): long rows
+// are split so that each CTA stages a quarter of the cache and more CTAs fit on an SM.
+#ifndef TSFM_ATTN_SKV
+#define TSFM_ATTN_SKV 4
+#endif
+#ifndef TSFM_ATTN_SKV_MIN_CAP
+#define TSFM_ATTN_SKV_MIN_CAP 192
+#endif
+inline int attn_key_split(int cap) { return cap >= TSFM_ATTN_SKV_MIN_CAP ? TSFM_ATTN_SKV : 1; }
+// key rows one CTA must hold: its share of the longest row, in whole 16-key MMA blocks
+inline int attn_rows_per_cta(int cap, int skv) { return ((cap + skv - 1) / skv + 15) & ~15; }
 
 template <typename T, int DH>
 int attn_set_attr(size_t bytes) {
   CU_TRY(cudaFuncSetAttribute(attn_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
   return TSFM_OK;
 }
+// Rows of at least this many keys (bf16 caches) take the running-softmax kernel.
+constexpr int kFlashMinCap = 192;
+template <int DH> int flash_set_attr() {
+  CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::SMEM_BYTES));
+  return TSFM_OK;
+}
 template <typename T>
 int attn_prepare(int dh, int cap) {
-  const size_t bytes = attn_smem_bytes<T>(dh, (cap + 15) & ~15);
+  if (sizeof(T) == 2) {
+    if (int rc = dh == 32 ? flash_set_attr<32>() : dh == 64 ? flash_set_attr<64>() : flash_set_attr<128>()) return rc;
+  }
+  const size_t bytes = attn_smem_bytes<T>(dh, attn_rows_per_cta(cap, attn_key_split(cap)));
   if (bytes > 227 * 1024) return TSFM_ERR_SHAPE;
   const size_t optin = 227 * 1024;        // opt in once to the per-CTA maximum; launches size themselves
   if (dh == 32) return attn_set_attr<T, 32>(optin);
@@ -322,6 +344,9 @@ template <typename T> void prefer_max_smem_typed() {
   prefer_max_smem(attn_kernel<T, 32>);
   prefer_max_smem(attn_kernel<T, 64>);
   prefer_max_smem(attn_kernel<T, 128>);
+  prefer_max_smem(kv_append_kernel<T, 32>);
+  prefer_max_smem(kv_append_kernel<T, 64>);
+  prefer_max_smem(kv_append_kernel<T, 128>);
 }
 void prefer_max_smem_all() {
   prefer_max_smem_typed<float>();
@@ -334,6 +359,9 @@ void prefer_max_smem_all() {
   prefer_max_smem(gemm_sk_kernel<1, false, true>);
   prefer_max_smem(gemm_sk_kernel<2, true, false>);
   prefer_max_smem(pass_cluster_kernel);
+  prefer_max_smem(attn_flash_kernel<32>);
+  prefer_max_smem(attn_flash_kernel<64>);
+  prefer_max_smem(attn_flash_kernel<128>);
   cudaGetLastError();
 }
 
@@ -352,6 +380,28 @@ void launch_ex(cudaStream_t s, bool pdl, void (*kernel)(KArgs...), dim3 grid, di
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+  LAUNCHED();
+}
+
+// The same with a thread-block cluster of cluster_z CTAs along z (grid.z a multiple of it).
+template <typename... KArgs, typename... Args>
+void launch_ex_cluster(cudaStream_t s, bool pdl, int cluster_z, void (*kernel)(KArgs...), dim3 grid, dim3 block,
+                       size_t smem, Args &&...args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 1;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = (unsigned)cluster_z;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 2 : 1;
   cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
   LAUNCHED();
 }
@@ -386,8 +436,9 @@ void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C,
 template <typename T, int DH>
 void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   const int QT = g.q_len <= ATTN_QT ? g.q_len : ATTN_QT;
-  dim3 grid(m.arch.n_heads, B, (g.q_len + QT - 1) / QT);
-  const int nk_max = (h->cap + 15) & ~15;      // keys padded to whole MMA blocks; regions stay 16-byte aligned
+  const int skv = attn_key_split(h->cap);
+  dim3 grid(m.arch.n_heads, B, ((g.q_len + QT - 1) / QT) * skv);
+  const int nk_max = attn_rows_per_cta(h->cap, skv);   // whole MMA blocks; regions stay 16-byte aligned
   const size_t smem = attn_smem_bytes<T>(DH, nk_max);
   T *Kc = (T *)m.Kc + (size_t)l * m.kv_layer_elems;
   T *Vc = (T *)m.Vc + (size_t)l * m.kv_layer_elems;
@@ -396,8 +447,29 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   const double Mr = (double)B * g.q_len;
   KTimer kt(h, KC_ATTN, Mr * 3 * m.arch.d_model * 4 + kv + Mr * m.arch.d_model * (2.0 * sizeof(T) + sizeof(T)),
             4.0 * Mr * (std::max(g.base, 0) + 0.5 * g.q_len) * m.arch.d_model);
-  launch_ex(h->ls, h->pdl, attn_kernel<T, DH>, grid, dim3(128), smem, h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
-            nk_max, (T *)h->ao);
+  // several query tiles, or long bf16 rows: the pass's keys and values go to the cache first, once
+  const bool flash = sizeof(T) == 2 && (g.q_len > ATTN_QT || h->cap >= kFlashMinCap);
+  const int pre = (g.q_len > ATTN_QT || flash) ? 1 : 0;
+  if (pre)
+    launch_ex(h->ls, h->pdl, kv_append_kernel<T, DH>, dim3(m.arch.n_heads, B, (g.q_len + 15) / 16), dim3(128), 0,
+              h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads);
+  if constexpr (sizeof(T) == 2) {
+    if (flash) {
+      // many queries: a warp per query tile; one tile: its keys dealt out over the four warps
+      const int split = g.q_len > ATTN_QT ? 1 : 4;
+      const int per_cta = split == 1 ? 4 * ATTN_QT : ATTN_QT;
+      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH>, dim3(m.arch.n_heads, B, (g.q_len + per_cta - 1) / per_cta),
+                dim3(128), (size_t)FlashGeom<DH>::SMEM_BYTES, h->qkv, (const bf16 *)Kc, (const bf16 *)Vc, m.rope, g,
+                m.arch.n_heads, split, (bf16 *)h->ao);
+      return;
+    }
+  }
+  if (skv > 1)
+    launch_ex_cluster(h->ls, h->pdl, skv, attn_kernel<T, DH>, grid, dim3(128), smem, h->qkv, Kc, Vc, m.rope, g,
+                      m.arch.n_heads, QT, nk_max, skv, pre, (T *)h->ao);
+  else
+    launch_ex(h->ls, h->pdl, attn_kernel<T, DH>, grid, dim3(128), smem, h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
+              nk_max, skv, pre, (T *)h->ao);
 }
 
 enum { HEAD_NONE = 0, HEAD_LAST_TO_HIST = 1, HEAD_ALL_TO_VOUT = 2 };

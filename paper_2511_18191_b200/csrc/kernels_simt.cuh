@@ -278,8 +278,8 @@ constexpr int ATTN_QT = 16;                             // queries per tile (at 
 // partial outputs.  NQ = compile-time bound on the number of queries (loops are unrolled to it).
 template <typename T, int DH, int NQ>
 __device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs, float *sc, const float *qs, float *po,
-                                          float *inv_sum, int nq, int nk, int nk_max, int p0, int j_lo, size_t row0,
-                                          int d, int h, T *__restrict__ out) {
+                                          float *row_max, float *row_sum, int nq, int nk, int nk_max, int k_lo,
+                                          int p0, int j_lo) {
   constexpr bool BF = sizeof(T) == 2;
   constexpr int VW = AttnWords<T>::per_row(DH), DPL = DH / 32;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, tid = threadIdx.x;
@@ -308,7 +308,7 @@ __device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs
     }
 #pragma unroll
     for (int i = 0; i < NQ; ++i)
-      if (i < nq) sc[(size_t)i * nk_max + t] = (t <= p0 + j_lo + i) ? sacc[i] : -INFINITY;   // causal mask
+      if (i < nq) sc[(size_t)i * nk_max + t] = (k_lo + t <= p0 + j_lo + i) ? sacc[i] : -INFINITY;   // causal mask
   }
   __syncthreads();
   for (int i = w; i < nq; i += 4) {
@@ -318,12 +318,12 @@ __device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs
     mx = warp_max(mx);
     float sum = 0.f;
     for (int t = lane; t < nk; t += 32) {
-      const float pv = expf(row[t] - mx);
+      const float pv = mx == -INFINITY ? 0.f : expf(row[t] - mx);   // no visible key in this CTA's range
       row[t] = pv;
       sum += pv;
     }
     sum = warp_sum(sum);
-    if (lane == 0) inv_sum[i] = 1.f / sum;
+    if (lane == 0) { row_max[i] = mx; row_sum[i] = sum; }
   }
   __syncthreads();
   float acc[NQ][DPL];
@@ -363,12 +363,6 @@ __device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs
 #pragma unroll
       for (int c = 0; c < DPL; ++c) po[((size_t)w * ATTN_QT + i) * DH + lane * DPL + c] = acc[i][c];
   __syncthreads();
-  for (int idx = tid; idx < nq * DH; idx += blockDim.x) {
-    const int i = idx / DH, c = idx % DH;
-    const float o = po[(size_t)(0 * ATTN_QT + i) * DH + c] + po[(size_t)(1 * ATTN_QT + i) * DH + c] +
-                    po[(size_t)(2 * ATTN_QT + i) * DH + c] + po[(size_t)(3 * ATTN_QT + i) * DH + c];
-    out[(row0 + j_lo + i) * d + h * DH + c] = from_f32<T>(o * inv_sum[i]);
-  }
 }
 
 // ----------------------------------------------------------------------------------
@@ -393,10 +387,10 @@ __device__ __forceinline__ void split_bf16x2(float x, float y, uint32_t &hi, uin
 
 template <int DH>
 __device__ __forceinline__ void attn_tile_mma(const uint32_t *Ks, const uint32_t *Vs, float *sc, const float *qs, float *po,
-                                              float *inv_sum, int nq, int nk, int nk_max, int p0, int j_lo, size_t row0,
-                                              int d, int h, bf16 *__restrict__ out) {
+                                              float *row_max, float *row_sum, int nq, int nk, int nk_max, int k_lo,
+                                              int p0, int j_lo) {
   constexpr int VW = DH / 2, KS = DH / 16;
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, tid = threadIdx.x;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int g = lane >> 2, q4 = lane & 3;            // fragment row group, column pair
   const int nk16 = (nk + 15) & ~15;
   {
@@ -427,7 +421,7 @@ __device__ __forceinline__ void attn_tile_mma(const uint32_t *Ks, const uint32_t
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int r = g + (e >> 1) * 8, tt = t + (e & 1);
-        if (r < nq) sc[(size_t)r * nk_max + tt] = (tt <= p0 + j_lo + r && tt < nk) ? c[e] : -INFINITY;
+        if (r < nq) sc[(size_t)r * nk_max + tt] = (k_lo + tt <= p0 + j_lo + r && tt < nk) ? c[e] : -INFINITY;
       }
     }
   }
@@ -439,12 +433,12 @@ __device__ __forceinline__ void attn_tile_mma(const uint32_t *Ks, const uint32_t
     mx = warp_max(mx);
     float sum = 0.f;
     for (int t = lane; t < nk16; t += 32) {
-      const float pv = expf(row[t] - mx);
+      const float pv = mx == -INFINITY ? 0.f : expf(row[t] - mx);   // no visible key in this CTA's range
       row[t] = pv;
       sum += pv;
     }
     sum = warp_sum(sum);
-    if (lane == 0) inv_sum[i] = 1.f / sum;
+    if (lane == 0) { row_max[i] = mx; row_sum[i] = sum; }
   }
   __syncthreads();
   {
@@ -487,18 +481,75 @@ __device__ __forceinline__ void attn_tile_mma(const uint32_t *Ks, const uint32_t
       }
   }
   __syncthreads();
-  for (int idx = tid; idx < nq * DH; idx += blockDim.x) {
-    const int i = idx / DH, c = idx % DH;
-    const float o = po[(size_t)(0 * ATTN_QT + i) * DH + c] + po[(size_t)(1 * ATTN_QT + i) * DH + c] +
-                    po[(size_t)(2 * ATTN_QT + i) * DH + c] + po[(size_t)(3 * ATTN_QT + i) * DH + c];
-    out[(row0 + j_lo + i) * d + h * DH + c] = __float2bfloat16_rn(o * inv_sum[i]);
+}
+
+// Keys and values of a pass with several query tiles go to the cache once, before attention:
+// rotated key and value of token j of series b, head h, to cache row pos0 + j.  Every tile of
+// attn_kernel (launched with pre = 1) then finds all keys of the pass in the cache instead of
+// rotating the earlier tiles' keys again.  grid = (heads, B, ceil(q_len / 16)), block = 128.
+template <typename T, int DH>
+__global__ void __launch_bounds__(128)
+kv_append_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
+                 const float2 *__restrict__ rope, PassGeom g, int n_heads) {
+  constexpr int HALF = DH / 2;
+  const int h = blockIdx.x, b = blockIdx.y, d = n_heads * DH;
+  pdl_sync();
+  const int p0 = pos0_of(g, b);
+  const int j_lo = blockIdx.z * 16, j_hi = min(g.q_len, j_lo + 16);
+  const size_t row0 = (size_t)b * g.q_len;
+  T *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
+  T *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
+  for (int i = threadIdx.x; i < (j_hi - j_lo) * (HALF / 2); i += blockDim.x) {
+    const int j = j_lo + i / (HALF / 2), c = (i % (HALF / 2)) * 2;
+    const float *src = qkv + (row0 + j) * 3 * d + h * DH;
+    const int tg = p0 + j;
+    const float4 cs = *reinterpret_cast<const float4 *>(rope + (size_t)tg * HALF + c);   // cos0 sin0 cos1 sin1
+    const float2 ka = *reinterpret_cast<const float2 *>(src + d + c);
+    const float2 kb = *reinterpret_cast<const float2 *>(src + d + c + HALF);
+    const float2 va = *reinterpret_cast<const float2 *>(src + 2 * d + c);
+    const float2 vb = *reinterpret_cast<const float2 *>(src + 2 * d + c + HALF);
+    const float r1a = ka.x * cs.x - kb.x * cs.y, r1b = ka.y * cs.z - kb.y * cs.w;    // first half
+    const float r2a = kb.x * cs.x + ka.x * cs.y, r2b = kb.y * cs.z + ka.y * cs.w;    // second half
+    if (sizeof(T) == 2) {
+      uint32_t *kg = reinterpret_cast<uint32_t *>(Kb + (size_t)tg * DH);
+      uint32_t *vg = reinterpret_cast<uint32_t *>(Vb + (size_t)tg * DH);
+      kg[c / 2] = pack_bf16x2(r1a, r1b); kg[(c + HALF) / 2] = pack_bf16x2(r2a, r2b);
+      vg[c / 2] = pack_bf16x2(va.x, va.y); vg[(c + HALF) / 2] = pack_bf16x2(vb.x, vb.y);
+    } else {
+      float *kg = reinterpret_cast<float *>(Kb + (size_t)tg * DH);
+      float *vg = reinterpret_cast<float *>(Vb + (size_t)tg * DH);
+      kg[c] = r1a; kg[c + 1] = r1b; kg[c + HALF] = r2a; kg[c + HALF + 1] = r2b;
+      vg[c] = va.x; vg[c + 1] = va.y; vg[c + HALF] = vb.x; vg[c + HALF + 1] = vb.y;
+    }
   }
 }
 
+// Thread-block-cluster helpers of the key-split attention: every CTA of a cluster reaches
+// attn_cluster_sync the same number of times; attn_peer_f32 reads one float of a peer CTA's
+// shared memory at the same offset as `local`.
+__device__ __forceinline__ void attn_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float attn_peer_f32(const float *local, uint32_t rank) {
+  uint32_t remote;
+  float v;
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(local);
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(a), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+  return v;
+}
+
+// skv = 1: one CTA holds every key of its (series, head).  skv > 1: the launch carries a cluster
+// of skv CTAs along z (blockIdx.z = tile * skv + rank); rank r holds the keys
+// [r * chunk, (r + 1) * chunk) of the row, chunk a multiple of 16, computes the softmax
+// numerator, its row maxima and row sums over them, and the ranks combine the pieces through
+// distributed shared memory: m = max_r m_r, l = sum_r l_r e^(m_r - m), o = sum_r o_r e^(m_r - m) / l.
+// nk_max is the number of key rows one CTA can hold.  pre = 1: kv_append_kernel has already put
+// the keys and values of this pass into the cache.
 template <typename T, int DH>
 __global__ void __launch_bounds__(128)
 attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
-            const float2 *__restrict__ rope, PassGeom g, int n_heads, int QT, int nk_max,
+            const float2 *__restrict__ rope, PassGeom g, int n_heads, int QT, int nk_max, int skv, int pre,
             T *__restrict__ out) {
   constexpr bool BF = sizeof(T) == 2;
   constexpr int VW = AttnWords<T>::per_row(DH);   // words per value row
@@ -511,15 +562,22 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   float *sc = reinterpret_cast<float *>(Ks + (size_t)nk_max * KW);
   float *qs = sc + (size_t)ATTN_QT * nk_max;        // [ATTN_QT][DH] rotated, scaled queries
   float *po = qs + ATTN_QT * DH;                    // [4][ATTN_QT][DH] partial outputs per warp
-  float *inv_sum = po + 4 * ATTN_QT * DH;           // [ATTN_QT]
+  float *row_max = po + 4 * ATTN_QT * DH;           // [ATTN_QT] maximum score over this CTA's keys
+  float *row_sum = row_max + ATTN_QT;               // [ATTN_QT] sum of exp(score - row_max)
 
-  const int h = blockIdx.x, b = blockIdx.y, qt = blockIdx.z;
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int qt = skv > 1 ? blockIdx.z / skv : blockIdx.z;
+  const int rank = skv > 1 ? blockIdx.z % skv : 0;   // == %cluster_ctarank: the cluster spans z only
   const int d = n_heads * DH;
   pdl_sync();
   const int p0 = pos0_of(g, b);
   const int j_lo = qt * QT;
   const int j_hi = min(g.q_len, j_lo + QT);          // queries [j_lo, j_hi)
   const size_t row0 = (size_t)b * g.q_len;
+  const int nk_all = p0 + j_hi;                      // keys visible to the tile's last query
+  const int chunk = skv > 1 ? (((nk_all + skv - 1) / skv + 15) & ~15) : nk_all;
+  const int k_lo = min(rank * chunk, nk_all);        // this CTA holds keys [k_lo, k_hi) at rows t - k_lo
+  const int k_hi = min(k_lo + chunk, nk_all);
   T *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
   T *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
 
@@ -527,20 +585,22 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   // front (the cache comes from HBM: the copy is bound by the bytes in flight)
   {
     constexpr int VPR = DH / EPV;                    // 16-byte chunks per row
-    const int nvec = p0 * VPR;
+    const int nvec = max(min(k_hi, pre ? nk_all : p0) - k_lo, 0) * VPR;
+    const T *Kg = Kb + (size_t)k_lo * DH, *Vg = Vb + (size_t)k_lo * DH;
     for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
       const int t = i / VPR, c = i % VPR;
-      cp_async16(Ks + (size_t)t * VW + (((c + t) & (VPR - 1)) << 2), Kb + (size_t)i * EPV);
-      cp_async16(Vs + (size_t)i * 4, Vb + (size_t)i * EPV);
+      cp_async16(Ks + (size_t)t * VW + (((c + t) & (VPR - 1)) << 2), Kg + (size_t)i * EPV);
+      cp_async16(Vs + (size_t)i * 4, Vg + (size_t)i * EPV);
     }
   }
   // keys/values of this pass (rotate keys; the owning tile appends to the cache).
   // One thread handles the element pair (c, c + 1) of the first half and its rotation partners.
-  for (int i = threadIdx.x; i < j_hi * (HALF / 2); i += blockDim.x) {
+  for (int i = threadIdx.x; i < (pre ? 0 : j_hi * (HALF / 2)); i += blockDim.x) {
     const int j = i / (HALF / 2), c = (i % (HALF / 2)) * 2;
     const float *src = qkv + (row0 + j) * 3 * d + h * DH;
-    const int t = p0 + j;
-    const float4 cs = *reinterpret_cast<const float4 *>(rope + (size_t)t * HALF + c);   // cos0 sin0 cos1 sin1
+    const int tg = p0 + j, t = tg - k_lo;            // position in the row, row in this CTA
+    if (tg < k_lo || tg >= k_hi) continue;
+    const float4 cs = *reinterpret_cast<const float4 *>(rope + (size_t)tg * HALF + c);   // cos0 sin0 cos1 sin1
     const float2 ka = *reinterpret_cast<const float2 *>(src + d + c);
     const float2 kb = *reinterpret_cast<const float2 *>(src + d + c + HALF);
     const float2 va = *reinterpret_cast<const float2 *>(src + 2 * d + c);
@@ -555,8 +615,8 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
       Vs[(size_t)t * VW + c / 2] = v1;
       Vs[(size_t)t * VW + (c + HALF) / 2] = v2;
       if (j >= j_lo) {
-        uint32_t *kg = reinterpret_cast<uint32_t *>(Kb + (size_t)t * DH);
-        uint32_t *vg = reinterpret_cast<uint32_t *>(Vb + (size_t)t * DH);
+        uint32_t *kg = reinterpret_cast<uint32_t *>(Kb + (size_t)tg * DH);
+        uint32_t *vg = reinterpret_cast<uint32_t *>(Vb + (size_t)tg * DH);
         kg[c / 2] = k1; kg[(c + HALF) / 2] = k2;
         vg[c / 2] = v1; vg[(c + HALF) / 2] = v2;
       }
@@ -567,8 +627,8 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
       kf[attn_kword<VW>(t, c + HALF)] = r2a; kf[attn_kword<VW>(t, c + HALF + 1)] = r2b;
       vf[c] = va.x; vf[c + 1] = va.y; vf[c + HALF] = vb.x; vf[c + HALF + 1] = vb.y;
       if (j >= j_lo) {
-        float *kg = reinterpret_cast<float *>(Kb + (size_t)t * DH);
-        float *vg = reinterpret_cast<float *>(Vb + (size_t)t * DH);
+        float *kg = reinterpret_cast<float *>(Kb + (size_t)tg * DH);
+        float *vg = reinterpret_cast<float *>(Vb + (size_t)tg * DH);
         kg[c] = r1a; kg[c + 1] = r1b; kg[c + HALF] = r2a; kg[c + HALF + 1] = r2b;
         vg[c] = va.x; vg[c + 1] = va.y; vg[c + HALF] = vb.x; vg[c + HALF + 1] = vb.y;
       }
@@ -578,9 +638,9 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   const int tid = threadIdx.x;
   const float scale = rsqrtf((float)DH);
   const int nq = j_hi - j_lo;                        // <= ATTN_QT
-  const int nk = p0 + j_hi;                          // keys visible to the tile's last query
+  const int nk = k_hi - k_lo;                        // key rows held here
   // rows the tile routine will touch: its compile-time query bound (16 on the tensor-core path)
-  const bool use_mma = BF && nq >= 3 && nk >= 96;
+  const bool use_mma = BF && nq >= 3 && nk_all >= 96;
   const int nqb = use_mma ? ATTN_QT : nq <= 2 ? nq : nq <= 4 ? 4 : nq <= 6 ? 6 : nq <= 9 ? 9 : ATTN_QT;
   for (int idx = tid; idx < nqb * HALF; idx += blockDim.x) {       // rotated, scaled queries (zero past nq)
     const int i = idx / HALF, c = idx % HALF, j = j_lo + i;
@@ -602,16 +662,49 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
     const int nk16 = (nk + 15) & ~15;
     for (int idx = tid + nk * VW; idx < nk16 * VW; idx += blockDim.x) Vs[idx] = 0u;   // value rows of the padding keys
     __syncthreads();
-    if constexpr (BF)
-      attn_tile_mma<DH>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, reinterpret_cast<bf16 *>(out));
+    if constexpr (BF) attn_tile_mma<DH>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
+  }
+  else if (nq == 1) attn_tile<T, DH, 1>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
+  else if (nq == 2) attn_tile<T, DH, 2>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
+  else if (nq <= 4) attn_tile<T, DH, 4>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
+  else if (nq <= 6) attn_tile<T, DH, 6>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
+  else if (nq <= 9) attn_tile<T, DH, 9>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
+  else attn_tile<T, DH, ATTN_QT>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
+  // the tile routines end on a block barrier: po holds each warp's unnormalised partial output
+
+  if (skv <= 1) {
+    for (int idx = tid; idx < nq * DH; idx += blockDim.x) {
+      const int i = idx / DH, c = idx % DH;
+      const float o = po[(size_t)(0 * ATTN_QT + i) * DH + c] + po[(size_t)(1 * ATTN_QT + i) * DH + c] +
+                      po[(size_t)(2 * ATTN_QT + i) * DH + c] + po[(size_t)(3 * ATTN_QT + i) * DH + c];
+      out[(row0 + j_lo + i) * d + h * DH + c] = from_f32<T>(o / row_sum[i]);
+    }
     return;
   }
-  if (nq == 1) attn_tile<T, DH, 1>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
-  else if (nq == 2) attn_tile<T, DH, 2>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
-  else if (nq <= 4) attn_tile<T, DH, 4>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
-  else if (nq <= 6) attn_tile<T, DH, 6>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
-  else if (nq <= 9) attn_tile<T, DH, 9>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
-  else attn_tile<T, DH, ATTN_QT>(Ks, Vs, sc, qs, po, inv_sum, nq, nk, nk_max, p0, j_lo, row0, d, h, out);
+  // key-split: fold the four warps' partials into qs (the queries are no longer needed), then
+  // rank (i mod skv) combines query i over the cluster
+  for (int idx = tid; idx < nq * DH; idx += blockDim.x) {
+    const int i = idx / DH, c = idx % DH;
+    qs[idx] = po[(size_t)(0 * ATTN_QT + i) * DH + c] + po[(size_t)(1 * ATTN_QT + i) * DH + c] +
+              po[(size_t)(2 * ATTN_QT + i) * DH + c] + po[(size_t)(3 * ATTN_QT + i) * DH + c];
+  }
+  attn_cluster_sync();
+  for (int idx = tid; idx < nq * DH; idx += blockDim.x) {
+    const int i = idx / DH, c = idx % DH;
+    if (i % skv != rank) continue;
+    float m = -INFINITY;
+    for (int r = 0; r < skv; ++r) m = fmaxf(m, attn_peer_f32(row_max + i, r));
+    float l = 0.f, o = 0.f;
+    for (int r = 0; r < skv; ++r) {
+      const float mr = attn_peer_f32(row_max + i, r);
+      if (mr == -INFINITY) continue;               // that rank saw no visible key of this query
+      const float w = expf(mr - m);
+      l = fmaf(attn_peer_f32(row_sum + i, r), w, l);
+      o = fmaf(attn_peer_f32(qs + idx, r), w, o);
+    }
+    out[(row0 + j_lo + i) * d + h * DH + c] = from_f32<T>(o / l);
+  }
+  attn_cluster_sync();                               // no CTA leaves while a peer still reads its shared memory
 }
 
 // ----------------------------------------------------------------------------------

@@ -144,6 +144,18 @@ def test_c4_subset():
     run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, [0, 63])
 
 
+@pytest.mark.parametrize("target,draft", [
+    (Arch(2, 256, 2, 512), Arch(1, 64, 2, 128)),      # head sizes 128 and 32
+    (Arch(2, 256, 4, 512), Arch(1, 128, 2, 256)),     # head size 64
+])
+def test_long_rows_small_models_bf16(target, draft):
+    """C4's row lengths (256 context tokens, K = 8) on small models: the running-softmax attention
+    with the keys of a row dealt out over four warps, for every head size, ragged batch of 3."""
+    wl = workload("C4", batch=3, horizon=32 * 11 + 7, target=target, draft=draft)
+    run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, [0, 1, 2])
+    run_and_compare(wl, 3, 2.0, 5, [2], exec_mode=1)
+
+
 @pytest.mark.parametrize("name,ids", [("C0", [0]), ("C1", [0, 7, 31]), ("C2", [3, 200])])
 def test_draft_only_forecast_matches_oracle(name, ids):
     """Third arm of the matched three-way protocol: the draft model decoding on its own (Eq. 1)."""

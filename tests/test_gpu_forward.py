@@ -37,6 +37,7 @@ def run_forward_case(wl, backend, n_tokens, B=5, seed=0):
 @pytest.mark.parametrize("target,draft,P,n", [
     (Arch(2, 128, 4, 512), Arch(1, 64, 2, 256), 96, 7),        # C0's models (head size 32)
     (Arch(2, 128, 2, 256), Arch(1, 128, 1, 128), 32, 21),      # head sizes 64 and 128, several query tiles
+    (Arch(1, 128, 2, 256), Arch(1, 64, 2, 128), 32, 197),      # long rows: keys split over a cluster, ragged tail
 ])
 def test_fp32_forward_matches_oracle(target, draft, P, n):
     wl = small_workload("f32", target, draft, P)
@@ -52,6 +53,8 @@ def test_fp32_forward_matches_oracle(target, draft, P, n):
     (Arch(4, 512, 8, 2048), Arch(2, 512, 8, 2048), 32, 6, "layer_skip"),   # 8-CTA clusters, two token tiles of 16
     (Arch(2, 384, 6, 1536), Arch(1, 128, 2, 256), 96, 3, "separate"),      # 6 heads: 3 feature tiles, ragged owners
     (Arch(2, 256, 4, 1024), Arch(1, 128, 2, 256), 32, 120, "separate"),    # 120 keys: tensor-core attention tiles
+    (Arch(2, 256, 4, 1024), Arch(1, 128, 2, 256), 32, 200, "separate"),    # 200 keys: several chunks of the key stream
+    (Arch(2, 256, 2, 512), Arch(1, 64, 2, 128), 32, 75, "separate"),       # head sizes 128 and 32, ragged last tile
 ])
 def test_bf16_forward_matches_oracle(backend, target, draft, P, n, mode):
     wl = small_workload("bf16", target, draft, P, mode)
