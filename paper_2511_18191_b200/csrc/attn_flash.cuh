@@ -1,6 +1,4 @@
-// Causal attention over a bf16 KV cache with a running softmax (one pass over the keys), for
-// long rows and for passes with many query tokens.  The keys and values of the pass itself are
-// already in the cache (kv_append_kernel runs first), so every key comes from one place.
+// Causal attention over a bf16 KV cache with a running softmax (one pass over the keys).
 //
 // Work unit = one warp: 16 queries (the M side of mma.sync m16n8k16) against a range of keys of
 // one (series, head).  The warp streams its keys in chunks of 32 through a private ring of
@@ -8,10 +6,18 @@
 // running maximum m, the running sum l of exp(s - m) and the unnormalised output o in registers:
 //     m' = max(m, max_t s_t),  l' = l e^(m - m') + sum_t e^(s_t - m'),  o' = o e^(m - m') + sum_t e^(s_t - m') v_t.
 // No block-wide barrier is needed while the keys stream.
-//   split = 1: the four warps of a CTA take four consecutive query tiles (64 queries), each over
-//              all keys its queries may see.  grid = (heads, B, ceil(q_len / 64)).
-//   split = 4: the four warps share one query tile and take a quarter of the keys each; the
-//              four (m, l, o) are merged through shared memory.  grid = (heads, B, ceil(q_len / 16)).
+//   mode FLASH_TILES: passes of more than 16 tokens.  kv_append_kernel has put the keys and values
+//              of the pass into the cache; the four warps of a CTA take four consecutive query
+//              tiles (64 queries), each over all keys its queries may see.
+//              grid = (heads, B, ceil(q_len / 64)).
+//   mode FLASH_SPLIT: passes of at most 16 tokens (one query tile), long rows.  The cached keys
+//              [0, pos0) are dealt out over the four warps; the last warp also takes the keys of
+//              the pass itself, which it rotates, rounds, puts into a stage of its ring and
+//              appends to the cache; the four (m, l, o) are merged through shared memory.
+//              grid = (heads, B, 1).
+//   mode FLASH_WARP: the same passes on short rows with many (series, head) pairs: each warp
+//              takes one pair on its own (cached keys, then the keys of the pass).
+//              grid = (ceil(B * heads / 4), 1, 1).
 // S = Q K^T uses the rotated, scaled fp32 queries split into a bf16 high and low part (two MMAs),
 // so the scores keep fp32-like accuracy; P is rounded to bf16 for P V.  Scores are kept in
 // base-2 units (the queries carry log2(e) / sqrt(DH)).
@@ -20,6 +26,8 @@
 #include "kernels_simt.cuh"
 
 namespace tsfm {
+
+enum { FLASH_WARP = 0, FLASH_TILES = 1, FLASH_SPLIT = 4 };
 
 template <int DH> struct FlashGeom {
   static constexpr int CHUNK = 32;                              // keys per stage
@@ -54,35 +62,45 @@ template <int N> __device__ __forceinline__ void flash_wait() { asm volatile("cp
 
 template <int DH>
 __global__ void __launch_bounds__(128)
-attn_flash_kernel(const float *__restrict__ qkv, const bf16 *__restrict__ Kc, const bf16 *__restrict__ Vc,
-                  const float2 *__restrict__ rope, PassGeom g, int n_heads, int split, bf16 *__restrict__ out) {
+attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
+                  const float2 *__restrict__ rope, PassGeom g, int n_heads, int n_pairs, int mode,
+                  bf16 *__restrict__ out) {
   using G = FlashGeom<DH>;
   constexpr int HALF = DH / 2, KS = DH / 16, CPR = DH / 8;     // k-steps of Q K^T, 16-byte chunks per row
   extern __shared__ __align__(128) unsigned char flash_smem[];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int gr = lane >> 2, q4 = lane & 3;                     // fragment row group, column pair
-  const int h = blockIdx.x, b = blockIdx.y, d = n_heads * DH;
+  const int d = n_heads * DH;
+  int h = blockIdx.x, b = blockIdx.y;
+  if (mode == FLASH_WARP) {
+    const int pair = blockIdx.x * 4 + w;
+    if (pair >= n_pairs) return;                               // no block-wide barrier in this mode
+    b = pair / n_heads;
+    h = pair % n_heads;
+  }
   unsigned char *ring = flash_smem + (size_t)w * G::WARP_BYTES;
   const uint32_t ring32 = (uint32_t)__cvta_generic_to_shared(ring);
   pdl_sync();
   const int p0 = pos0_of(g, b);
   const size_t row0 = (size_t)b * g.q_len;
-  const bf16 *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
-  const bf16 *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
+  bf16 *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
+  bf16 *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
 
-  // this warp's queries [jq, jq + 16) and keys [t_beg, t_end)
-  int jq, t_beg, t_end;
-  if (split == 1) {
+  // this warp's queries [jq, jq + 16), cached keys [t_beg, t_end), and whether it takes the
+  // keys of the pass itself as one more chunk
+  int jq = 0, t_beg = 0, t_end = p0;
+  bool own_pass_keys = true;
+  if (mode == FLASH_TILES) {
     jq = (blockIdx.z * 4 + w) * 16;
-    if (jq >= g.q_len) return;                                 // no block-wide barrier on this path
-    t_beg = 0;
+    if (jq >= g.q_len) return;                                 // no block-wide barrier in this mode
     t_end = p0 + min(jq + 16, g.q_len);
-  } else {
-    jq = blockIdx.z * 16;
-    const int nk = p0 + min(jq + 16, g.q_len);
-    const int R = ((nk + 3) / 4 + 15) & ~15;
-    t_beg = min(w * R, nk);
-    t_end = min(t_beg + R, nk);
+    own_pass_keys = false;
+  } else if (mode == FLASH_SPLIT) {
+    // whole chunks, the keys of the pass counted as one more chunk at the end
+    const int R = (((p0 + G::CHUNK - 1) / G::CHUNK + 1 + 3) / 4) * G::CHUNK;
+    t_beg = min(w * R, p0);
+    t_end = min(t_beg + R, p0);
+    own_pass_keys = w == 3;
   }
   const int nq = min(16, g.q_len - jq);
   const int nch = (t_end - t_beg + G::CHUNK - 1) / G::CHUNK;
@@ -138,13 +156,9 @@ attn_flash_kernel(const float *__restrict__ qkv, const bf16 *__restrict__ Kc, co
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
   const int qpos0 = p0 + jq + gr;                              // position of row gr; row gr + 8 is 8 further
 
-  for (int c = 0; c < nch; ++c) {
-    flash_wait<G::STAGES - 2>();
-    __syncwarp();
-    issue(c + G::STAGES - 1);                                  // refills the stage consumed in the previous turn
-    const int t0 = t_beg + c * G::CHUNK;
-    const uint32_t kst = ring32 + (uint32_t)((c % G::STAGES) * G::STAGE_BYTES), vst = kst + G::TILE_BYTES;
-
+  // one chunk: 32 keys at positions t0.. from the stage at kst (values at vst); keys at or past
+  // t_lim, and keys after a query's own position, are masked
+  auto chunk = [&](uint32_t kst, uint32_t vst, int t0, int t_lim) {
     // ---- scores of 16 queries x 32 keys
     float s[4][4];
 #pragma unroll
@@ -163,13 +177,13 @@ attn_flash_kernel(const float *__restrict__ qkv, const bf16 *__restrict__ Kc, co
       }
     }
     // ---- causal mask and range end (only chunks that reach either)
-    if (t0 + G::CHUNK > t_end || t0 + G::CHUNK - 1 > p0 + jq) {
+    if (t0 + G::CHUNK > t_lim || t0 + G::CHUNK - 1 > p0 + jq) {
 #pragma unroll
       for (int n = 0; n < 4; ++n)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int t = t0 + n * 8 + q4 * 2 + (e & 1);
-          if (t >= t_end || t > qpos0 + (e >> 1) * 8) s[n][e] = -INFINITY;
+          if (t >= t_lim || t > qpos0 + (e >> 1) * 8) s[n][e] = -INFINITY;
         }
     }
     // ---- running softmax
@@ -208,6 +222,53 @@ attn_flash_kernel(const float *__restrict__ qkv, const bf16 *__restrict__ Kc, co
         mma_bf16_16816(o[n0 + 1], pa[kk], bv[2], bv[3]);
       }
     }
+  };
+
+  if (own_pass_keys) {
+    // keys and values of this pass (at most 16 tokens) first, while the copies of the first
+    // cached chunks are in flight: rotate the keys, round both to bf16, put them into the last
+    // stage, which the ring does not use before its first refill (value rows past the last token
+    // are zeroed: their probabilities are 0, but 0 x NaN would not be) and append them to the
+    // cache.  One lane handles the element pairs (c, c + 1) and (c + HALF, c + HALF + 1) of a token.
+    unsigned char *st = ring + (G::STAGES - 1) * G::STAGE_BYTES;
+    uint32_t *ks = reinterpret_cast<uint32_t *>(st), *vs = reinterpret_cast<uint32_t *>(st + G::TILE_BYTES);
+#pragma unroll 2
+    for (int i = lane; i < g.q_len * (HALF / 2); i += 32) {
+      const int j = i / (HALF / 2), c = (i % (HALF / 2)) * 2;
+      const float *src = qkv + (row0 + j) * 3 * d + h * DH;
+      const int tg = p0 + j;
+      const float4 cs = *reinterpret_cast<const float4 *>(rope + (size_t)tg * HALF + c);   // cos0 sin0 cos1 sin1
+      const float2 ka = *reinterpret_cast<const float2 *>(src + d + c);
+      const float2 kb = *reinterpret_cast<const float2 *>(src + d + c + HALF);
+      const float2 va = *reinterpret_cast<const float2 *>(src + 2 * d + c);
+      const float2 vb = *reinterpret_cast<const float2 *>(src + 2 * d + c + HALF);
+      const uint32_t k1 = pack_bf16x2(ka.x * cs.x - kb.x * cs.y, ka.y * cs.z - kb.y * cs.w);
+      const uint32_t k2 = pack_bf16x2(kb.x * cs.x + ka.x * cs.y, kb.y * cs.z + ka.y * cs.w);
+      const uint32_t v1 = pack_bf16x2(va.x, va.y), v2 = pack_bf16x2(vb.x, vb.y);
+      const int w1 = c / 2, w2 = (c + HALF) / 2;               // 32-bit words of the row
+      const int a1 = j * (DH / 2) + flash_swz<DH>(j, w1 >> 2) * 4 + (w1 & 3);
+      const int a2 = j * (DH / 2) + flash_swz<DH>(j, w2 >> 2) * 4 + (w2 & 3);
+      ks[a1] = k1; ks[a2] = k2;
+      vs[a1] = v1; vs[a2] = v2;
+      uint32_t *kg = reinterpret_cast<uint32_t *>(Kb + (size_t)tg * DH);
+      uint32_t *vg = reinterpret_cast<uint32_t *>(Vb + (size_t)tg * DH);
+      kg[w1] = k1; kg[w2] = k2;
+      vg[w1] = v1; vg[w2] = v2;
+    }
+    for (int i = g.q_len * (DH / 2) + lane; i < G::CHUNK * (DH / 2); i += 32) vs[i] = 0u;
+    __syncwarp();
+    const uint32_t st32 = ring32 + (uint32_t)((G::STAGES - 1) * G::STAGE_BYTES);
+    chunk(st32, st32 + G::TILE_BYTES, p0, p0 + g.q_len);
+    // the first refill of this stage follows the warp barrier at the top of the loop below
+  }
+
+
+  for (int c = 0; c < nch; ++c) {
+    flash_wait<G::STAGES - 2>();
+    __syncwarp();
+    issue(c + G::STAGES - 1);                                  // refills the stage consumed in the previous turn
+    const uint32_t kst = ring32 + (uint32_t)((c % G::STAGES) * G::STAGE_BYTES);
+    chunk(kst, kst + G::TILE_BYTES, t_beg + c * G::CHUNK, t_end);
   }
   flash_wait<0>();
   __syncwarp();
@@ -217,7 +278,7 @@ attn_flash_kernel(const float *__restrict__ qkv, const bf16 *__restrict__ Kc, co
     l_run[rr] += __shfl_xor_sync(0xffffffffu, l_run[rr], 1);
     l_run[rr] += __shfl_xor_sync(0xffffffffu, l_run[rr], 2);
   }
-  if (split == 1) {
+  if (mode != FLASH_SPLIT) {
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
       const int i = gr + rr * 8;

@@ -309,8 +309,14 @@ int attn_set_attr(size_t bytes) {
   CU_TRY(cudaFuncSetAttribute(attn_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
   return TSFM_OK;
 }
-// Rows of at least this many keys (bf16 caches) take the running-softmax kernel.
-constexpr int kFlashMinCap = 192;
+// bf16 caches of at least this many rows take the running-softmax kernel for every pass (passes
+// of more than one query tile always do).
+#ifndef TSFM_FLASH_MIN_CAP
+#define TSFM_FLASH_MIN_CAP 0
+#endif
+constexpr int kFlashMinCap = TSFM_FLASH_MIN_CAP;
+// Short rows with at least this many (series, head) pairs: one warp per pair instead of four.
+constexpr int kFlashWarpMaxCap = 64, kFlashWarpMinPairs = 8 * 148;
 template <int DH> int flash_set_attr() {
   CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::SMEM_BYTES));
   return TSFM_OK;
@@ -449,18 +455,19 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
             4.0 * Mr * (std::max(g.base, 0) + 0.5 * g.q_len) * m.arch.d_model);
   // several query tiles, or long bf16 rows: the pass's keys and values go to the cache first, once
   const bool flash = sizeof(T) == 2 && (g.q_len > ATTN_QT || h->cap >= kFlashMinCap);
-  const int pre = (g.q_len > ATTN_QT || flash) ? 1 : 0;
+  const int pre = g.q_len > ATTN_QT ? 1 : 0;
   if (pre)
     launch_ex(h->ls, h->pdl, kv_append_kernel<T, DH>, dim3(m.arch.n_heads, B, (g.q_len + 15) / 16), dim3(128), 0,
               h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads);
   if constexpr (sizeof(T) == 2) {
     if (flash) {
-      // many queries: a warp per query tile; one tile: its keys dealt out over the four warps
-      const int split = g.q_len > ATTN_QT ? 1 : 4;
-      const int per_cta = split == 1 ? 4 * ATTN_QT : ATTN_QT;
-      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH>, dim3(m.arch.n_heads, B, (g.q_len + per_cta - 1) / per_cta),
-                dim3(128), (size_t)FlashGeom<DH>::SMEM_BYTES, h->qkv, (const bf16 *)Kc, (const bf16 *)Vc, m.rope, g,
-                m.arch.n_heads, split, (bf16 *)h->ao);
+      const int pairs = B * m.arch.n_heads;
+      const int mode = pre ? FLASH_TILES
+                           : (h->cap <= kFlashWarpMaxCap && pairs >= kFlashWarpMinPairs) ? FLASH_WARP : FLASH_SPLIT;
+      const dim3 fgrid = mode == FLASH_WARP ? dim3((pairs + 3) / 4)
+                                            : dim3(m.arch.n_heads, B, pre ? (g.q_len + 4 * ATTN_QT - 1) / (4 * ATTN_QT) : 1);
+      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH>, fgrid, dim3(128), (size_t)FlashGeom<DH>::SMEM_BYTES, h->qkv,
+                (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
       return;
     }
   }
