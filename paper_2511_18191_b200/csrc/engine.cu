@@ -292,15 +292,10 @@ template <typename T> size_t attn_smem_bytes(int dh, int nk) {
          2 * ATTN_QT * sizeof(float);
 }
 
-// Number of CTAs (one cluster) that share the keys of one (series, head, query tile): long rows
-// are split so that each CTA stages a quarter of the cache and more CTAs fit on an SM.
-#ifndef TSFM_ATTN_SKV
-#define TSFM_ATTN_SKV 4
-#endif
-#ifndef TSFM_ATTN_SKV_MIN_CAP
-#define TSFM_ATTN_SKV_MIN_CAP 192
-#endif
-inline int attn_key_split(int cap) { return cap >= TSFM_ATTN_SKV_MIN_CAP ? TSFM_ATTN_SKV : 1; }
+// fp32 caches: number of CTAs (one cluster) that share the keys of one (series, head, query
+// tile): long rows are split so that each CTA stages a quarter of the cache and more CTAs fit
+// on an SM.
+inline int attn_key_split(int cap) { return cap >= 192 ? 4 : 1; }
 // key rows one CTA must hold: its share of the longest row, in whole 16-key MMA blocks
 inline int attn_rows_per_cta(int cap, int skv) { return ((cap + skv - 1) / skv + 15) & ~15; }
 
@@ -309,12 +304,7 @@ int attn_set_attr(size_t bytes) {
   CU_TRY(cudaFuncSetAttribute(attn_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
   return TSFM_OK;
 }
-// bf16 caches of at least this many rows take the running-softmax kernel for every pass (passes
-// of more than one query tile always do).
-#ifndef TSFM_FLASH_MIN_CAP
-#define TSFM_FLASH_MIN_CAP 0
-#endif
-constexpr int kFlashMinCap = TSFM_FLASH_MIN_CAP;
+// bf16 caches take the running-softmax kernel (attn_flash_kernel), fp32 caches attn_kernel.
 // Short rows with at least this many (series, head) pairs: one warp per pair instead of four.
 constexpr int kFlashWarpMaxCap = 64, kFlashWarpMinPairs = 8 * 148;
 template <int DH> int flash_set_attr() {
@@ -323,15 +313,16 @@ template <int DH> int flash_set_attr() {
 }
 template <typename T>
 int attn_prepare(int dh, int cap) {
-  if (sizeof(T) == 2) {
-    if (int rc = dh == 32 ? flash_set_attr<32>() : dh == 64 ? flash_set_attr<64>() : flash_set_attr<128>()) return rc;
+  if constexpr (sizeof(T) == 2) {
+    return dh == 32 ? flash_set_attr<32>() : dh == 64 ? flash_set_attr<64>() : flash_set_attr<128>();
+  } else {
+    const size_t bytes = attn_smem_bytes<T>(dh, attn_rows_per_cta(cap, attn_key_split(cap)));
+    if (bytes > 227 * 1024) return TSFM_ERR_SHAPE;
+    const size_t optin = 227 * 1024;        // opt in once to the per-CTA maximum; launches size themselves
+    if (dh == 32) return attn_set_attr<T, 32>(optin);
+    if (dh == 64) return attn_set_attr<T, 64>(optin);
+    return attn_set_attr<T, 128>(optin);
   }
-  const size_t bytes = attn_smem_bytes<T>(dh, attn_rows_per_cta(cap, attn_key_split(cap)));
-  if (bytes > 227 * 1024) return TSFM_ERR_SHAPE;
-  const size_t optin = 227 * 1024;        // opt in once to the per-CTA maximum; launches size themselves
-  if (dh == 32) return attn_set_attr<T, 32>(optin);
-  if (dh == 64) return attn_set_attr<T, 64>(optin);
-  return attn_set_attr<T, 128>(optin);
 }
 
 // Every kernel of the library asks for the same (maximum) shared-memory carve-out, so that the
@@ -347,9 +338,11 @@ template <typename T> void prefer_max_smem_typed() {
   prefer_max_smem(gemm_simt_kernel<T, EPI_T>);
   prefer_max_smem(gemm_simt_kernel<T, EPI_GELU_T>);
   prefer_max_smem(gemm_simt_kernel<T, EPI_RESID>);
-  prefer_max_smem(attn_kernel<T, 32>);
-  prefer_max_smem(attn_kernel<T, 64>);
-  prefer_max_smem(attn_kernel<T, 128>);
+  if constexpr (sizeof(T) == 4) {
+    prefer_max_smem(attn_kernel<T, 32>);
+    prefer_max_smem(attn_kernel<T, 64>);
+    prefer_max_smem(attn_kernel<T, 128>);
+  }
   prefer_max_smem(kv_append_kernel<T, 32>);
   prefer_max_smem(kv_append_kernel<T, 64>);
   prefer_max_smem(kv_append_kernel<T, 128>);
@@ -441,11 +434,6 @@ void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C,
 
 template <typename T, int DH>
 void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
-  const int QT = g.q_len <= ATTN_QT ? g.q_len : ATTN_QT;
-  const int skv = attn_key_split(h->cap);
-  dim3 grid(m.arch.n_heads, B, ((g.q_len + QT - 1) / QT) * skv);
-  const int nk_max = attn_rows_per_cta(h->cap, skv);   // whole MMA blocks; regions stay 16-byte aligned
-  const size_t smem = attn_smem_bytes<T>(DH, nk_max);
   T *Kc = (T *)m.Kc + (size_t)l * m.kv_layer_elems;
   T *Vc = (T *)m.Vc + (size_t)l * m.kv_layer_elems;
   // algorithmic bytes: q/k/v of the pass + the cached keys and values (lower bound: done = 0)
@@ -453,30 +441,32 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   const double Mr = (double)B * g.q_len;
   KTimer kt(h, KC_ATTN, Mr * 3 * m.arch.d_model * 4 + kv + Mr * m.arch.d_model * (2.0 * sizeof(T) + sizeof(T)),
             4.0 * Mr * (std::max(g.base, 0) + 0.5 * g.q_len) * m.arch.d_model);
-  // several query tiles, or long bf16 rows: the pass's keys and values go to the cache first, once
-  const bool flash = sizeof(T) == 2 && (g.q_len > ATTN_QT || h->cap >= kFlashMinCap);
+  // several query tiles: the pass's keys and values go to the cache first, once
   const int pre = g.q_len > ATTN_QT ? 1 : 0;
   if (pre)
     launch_ex(h->ls, h->pdl, kv_append_kernel<T, DH>, dim3(m.arch.n_heads, B, (g.q_len + 15) / 16), dim3(128), 0,
               h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads);
   if constexpr (sizeof(T) == 2) {
-    if (flash) {
-      const int pairs = B * m.arch.n_heads;
-      const int mode = pre ? FLASH_TILES
-                           : (h->cap <= kFlashWarpMaxCap && pairs >= kFlashWarpMinPairs) ? FLASH_WARP : FLASH_SPLIT;
-      const dim3 fgrid = mode == FLASH_WARP ? dim3((pairs + 3) / 4)
-                                            : dim3(m.arch.n_heads, B, pre ? (g.q_len + 4 * ATTN_QT - 1) / (4 * ATTN_QT) : 1);
-      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH>, fgrid, dim3(128), (size_t)FlashGeom<DH>::SMEM_BYTES, h->qkv,
-                (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
-      return;
-    }
+    const int pairs = B * m.arch.n_heads;
+    const int mode = pre ? FLASH_TILES
+                         : (h->cap <= kFlashWarpMaxCap && pairs >= kFlashWarpMinPairs) ? FLASH_WARP : FLASH_SPLIT;
+    const dim3 grid = mode == FLASH_WARP ? dim3((pairs + 3) / 4)
+                                         : dim3(m.arch.n_heads, B, pre ? (g.q_len + 4 * ATTN_QT - 1) / (4 * ATTN_QT) : 1);
+    launch_ex(h->ls, h->pdl, attn_flash_kernel<DH>, grid, dim3(128), (size_t)FlashGeom<DH>::SMEM_BYTES, h->qkv,
+              (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
+  } else {
+    const int QT = g.q_len <= ATTN_QT ? g.q_len : ATTN_QT;
+    const int skv = attn_key_split(h->cap);
+    const dim3 grid(m.arch.n_heads, B, ((g.q_len + QT - 1) / QT) * skv);
+    const int nk_max = attn_rows_per_cta(h->cap, skv);   // regions stay 16-byte aligned
+    const size_t smem = attn_smem_bytes<T>(DH, nk_max);
+    if (skv > 1)
+      launch_ex_cluster(h->ls, h->pdl, skv, attn_kernel<T, DH>, grid, dim3(128), smem, h->qkv, Kc, Vc, m.rope, g,
+                        m.arch.n_heads, QT, nk_max, skv, pre, (T *)h->ao);
+    else
+      launch_ex(h->ls, h->pdl, attn_kernel<T, DH>, grid, dim3(128), smem, h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads,
+                QT, nk_max, skv, pre, (T *)h->ao);
   }
-  if (skv > 1)
-    launch_ex_cluster(h->ls, h->pdl, skv, attn_kernel<T, DH>, grid, dim3(128), smem, h->qkv, Kc, Vc, m.rope, g,
-                      m.arch.n_heads, QT, nk_max, skv, pre, (T *)h->ao);
-  else
-    launch_ex(h->ls, h->pdl, attn_kernel<T, DH>, grid, dim3(128), smem, h->qkv, Kc, Vc, m.rope, g, m.arch.n_heads, QT,
-              nk_max, skv, pre, (T *)h->ao);
 }
 
 enum { HEAD_NONE = 0, HEAD_LAST_TO_HIST = 1, HEAD_ALL_TO_VOUT = 2 };

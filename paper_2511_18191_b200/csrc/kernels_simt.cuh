@@ -233,19 +233,21 @@ gemm_simt_kernel(const T *__restrict__ A, const T *__restrict__ W, void *__restr
 }
 
 // ----------------------------------------------------------------------------------
-// RoPE + KV append + causal attention for one (head, series, query tile).
+// RoPE + KV append + causal attention for one (head, series, query tile): the kernel of the
+// fp32 caches (bf16 caches take attn_flash_kernel).
 //   qkv   [M, 3 d] fp32: q | k | v of this pass's tokens (row = b * q_len + j)
 //   Kc,Vc [B, heads, cap, DH] T: this layer's cache; positions < pos0 are valid
 //   rope  [cap, DH/2] float2 (cos, sin), rotate-half pairing (i, i + DH/2)
 //   out   [M, d] T
-// The CTA loads keys 0..pos0-1 from the cache (16-byte loads) and the keys of this pass
-// (rotated here) up to its last query into shared memory once; all queries of the tile share
-// that read.  The tile that owns a token writes its rotated key and its value to the cache.
-// grid = (heads, B, ceil(q_len / QT)), block = 128; the queries of a tile are processed together.
-// Shared memory is addressed in 32-bit words: K rows are padded by one word so that lanes
-// reading different keys hit different banks.
-//   K tile [nk][KW] words, V tile [nk][VW] words, scores [16][nk] f32, q [16][DH] f32,
-//   partial outputs [4][16][DH] f32, 1/sum [16] f32.
+// The CTA loads keys 0..pos0-1 from the cache (16-byte asynchronous copies) and the keys of this
+// pass (rotated here, or appended beforehand by kv_append_kernel when the pass has several query
+// tiles) up to its last query into shared memory once; all queries of the tile share that read.
+// The tile that owns a token writes its rotated key and its value to the cache.
+// grid = (heads, B, ceil(q_len / QT) * skv), block = 128; the queries of a tile are processed
+// together.  Shared memory is addressed in 32-bit words; key rows are dense with their 16-byte
+// chunks rotated by the row index (attn_kword).
+//   V tile [nk][VW] words, K tile [nk][KW] words, scores [16][nk] f32, q [16][DH] f32,
+//   partial outputs [4][16][DH] f32, row maxima [16] and row sums [16] f32.
 // ----------------------------------------------------------------------------------
 template <typename T> struct AttnWords;                 // words per DH elements
 template <> struct AttnWords<float> {
@@ -365,15 +367,8 @@ __device__ __forceinline__ void attn_tile(const uint32_t *Ks, const uint32_t *Vs
   __syncthreads();
 }
 
-// ----------------------------------------------------------------------------------
-// The same tile computation on the warp-level tensor-core path (mma.sync m16n8k16, bf16 operands,
-// fp32 accumulate) for bf16 caches: the query tile (at most 16 rows) is the M side of both
-// products.  S = Q K^T: each warp takes every fourth block of 8 keys; the rotated fp32 queries
-// are split into a bf16 high and low part (two MMAs) so that the scores keep fp32-like accuracy.
-// O = P V: each warp takes every fourth block of 16 keys, P rounded to bf16, V fragments by
-// ldmatrix.trans; the four partial outputs are summed as in attn_tile.  sc rows >= nq are zero,
-// key columns in [nk, round_up(nk, 16)) get probability 0 and V rows there are zero.
-// ----------------------------------------------------------------------------------
+// Warp-level tensor-core helpers (mma.sync m16n8k16, bf16 operands, fp32 accumulate) and the
+// split of an fp32 pair into bf16 high and low parts, used by the bf16 attention kernel.
 __device__ __forceinline__ void mma_bf16_16816(float *c, const uint32_t *a, uint32_t b0, uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -383,104 +378,6 @@ __device__ __forceinline__ void split_bf16x2(float x, float y, uint32_t &hi, uin
   const float xh = __bfloat162float(__float2bfloat16_rn(x)), yh = __bfloat162float(__float2bfloat16_rn(y));
   hi = pack_bf16x2(xh, yh);
   lo = pack_bf16x2(x - xh, y - yh);
-}
-
-template <int DH>
-__device__ __forceinline__ void attn_tile_mma(const uint32_t *Ks, const uint32_t *Vs, float *sc, const float *qs, float *po,
-                                              float *row_max, float *row_sum, int nq, int nk, int nk_max, int k_lo,
-                                              int p0, int j_lo) {
-  constexpr int VW = DH / 2, KS = DH / 16;
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int g = lane >> 2, q4 = lane & 3;            // fragment row group, column pair
-  const int nk16 = (nk + 15) & ~15;
-  {
-    // ---- scores
-    uint32_t qhi[KS][4], qlo[KS][4];
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      const int c = ks * 16 + q4 * 2;
-      const float2 a = *reinterpret_cast<const float2 *>(qs + g * DH + c);
-      const float2 b = *reinterpret_cast<const float2 *>(qs + (g + 8) * DH + c);
-      const float2 a8 = *reinterpret_cast<const float2 *>(qs + g * DH + c + 8);
-      const float2 b8 = *reinterpret_cast<const float2 *>(qs + (g + 8) * DH + c + 8);
-      split_bf16x2(a.x, a.y, qhi[ks][0], qlo[ks][0]);
-      split_bf16x2(b.x, b.y, qhi[ks][1], qlo[ks][1]);
-      split_bf16x2(a8.x, a8.y, qhi[ks][2], qlo[ks][2]);
-      split_bf16x2(b8.x, b8.y, qhi[ks][3], qlo[ks][3]);
-    }
-    for (int nt = w; nt < nk16 / 8; nt += 4) {
-      const int key = nt * 8 + g;                    // B fragment: this lane's key row
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        const uint32_t b0 = Ks[attn_kword<VW>(key, ks * 8 + q4)], b1 = Ks[attn_kword<VW>(key, ks * 8 + 4 + q4)];
-        mma_bf16_16816(c, qhi[ks], b0, b1);
-        mma_bf16_16816(c, qlo[ks], b0, b1);
-      }
-      const int t = nt * 8 + q4 * 2;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int r = g + (e >> 1) * 8, tt = t + (e & 1);
-        if (r < nq) sc[(size_t)r * nk_max + tt] = (k_lo + tt <= p0 + j_lo + r && tt < nk) ? c[e] : -INFINITY;
-      }
-    }
-  }
-  __syncthreads();
-  for (int i = w; i < nq; i += 4) {
-    float *row = sc + (size_t)i * nk_max;
-    float mx = -INFINITY;
-    for (int t = lane; t < nk16; t += 32) mx = fmaxf(mx, row[t]);
-    mx = warp_max(mx);
-    float sum = 0.f;
-    for (int t = lane; t < nk16; t += 32) {
-      const float pv = mx == -INFINITY ? 0.f : expf(row[t] - mx);   // no visible key in this CTA's range
-      row[t] = pv;
-      sum += pv;
-    }
-    sum = warp_sum(sum);
-    if (lane == 0) { row_max[i] = mx; row_sum[i] = sum; }
-  }
-  __syncthreads();
-  {
-    // ---- P . V
-    float acc[DH / 8][4];
-#pragma unroll
-    for (int n = 0; n < DH / 8; ++n)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[n][e] = 0.f;
-    const uint32_t vbase = (uint32_t)__cvta_generic_to_shared(Vs);
-    for (int kb = w; kb < nk16 / 16; kb += 4) {
-      const int t = kb * 16 + q4 * 2;
-      uint32_t a[4];
-      {
-        const float2 p0v = *reinterpret_cast<const float2 *>(sc + (size_t)g * nk_max + t);
-        const float2 p1v = *reinterpret_cast<const float2 *>(sc + (size_t)(g + 8) * nk_max + t);
-        const float2 p2v = *reinterpret_cast<const float2 *>(sc + (size_t)g * nk_max + t + 8);
-        const float2 p3v = *reinterpret_cast<const float2 *>(sc + (size_t)(g + 8) * nk_max + t + 8);
-        a[0] = pack_bf16x2(p0v.x, p0v.y); a[1] = pack_bf16x2(p1v.x, p1v.y);
-        a[2] = pack_bf16x2(p2v.x, p2v.y); a[3] = pack_bf16x2(p3v.x, p3v.y);
-      }
-      // ldmatrix.x4.trans: matrices (keys 0-7 | 8-15) x (dims n0..n0+7 | n0+8..n0+15)
-      const int mrow = kb * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
-#pragma unroll
-      for (int n0 = 0; n0 < DH; n0 += 16) {
-        uint32_t b[4];
-        const uint32_t addr = vbase + (uint32_t)(mrow * VW * 4 + (n0 + mcol) * 2);
-        asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]) : "r"(addr));
-        mma_bf16_16816(acc[n0 / 8], a, b[0], b[1]);
-        mma_bf16_16816(acc[n0 / 8 + 1], a, b[2], b[3]);
-      }
-    }
-#pragma unroll
-    for (int n = 0; n < DH / 8; ++n)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int r = g + (e >> 1) * 8, c = n * 8 + q4 * 2 + (e & 1);
-        if (r < nq) po[((size_t)w * ATTN_QT + r) * DH + c] = acc[n][e];
-      }
-  }
-  __syncthreads();
 }
 
 // Keys and values of a pass with several query tiles go to the cache once, before attention:
@@ -639,9 +536,8 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   const float scale = rsqrtf((float)DH);
   const int nq = j_hi - j_lo;                        // <= ATTN_QT
   const int nk = k_hi - k_lo;                        // key rows held here
-  // rows the tile routine will touch: its compile-time query bound (16 on the tensor-core path)
-  const bool use_mma = BF && nq >= 3 && nk_all >= 96;
-  const int nqb = use_mma ? ATTN_QT : nq <= 2 ? nq : nq <= 4 ? 4 : nq <= 6 ? 6 : nq <= 9 ? 9 : ATTN_QT;
+  // rows the tile routine will touch: its compile-time query bound
+  const int nqb = nq <= 2 ? nq : nq <= 4 ? 4 : nq <= 6 ? 6 : nq <= 9 ? 9 : ATTN_QT;
   for (int idx = tid; idx < nqb * HALF; idx += blockDim.x) {       // rotated, scaled queries (zero past nq)
     const int i = idx / HALF, c = idx % HALF, j = j_lo + i;
     float r1 = 0.f, r2 = 0.f;
@@ -658,13 +554,7 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   for (int idx = tid + nq * nk_max; idx < nqb * nk_max; idx += blockDim.x) sc[idx] = 0.f;       // unused score rows
   asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
-  if (use_mma) {                                     // tensor-core tile routine (bf16 caches, long rows: measured)
-    const int nk16 = (nk + 15) & ~15;
-    for (int idx = tid + nk * VW; idx < nk16 * VW; idx += blockDim.x) Vs[idx] = 0u;   // value rows of the padding keys
-    __syncthreads();
-    if constexpr (BF) attn_tile_mma<DH>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
-  }
-  else if (nq == 1) attn_tile<T, DH, 1>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
+  if (nq == 1) attn_tile<T, DH, 1>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
   else if (nq == 2) attn_tile<T, DH, 2>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
   else if (nq <= 4) attn_tile<T, DH, 4>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
   else if (nq <= 6) attn_tile<T, DH, 6>(Ks, Vs, sc, qs, po, row_max, row_sum, nq, nk, nk_max, k_lo, p0, j_lo);
