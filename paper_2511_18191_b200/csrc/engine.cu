@@ -354,9 +354,9 @@ void prefer_max_smem_all() {
   prefer_max_smem(denorm_kernel);
   prefer_max_smem(accept_kernel);
   prefer_max_smem(round_end_kernel);
-  prefer_max_smem(gemm_sk_kernel<1, false, false>);
-  prefer_max_smem(gemm_sk_kernel<1, false, true>);
-  prefer_max_smem(gemm_sk_kernel<2, true, false>);
+  prefer_max_smem(gemm_sk_kernel<1, false>);
+  prefer_max_smem(gemm_sk_kernel<1, true>);
+  prefer_max_smem(gemm_sk_kernel<2, false>);
   prefer_max_smem(pass_cluster_kernel);
   prefer_max_smem(attn_flash_kernel<32>);
   prefer_max_smem(attn_flash_kernel<64>);

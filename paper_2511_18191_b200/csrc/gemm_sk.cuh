@@ -13,9 +13,14 @@
 //     r, r + S, ... of all S partial tiles through distributed shared memory and applies the
 //     epilogue once.  No atomics, no pre-zeroed accumulator, a fixed summation order, and every
 //     epilogue (GELU included) can be split.
+//   * a residual epilogue (x += A W^T) on a feature count that is a multiple of 128 leaves the
+//     read-modify-write to the TMA unit: the tile (summed over the cluster first) is staged in
+//     shared memory as [token][128 features] fp32 and added to x by one
+//     cp.reduce.async.bulk.tensor per CTA, so no thread waits for the old values of x.
 // Warp roles and bounded waits as in gemm_tc.cuh.
 #pragma once
 #include "gemm_tc.cuh"
+#include <vector>
 
 namespace tsfm {
 
@@ -80,14 +85,22 @@ __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi)
 
 // grid = (ceil(N / 128), ceil(M / BN), S), cluster = (1, 1, S), block = 192.
 // ring_bytes = size of the tile region (a multiple of 1024); barriers sit behind it.
-// WT = weight tiles per CTA; WIDE = compile the 64-token residual epilogue (only with two weight
-// tiles, one CTA per SM: it costs registers that launches with several CTAs per SM cannot spare).
+// WT = weight tiles per CTA.
 // NORM = compile the folded-RMSNorm epilogues (SkNorm); the plain instantiations carry none of it.
-template <int WT, bool WIDE, bool NORM>
+// tma_c != 0: residual epilogue through mapC (fp32 [M][N], box = BN / S tokens x 128 features).
+__device__ __forceinline__ void sk_tma_reduce_add(const CUtensorMap *map, uint32_t src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+template <int WT, bool NORM>
 __global__ void __launch_bounds__(192, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
-               void *__restrict__ C, int M, int N, int K, int BN, int stages, int tmem_cols, int ring_bytes,
-               int epi, const SkNorm nm, int *__restrict__ status) {
+               const __grid_constant__ CUtensorMap mapC, void *__restrict__ C, int M, int N, int K, int BN,
+               int stages, int tmem_cols, int ring_bytes, int epi, int tma_c, const SkNorm nm,
+               int *__restrict__ status) {
   constexpr int wt = WT;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -185,72 +198,61 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       umma_commit(empty0 + 8 * s);
     }
     if (ok) umma_commit(accum);
-  } else if (warp < 4) {
-    // ---------------- epilogue, part 1: drain the accumulator
-    if (KB > 0 && mbar_wait(accum, 0)) {
-      tc_fence_after();
-      const int fl = warp * 32 + lane;
-      const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16);
+  }
+  // ---------------- epilogue, part 1: drain the accumulator(s), one weight tile at a time
+  const bool staged = S > 1 || tma_c;                  // through shared memory ([token][128 features] fp32)
+  bool acc_ok = false;
+  if (warp < 4) {
+    acc_ok = KB > 0 && mbar_wait(accum, 0);
+    if (!acc_ok && KB > 0 && lane == 0) atomicExch(status, DEV_TIMEOUT_EPILOGUE);
+    tc_fence_after();
+  }
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN * wt; c0 += 16) {
-        const int q = c0 >= BN ? 1 : 0, cc = c0 - q * BN;      // weight tile, column inside it
-        const int f = f0 + q * TC_BM + fl;
-        if (t0 + cc >= M) { if (q + 1 < wt) { c0 = BN - 16; continue; } break; }
-        if (WIDE && S == 1 && epi == EPI_RESID && f < N && cc + 64 <= BN && t0 + cc + 64 <= M) {
-          // residual epilogue, 64 tokens at a time: the 64 old values are requested before the
-          // accumulator is read, so one L2 round trip covers them all
-          float r[64], v[64];
-          float *cp = (float *)C + (size_t)(t0 + cc) * N + f;
-#pragma unroll
-          for (int j = 0; j < 64; ++j) r[j] = cp[(size_t)j * N];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) tmem_ld16(tbase + c0 + 16 * u, v + 16 * u);
-#pragma unroll
-          for (int j = 0; j < 64; ++j) {
-            const float xn = r[j] + v[j];
-            cp[(size_t)j * N] = xn;
-            if (NORM && nm.a_out) {
-              nm.a_out[(size_t)(t0 + cc + j) * N + f] = __float2bfloat16_rn(nm.gain[f] * xn);
-              const float sq = warp_sum(xn * xn);
-              if (lane == 0) nm.ssq_out[(size_t)(t0 + cc + j) * (N >> 5) + (f >> 5)] = sq;
-            }
-          }
-          c0 += 48;
-          continue;
-        }
+  for (int q = 0; q < wt; ++q) {
+    if (warp < 4 && acc_ok) {
+      const int fl = warp * 32 + lane, f = f0 + q * TC_BM + fl;
+      const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(q * BN);
+#pragma unroll 1
+      for (int cc = 0; cc < BN; cc += 16) {
+        if (t0 + cc >= M) break;
         float v[16];
-        tmem_ld16(tbase + c0, v);
-        if (S == 1) {
-          if (f < N) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (t0 + cc + j < M) {
-                const size_t o = (size_t)(t0 + cc + j) * N + f;
-                if (NORM && nm.ssq_in) v[j] *= rs[cc + j];
-                if (NORM && epi == EPI_RESID && nm.a_out) {
-                  const float xn = ((float *)C)[o] + v[j];
-                  ((float *)C)[o] = xn;
-                  nm.a_out[o] = __float2bfloat16_rn(nm.gain[f] * xn);
-                  v[j] = xn * xn;
-                } else {
-                  sk_store_rt(C, o, v[j], epi);
-                }
-              }
-          }
-          if (NORM && epi == EPI_RESID && nm.a_out) {          // slice sums of squares (N is a multiple of 32 here)
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const float sq = warp_sum(v[j]);
-              if (lane == 0 && t0 + cc + j < M) nm.ssq_out[(size_t)(t0 + cc + j) * (N >> 5) + (f >> 5)] = sq;
-            }
-          }
-        } else {
+        tmem_ld16(tbase + cc, v);
+        if (staged) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) stage_f[(cc + j) * TC_BM + fl] = v[j];
+          continue;
+        }
+        if (f < N) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (t0 + cc + j < M) {
+              const size_t o = (size_t)(t0 + cc + j) * N + f;
+              if (NORM && nm.ssq_in) v[j] *= rs[cc + j];
+              if (NORM && epi == EPI_RESID && nm.a_out) {
+                const float xn = ((float *)C)[o] + v[j];
+                ((float *)C)[o] = xn;
+                nm.a_out[o] = __float2bfloat16_rn(nm.gain[f] * xn);
+                v[j] = xn * xn;
+              } else {
+                sk_store_rt(C, o, v[j], epi);
+              }
+            }
+        }
+        if (NORM && epi == EPI_RESID && nm.a_out) {          // slice sums of squares (N is a multiple of 32 here)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float sq = warp_sum(v[j]);
+            if (lane == 0 && t0 + cc + j < M) nm.ssq_out[(size_t)(t0 + cc + j) * (N >> 5) + (f >> 5)] = sq;
+          }
         }
       }
-    } else if (KB > 0 && lane == 0) {
-      atomicExch(status, DEV_TIMEOUT_EPILOGUE);
+    }
+    if (tma_c && S == 1 && warp < 4) {
+      // the staged tile goes to x as one TMA reduction (rows past M are clipped by the map)
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("bar.sync 2, 128;" ::: "memory");
+      if (threadIdx.x == 0 && acc_ok) sk_tma_reduce_add(&mapC, tiles, f0 + q * TC_BM, t0);
+      asm volatile("bar.sync 2, 128;" ::: "memory");       // the stage is free again
     }
   }
   __syncwarp();
@@ -258,7 +260,36 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
     // ---------------- epilogue, part 2: reduce the S partial tiles through distributed shared memory
     tc_fence_before();
     cluster_sync_all();
-    if (warp < 4) {
+    if (warp < 4 && tma_c) {
+      // CTA r sums its block of BN / S rows over the S partial tiles, in place in its own tile,
+      // and hands the block to the TMA unit
+      const int RB = BN / S, rg = threadIdx.x >> 5, c4 = (threadIdx.x & 31) * 4;
+      uint32_t remote[SK_MAX_SPLIT];
+#pragma unroll
+      for (int r = 0; r < SK_MAX_SPLIT; ++r) {
+        const uint32_t a = tiles + (uint32_t)c4 * 4;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote[r]) : "r"(a), "r"((uint32_t)(r < S ? r : 0)));
+      }
+      for (int tl = rank * RB + rg; tl < (rank + 1) * RB; tl += 4) {
+        if (t0 + tl >= M) break;
+        float4 v[SK_MAX_SPLIT];
+#pragma unroll
+        for (int r = 0; r < SK_MAX_SPLIT; ++r)
+          if (r < S)
+            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                         : "=f"(v[r].x), "=f"(v[r].y), "=f"(v[r].z), "=f"(v[r].w)
+                         : "r"(remote[r] + (uint32_t)tl * (TC_BM * 4)) : "memory");
+        float4 sum = v[0];
+#pragma unroll
+        for (int r = 1; r < SK_MAX_SPLIT; ++r)
+          if (r < S) { sum.x += v[r].x; sum.y += v[r].y; sum.z += v[r].z; sum.w += v[r].w; }
+        *reinterpret_cast<float4 *>(stage_f + (size_t)tl * TC_BM + c4) = sum;
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("bar.sync 2, 128;" ::: "memory");
+      if (threadIdx.x == 0 && t0 + rank * RB < M)
+        sk_tma_reduce_add(&mapC, tiles + (uint32_t)(rank * RB) * (TC_BM * 4), f0, t0 + rank * RB);
+    } else if (warp < 4) {
       // thread -> (row group, 4 consecutive features): one 16-byte load per partial tile, all S
       // loads of a row in flight together, one 16-byte (fp32) or 8-byte (bf16) store per row
       const int rg = threadIdx.x >> 5, c4 = (threadIdx.x & 31) * 4, f = f0 + c4;
@@ -339,15 +370,30 @@ struct GemmSkPlan {
   CUtensorMap mapW;
   CUtensorMap mapA[16];            // box (BN = 16 * (i + 1)) x 64, encoded on first use
   bool haveA[16] = {false};
+  // residual outputs x [M][N] fp32 for the TMA reduction, one map per (x, M, rows per box)
+  struct CMap { const void *C; int M, rows; CUtensorMap map; };
+  std::vector<CMap> mapC;
 };
+
+// fp32 [rows][N] row-major, box = box_rows x 128 features, no swizzle.
+static int sk_encode_c(CUtensorMap *map, const void *base, int rows, int N, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+  cuuint32_t box[2] = {(cuuint32_t)TC_BM, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -4;
+}
 
 static int gemm_sk_init() {
   if (int rc = gemm_tc_init()) return rc;
   static bool done = false;
   if (done) return 0;
-  if (cudaFuncSetAttribute(gemm_sk_kernel<1, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_sk_kernel<1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_sk_kernel<2, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+  if (cudaFuncSetAttribute(gemm_sk_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_sk_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_sk_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
     return -4;
   done = true;
   return 0;
@@ -357,6 +403,7 @@ static int gemm_sk_plan(GemmSkPlan *plan, const void *W, int N, int K, const voi
   plan->valid = false;
   plan->N = N; plan->K = K; plan->M_max = M_max; plan->A = A;
   for (bool &b : plan->haveA) b = false;
+  plan->mapC.clear();
   if (K % 8 || K < 16 || N < 1 || M_max < 1) return 0;
   if (((uintptr_t)W & 15) || ((uintptr_t)A & 15)) return 0;
   if (!g_encode) return -4;
@@ -414,9 +461,26 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   }
   const int KB = (p.K + TC_BK - 1) / TC_BK;
   const int FT = (p.N + TC_BM - 1) / TC_BM, TT = (M + BN - 1) / BN;
-  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1, wt);
+  // residual epilogue through the TMA unit: x and its row pitch 16-byte aligned, whole feature tiles
+  const bool tma_c = epi == EPI_RESID && !norm && p.N % TC_BM == 0 && BN % S == 0 && !((uintptr_t)C & 15);
+  const CUtensorMap *mapC = &p.mapW;                         // placeholder when unused
+  if (tma_c) {
+    const int rows = BN / S;
+    const GemmSkPlan::CMap *hit = nullptr;
+    for (const auto &c : p.mapC)
+      if (c.C == C && c.M == M && c.rows == rows) { hit = &c; break; }
+    if (!hit) {
+      GemmSkPlan::CMap c{C, M, rows, {}};
+      if (sk_encode_c(&c.map, C, M, p.N, rows)) return false;
+      p.mapC.push_back(c);
+      hit = &p.mapC.back();
+    }
+    mapC = &hit->map;
+  }
+  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1 || tma_c, wt);
   const int ring_bytes = sh.smem_bytes - 1024 - 256 - 1024;
   const SkNorm nm = norm ? *norm : SkNorm{};
+  const int tc = tma_c ? 1 : 0;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((FT + wt - 1) / wt, TT, S);
   cfg.blockDim = dim3(192);
@@ -431,13 +495,13 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   cfg.numAttrs = pdl ? 2 : 1;
   int N = p.N, K = p.K, stages = sh.stages, cols = sh.tmem_cols, rb = ring_bytes;
   if (wt == 2)
-    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<2, true, false>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
-                              nm, status) == cudaSuccess;
+    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<2, false>, p.mapW, p.mapA[idx], *mapC, C, M, N, K, BN, stages, cols, rb,
+                              epi, tc, nm, status) == cudaSuccess;
   if (norm)
-    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, false, true>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb,
-                              epi, nm, status) == cudaSuccess;
-  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, false, false>, p.mapW, p.mapA[idx], C, M, N, K, BN, stages, cols, rb, epi,
-                            nm, status) == cudaSuccess;
+    return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, true>, p.mapW, p.mapA[idx], *mapC, C, M, N, K, BN, stages, cols, rb,
+                              epi, tc, nm, status) == cudaSuccess;
+  return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, false>, p.mapW, p.mapA[idx], *mapC, C, M, N, K, BN, stages, cols, rb,
+                            epi, tc, nm, status) == cudaSuccess;
 }
 
 }  // namespace tsfm
