@@ -94,4 +94,20 @@ __device__ __forceinline__ float gelu_erf(float v) {
   return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
 }
 
+// The same function for epilogues that round their result to bf16: v * Phi(v) with
+// erfc(z) = t (a1 + t (a2 + t (a3 + t (a4 + t a5)))) exp(-z^2), t = 1 / (1 + p z), z = |v| / sqrt(2)
+// (Abramowitz & Stegun 7.1.26, absolute error of erf below 1.5e-7, far inside half a bf16 ulp),
+// two special-function instructions and no branch instead of erff's two divergent paths.
+// Phi(-|v|) = erfc(z) / 2 is taken directly, so the negative side has no cancellation.
+__device__ __forceinline__ float gelu_erf_fast(float v) {
+  const float z = fabsf(v) * 0.70710678118654752440f;
+  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+  float poly = fmaf(t, 1.061405429f, -1.453152027f);
+  poly = fmaf(t, poly, 1.421413741f);
+  poly = fmaf(t, poly, -0.284496736f);
+  poly = fmaf(t, poly, 0.254829592f);
+  const float half_erfc = 0.5f * t * poly * __expf(-z * z);
+  return v * (v >= 0.f ? 1.0f - half_erfc : half_erfc);
+}
+
 }  // namespace tsfm

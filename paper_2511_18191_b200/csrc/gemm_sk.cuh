@@ -79,7 +79,7 @@ static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1) {
 __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi) {
   if (epi == EPI_F32) ((float *)C)[o] = v;
   else if (epi == EPI_T) ((bf16 *)C)[o] = __float2bfloat16_rn(v);
-  else if (epi == EPI_GELU_T) ((bf16 *)C)[o] = __float2bfloat16_rn(gelu_erf(v));
+  else if (epi == EPI_GELU_T) ((bf16 *)C)[o] = __float2bfloat16_rn(gelu_erf_fast(v));
   else ((float *)C)[o] += v;
 }
 
@@ -87,7 +87,18 @@ __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi)
 // ring_bytes = size of the tile region (a multiple of 1024); barriers sit behind it.
 // WT = weight tiles per CTA.
 // NORM = compile the folded-RMSNorm epilogues (SkNorm); the plain instantiations carry none of it.
-// tma_c != 0: residual epilogue through mapC (fp32 [M][N], box = BN / S tokens x 128 features).
+// tma_c = SK_TMA_ADD: residual epilogue through mapC (fp32 [M][N], box = BN / S tokens x 128 features);
+// tma_c = SK_TMA_BF16 (S = 1 only): bf16 output (with or without GELU) staged as [token][128
+// features] bf16 and written by one TMA store per weight tile through mapC (bf16 [M][N]) -- whole
+// 128-byte lines at once, where per-thread 2-byte stores leave each line to be completed by a
+// second warp later.
+enum { SK_TMA_NONE = 0, SK_TMA_ADD = 1, SK_TMA_BF16 = 2 };
+__device__ __forceinline__ void sk_tma_store(const CUtensorMap *map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
 __device__ __forceinline__ void sk_tma_reduce_add(const CUtensorMap *map, uint32_t src, int x, int y) {
   asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
@@ -217,6 +228,13 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
         if (t0 + cc >= M) break;
         float v[16];
         tmem_ld16(tbase + cc, v);
+        if (tma_c == SK_TMA_BF16) {
+          bf16 *stage_h = reinterpret_cast<bf16 *>(stage_f);
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            stage_h[(cc + j) * TC_BM + fl] = __float2bfloat16_rn(epi == EPI_GELU_T ? gelu_erf_fast(v[j]) : v[j]);
+          continue;
+        }
         if (staged) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) stage_f[(cc + j) * TC_BM + fl] = v[j];
@@ -251,7 +269,10 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       // the staged tile goes to x as one TMA reduction (rows past M are clipped by the map)
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("bar.sync 2, 128;" ::: "memory");
-      if (threadIdx.x == 0 && acc_ok) sk_tma_reduce_add(&mapC, tiles, f0 + q * TC_BM, t0);
+      if (threadIdx.x == 0 && acc_ok) {
+        if (tma_c == SK_TMA_ADD) sk_tma_reduce_add(&mapC, tiles, f0 + q * TC_BM, t0);
+        else sk_tma_store(&mapC, tiles, f0 + q * TC_BM, t0);
+      }
       asm volatile("bar.sync 2, 128;" ::: "memory");       // the stage is free again
     }
   }
@@ -260,7 +281,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
     // ---------------- epilogue, part 2: reduce the S partial tiles through distributed shared memory
     tc_fence_before();
     cluster_sync_all();
-    if (warp < 4 && tma_c) {
+    if (warp < 4 && tma_c == SK_TMA_ADD) {
       // CTA r sums its block of BN / S rows over the S partial tiles, in place in its own tile,
       // and hands the block to the TMA unit
       const int RB = BN / S, rg = threadIdx.x >> 5, c4 = (threadIdx.x & 31) * 4;
@@ -337,7 +358,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
               if ((threadIdx.x & 7) == 0) nm.ssq_out[(size_t)t * (N >> 5) + (f >> 5)] = sq;
             }
           } else {
-            if (epi == EPI_GELU_T) { sum.x = gelu_erf(sum.x); sum.y = gelu_erf(sum.y); sum.z = gelu_erf(sum.z); sum.w = gelu_erf(sum.w); }
+            if (epi == EPI_GELU_T) { sum.x = gelu_erf_fast(sum.x); sum.y = gelu_erf_fast(sum.y); sum.z = gelu_erf_fast(sum.z); sum.w = gelu_erf_fast(sum.w); }
             const __nv_bfloat162 lo = __floats2bfloat162_rn(sum.x, sum.y), hi = __floats2bfloat162_rn(sum.z, sum.w);
             uint2 pk;
             pk.x = *reinterpret_cast<const uint32_t *>(&lo);
@@ -370,18 +391,20 @@ struct GemmSkPlan {
   CUtensorMap mapW;
   CUtensorMap mapA[16];            // box (BN = 16 * (i + 1)) x 64, encoded on first use
   bool haveA[16] = {false};
-  // residual outputs x [M][N] fp32 for the TMA reduction, one map per (x, M, rows per box)
-  struct CMap { const void *C; int M, rows; CUtensorMap map; };
+  // outputs written by the TMA unit (fp32 residual stream, bf16 activations): one map per
+  // (buffer, M, rows per box, element type)
+  struct CMap { const void *C; int M, rows; bool is_bf16; CUtensorMap map; };
   std::vector<CMap> mapC;
 };
 
 // fp32 [rows][N] row-major, box = box_rows x 128 features, no swizzle.
-static int sk_encode_c(CUtensorMap *map, const void *base, int rows, int N, int box_rows) {
+static int sk_encode_c(CUtensorMap *map, const void *base, int rows, int N, int box_rows, bool is_bf16) {
   cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+  cuuint64_t strides[1] = {(cuuint64_t)N * (is_bf16 ? 2 : 4)};
   cuuint32_t box[2] = {(cuuint32_t)TC_BM, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), dims, strides, box, estr,
+  CUresult r = g_encode(map, is_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                        const_cast<void *>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : -4;
@@ -462,16 +485,21 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   const int KB = (p.K + TC_BK - 1) / TC_BK;
   const int FT = (p.N + TC_BM - 1) / TC_BM, TT = (M + BN - 1) / BN;
   // residual epilogue through the TMA unit: x and its row pitch 16-byte aligned, whole feature tiles
-  const bool tma_c = epi == EPI_RESID && !norm && p.N % TC_BM == 0 && BN % S == 0 && !((uintptr_t)C & 15);
+  int tma_c = SK_TMA_NONE;
+  if (!norm && p.N % TC_BM == 0 && BN % S == 0 && !((uintptr_t)C & 15)) {
+    if (epi == EPI_RESID) tma_c = SK_TMA_ADD;
+    else if ((epi == EPI_T || epi == EPI_GELU_T) && S == 1) tma_c = SK_TMA_BF16;
+  }
   const CUtensorMap *mapC = &p.mapW;                         // placeholder when unused
   if (tma_c) {
     const int rows = BN / S;
+    const bool hb = tma_c == SK_TMA_BF16;
     const GemmSkPlan::CMap *hit = nullptr;
     for (const auto &c : p.mapC)
-      if (c.C == C && c.M == M && c.rows == rows) { hit = &c; break; }
+      if (c.C == C && c.M == M && c.rows == rows && c.is_bf16 == hb) { hit = &c; break; }
     if (!hit) {
-      GemmSkPlan::CMap c{C, M, rows, {}};
-      if (sk_encode_c(&c.map, C, M, p.N, rows)) return false;
+      GemmSkPlan::CMap c{C, M, rows, hb, {}};
+      if (sk_encode_c(&c.map, C, M, p.N, rows, hb)) return false;
       p.mapC.push_back(c);
       hit = &p.mapC.back();
     }
@@ -480,7 +508,7 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1 || tma_c, wt);
   const int ring_bytes = sh.smem_bytes - 1024 - 256 - 1024;
   const SkNorm nm = norm ? *norm : SkNorm{};
-  const int tc = tma_c ? 1 : 0;
+  const int tc = tma_c;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((FT + wt - 1) / wt, TT, S);
   cfg.blockDim = dim3(192);
