@@ -92,7 +92,8 @@ __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi)
 // features] bf16 and written by one TMA store per weight tile through mapC (bf16 [M][N]) -- whole
 // 128-byte lines at once, where per-thread 2-byte stores leave each line to be completed by a
 // second warp later.
-enum { SK_TMA_NONE = 0, SK_TMA_ADD = 1, SK_TMA_BF16 = 2 };
+// tma_c = SK_TMA_F32: fp32 output, staged (and summed over the cluster) like SK_TMA_ADD, stored.
+enum { SK_TMA_NONE = 0, SK_TMA_ADD = 1, SK_TMA_BF16 = 2, SK_TMA_F32 = 3 };
 __device__ __forceinline__ void sk_tma_store(const CUtensorMap *map, uint32_t src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
@@ -281,7 +282,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
     // ---------------- epilogue, part 2: reduce the S partial tiles through distributed shared memory
     tc_fence_before();
     cluster_sync_all();
-    if (warp < 4 && tma_c == SK_TMA_ADD) {
+    if (warp < 4 && (tma_c == SK_TMA_ADD || tma_c == SK_TMA_F32)) {
       // CTA r sums its block of BN / S rows over the S partial tiles, in place in its own tile,
       // and hands the block to the TMA unit
       const int RB = BN / S, rg = threadIdx.x >> 5, c4 = (threadIdx.x & 31) * 4;
@@ -308,8 +309,10 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("bar.sync 2, 128;" ::: "memory");
-      if (threadIdx.x == 0 && t0 + rank * RB < M)
-        sk_tma_reduce_add(&mapC, tiles + (uint32_t)(rank * RB) * (TC_BM * 4), f0, t0 + rank * RB);
+      if (threadIdx.x == 0 && t0 + rank * RB < M) {
+        if (tma_c == SK_TMA_ADD) sk_tma_reduce_add(&mapC, tiles + (uint32_t)(rank * RB) * (TC_BM * 4), f0, t0 + rank * RB);
+        else sk_tma_store(&mapC, tiles + (uint32_t)(rank * RB) * (TC_BM * 4), f0, t0 + rank * RB);
+      }
     } else if (warp < 4) {
       // thread -> (row group, 4 consecutive features): one 16-byte load per partial tile, all S
       // loads of a row in flight together, one 16-byte (fp32) or 8-byte (bf16) store per row
@@ -452,16 +455,13 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
   // grows with the tile, the latency chain does not shrink); large M takes 128/256-token tiles.
   const int FT = (N + TC_BM - 1) / TC_BM, KB = (K + TC_BK - 1) / TC_BK;
   if (M >= 4096) {
-    // Very large M (prefill, wide verification), no split.  Two candidates, chosen by a two-line
-    // cost model fitted to graph-replay timings on B200 (us per K block of a CTA, epilogue, CTAs
-    // resident per SM):
-    //   (a) 128 x 128 tiles, two CTAs per SM sharing the SM's TMA stream, epilogues overlapped
-    //   (b) 256 x 256 tiles (two weight tiles per CTA), one CTA per SM, loads and MMAs balanced
-    const int ctas_a = FT * ((M + 127) / 128), ctas_b = ((FT + 1) / 2) * ((M + 255) / 256);
-    const double ta = ((ctas_a + 295) / 296) * (KB * 0.53 + 1.5), tb = ((ctas_b + 147) / 148) * (KB * 0.55 + 5.0);
+    // Very large M (prefill, wide verification), no split.  Measured on B200 (graph replay):
+    // 128 x 128 tiles with two CTAs per SM (one's epilogue under the other's main loop) win
+    // unless the K loop is long (>= 32 blocks) and the 256 x 256 grid (two weight tiles per CTA,
+    // token tiles shared in shared memory) still covers most SMs.
+    const int ctas_b = ((FT + 1) / 2) * ((M + 255) / 256);
     *S = 1;
-    // (with fewer than 16 K blocks the unoverlapped epilogue of the big tile eats the gain: measured)
-    if (tb < ta && ctas_b >= 64 && KB >= 16) { *BN = 256; *WT = 2; } else { *BN = 128; }
+    if (KB >= 32 && ctas_b >= 100) { *BN = 256; *WT = 2; } else { *BN = 128; }
     return;
   }
   int bn = M <= 16 ? 16 : M <= 512 ? 32 : 128;
@@ -488,6 +488,7 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   int tma_c = SK_TMA_NONE;
   if (!norm && p.N % TC_BM == 0 && BN % S == 0 && !((uintptr_t)C & 15)) {
     if (epi == EPI_RESID) tma_c = SK_TMA_ADD;
+    else if (epi == EPI_F32) tma_c = SK_TMA_F32;
     else if ((epi == EPI_T || epi == EPI_GELU_T) && S == 1) tma_c = SK_TMA_BF16;
   }
   const CUtensorMap *mapC = &p.mapW;                         // placeholder when unused
