@@ -18,6 +18,10 @@
 //   mode FLASH_WARP: the same passes on short rows with many (series, head) pairs: each warp
 //              takes one pair on its own (cached keys, then the keys of the pass).
 //              grid = (ceil(B * heads / 4), 1, 1).
+//   NB = 1, 2 (the last two modes, caches of at most 32 NB rows): a warp's cached keys and the
+//              keys of the pass share one stage of 32 NB rows and are processed as NB chunks; the
+//              CTA then asks for 8 NB KB per warp (head size 64) instead of a ring of 24 KB, so
+//              that more of these latency-bound warps fit on an SM.  NB = 0: the ring.
 // S = Q K^T uses the rotated, scaled fp32 queries split into a bf16 high and low part (two MMAs),
 // so the scores keep fp32-like accuracy; P is rounded to bf16 for P V.  Scores are kept in
 // base-2 units (the queries carry log2(e) / sqrt(DH)).
@@ -37,7 +41,8 @@ template <int DH> struct FlashGeom {
   static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
   static constexpr int WARP_BYTES = STAGES * STAGE_BYTES;       // also holds (o, m, l) for the merge
   static constexpr int SMEM_BYTES = 4 * WARP_BYTES;
-  static_assert(WARP_BYTES >= 16 * DH * 4 + 2 * 16 * 4, "merge buffers must fit in the ring");
+  static_assert(STAGE_BYTES >= 16 * DH * 4 + 2 * 16 * 4, "merge buffers must fit in one stage");
+  static constexpr int single_bytes(int nb) { return 4 * nb * STAGE_BYTES; }   // CTA, single stage of 32 nb rows
 };
 
 // 16-byte chunk c of row r sits at chunk (c ^ f(r)) of that row: the eight rows that one
@@ -60,12 +65,14 @@ __device__ __forceinline__ void flash_cp16(uint32_t dst, const void *src) {
 __device__ __forceinline__ void flash_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void flash_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <int DH>
-__global__ void __launch_bounds__(128)
-attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
-                  const float2 *__restrict__ rope, PassGeom g, int n_heads, int n_pairs, int mode,
-                  bf16 *__restrict__ out) {
+template <int DH, int NB>
+__device__ __forceinline__ void
+attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
+                const float2 *__restrict__ rope, const PassGeom &g, int n_heads, int n_pairs, int mode,
+                bf16 *__restrict__ out) {
+  constexpr bool single = NB > 0;
   using G = FlashGeom<DH>;
+  constexpr int S_TILE = (NB > 0 ? NB : 1) * G::TILE_BYTES;     // key (or value) rows of the single stage
   constexpr int HALF = DH / 2, KS = DH / 16, CPR = DH / 8;     // k-steps of Q K^T, 16-byte chunks per row
   extern __shared__ __align__(128) unsigned char flash_smem[];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -78,7 +85,8 @@ attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__
     b = pair / n_heads;
     h = pair % n_heads;
   }
-  unsigned char *ring = flash_smem + (size_t)w * G::WARP_BYTES;
+  const int warp_bytes = single ? 2 * S_TILE : G::WARP_BYTES;   // shared memory of one warp
+  unsigned char *ring = flash_smem + (size_t)w * warp_bytes;
   const uint32_t ring32 = (uint32_t)__cvta_generic_to_shared(ring);
   pdl_sync();
   const int p0 = pos0_of(g, b);
@@ -103,7 +111,8 @@ attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__
     own_pass_keys = w == 3;
   }
   const int nq = min(16, g.q_len - jq);
-  const int nch = (t_end - t_beg + G::CHUNK - 1) / G::CHUNK;
+  const int n_c = t_end - t_beg;                               // cached keys of this warp
+  const int nch = single ? 0 : (n_c + G::CHUNK - 1) / G::CHUNK;   // chunks that go through the ring
 
   auto issue = [&](int c) {
     if (c < nch) {
@@ -120,8 +129,18 @@ attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__
     }
     flash_commit();
   };
+  if (single) {
+    for (int idx = lane; idx < n_c * CPR; idx += 32) {
+      const int r = idx / CPR, ch = idx % CPR;
+      const uint32_t off = (uint32_t)(r * G::ROW_BYTES + flash_swz<DH>(r, ch) * 16);
+      flash_cp16(ring32 + off, Kb + (size_t)(t_beg + r) * DH + ch * 8);
+      flash_cp16(ring32 + S_TILE + off, Vb + (size_t)(t_beg + r) * DH + ch * 8);
+    }
+    flash_commit();
+  } else {
 #pragma unroll
-  for (int c = 0; c < G::STAGES - 1; ++c) issue(c);
+    for (int c = 0; c < G::STAGES - 1; ++c) issue(c);
+  }
 
   // rotated, scaled queries as A fragments (rows gr and gr + 8), high and low bf16 parts
   uint32_t qhi[KS][4], qlo[KS][4];
@@ -224,44 +243,61 @@ attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__
     }
   };
 
-  if (own_pass_keys) {
-    // keys and values of this pass (at most 16 tokens) first, while the copies of the first
-    // cached chunks are in flight: rotate the keys, round both to bf16, put them into the last
-    // stage, which the ring does not use before its first refill (value rows past the last token
-    // are zeroed: their probabilities are 0, but 0 x NaN would not be) and append them to the
-    // cache.  One lane handles the element pairs (c, c + 1) and (c + HALF, c + HALF + 1) of a token.
-    unsigned char *st = ring + (G::STAGES - 1) * G::STAGE_BYTES;
-    uint32_t *ks = reinterpret_cast<uint32_t *>(st), *vs = reinterpret_cast<uint32_t *>(st + G::TILE_BYTES);
+  // Keys and values of this pass (at most 16 tokens) first, while the copies of the first cached
+  // chunks are in flight: rotate the keys, round both to bf16, append them to the cache and put
+  // them into the ring's last stage, which is not used before its first refill -- or, with a
+  // single stage, behind the cached rows.  Value rows past the last key of a stage are zeroed:
+  // their probabilities are 0, but 0 x NaN would not be.  One lane handles the element pairs
+  // (c, c + 1) and (c + HALF, c + HALF + 1) of a token.
+  {
+    unsigned char *st = ring + (single ? 0 : (G::STAGES - 1) * G::STAGE_BYTES);
+    uint32_t *ks = reinterpret_cast<uint32_t *>(st), *vs = reinterpret_cast<uint32_t *>(st + S_TILE);
+    const int in_base = single ? n_c : 0;                      // stage row of the pass's first key
+    int filled = single ? n_c : G::CHUNK;                      // stage rows that hold (or will hold) keys
+    if (own_pass_keys) {
 #pragma unroll 2
-    for (int i = lane; i < g.q_len * (HALF / 2); i += 32) {
-      const int j = i / (HALF / 2), c = (i % (HALF / 2)) * 2;
-      const float *src = qkv + (row0 + j) * 3 * d + h * DH;
-      const int tg = p0 + j;
-      const float4 cs = *reinterpret_cast<const float4 *>(rope + (size_t)tg * HALF + c);   // cos0 sin0 cos1 sin1
-      const float2 ka = *reinterpret_cast<const float2 *>(src + d + c);
-      const float2 kb = *reinterpret_cast<const float2 *>(src + d + c + HALF);
-      const float2 va = *reinterpret_cast<const float2 *>(src + 2 * d + c);
-      const float2 vb = *reinterpret_cast<const float2 *>(src + 2 * d + c + HALF);
-      const uint32_t k1 = pack_bf16x2(ka.x * cs.x - kb.x * cs.y, ka.y * cs.z - kb.y * cs.w);
-      const uint32_t k2 = pack_bf16x2(kb.x * cs.x + ka.x * cs.y, kb.y * cs.z + ka.y * cs.w);
-      const uint32_t v1 = pack_bf16x2(va.x, va.y), v2 = pack_bf16x2(vb.x, vb.y);
-      const int w1 = c / 2, w2 = (c + HALF) / 2;               // 32-bit words of the row
-      const int a1 = j * (DH / 2) + flash_swz<DH>(j, w1 >> 2) * 4 + (w1 & 3);
-      const int a2 = j * (DH / 2) + flash_swz<DH>(j, w2 >> 2) * 4 + (w2 & 3);
-      ks[a1] = k1; ks[a2] = k2;
-      vs[a1] = v1; vs[a2] = v2;
-      uint32_t *kg = reinterpret_cast<uint32_t *>(Kb + (size_t)tg * DH);
-      uint32_t *vg = reinterpret_cast<uint32_t *>(Vb + (size_t)tg * DH);
-      kg[w1] = k1; kg[w2] = k2;
-      vg[w1] = v1; vg[w2] = v2;
+      for (int i = lane; i < g.q_len * (HALF / 2); i += 32) {
+        const int j = i / (HALF / 2), c = (i % (HALF / 2)) * 2, jr = in_base + j;
+        const float *src = qkv + (row0 + j) * 3 * d + h * DH;
+        const int tg = p0 + j;
+        const float4 cs = *reinterpret_cast<const float4 *>(rope + (size_t)tg * HALF + c);   // cos0 sin0 cos1 sin1
+        const float2 ka = *reinterpret_cast<const float2 *>(src + d + c);
+        const float2 kb = *reinterpret_cast<const float2 *>(src + d + c + HALF);
+        const float2 va = *reinterpret_cast<const float2 *>(src + 2 * d + c);
+        const float2 vb = *reinterpret_cast<const float2 *>(src + 2 * d + c + HALF);
+        const uint32_t k1 = pack_bf16x2(ka.x * cs.x - kb.x * cs.y, ka.y * cs.z - kb.y * cs.w);
+        const uint32_t k2 = pack_bf16x2(kb.x * cs.x + ka.x * cs.y, kb.y * cs.z + ka.y * cs.w);
+        const uint32_t v1 = pack_bf16x2(va.x, va.y), v2 = pack_bf16x2(vb.x, vb.y);
+        const int w1 = c / 2, w2 = (c + HALF) / 2;               // 32-bit words of the row
+        const int a1 = jr * (DH / 2) + flash_swz<DH>(jr, w1 >> 2) * 4 + (w1 & 3);
+        const int a2 = jr * (DH / 2) + flash_swz<DH>(jr, w2 >> 2) * 4 + (w2 & 3);
+        ks[a1] = k1; ks[a2] = k2;
+        vs[a1] = v1; vs[a2] = v2;
+        uint32_t *kg = reinterpret_cast<uint32_t *>(Kb + (size_t)tg * DH);
+        uint32_t *vg = reinterpret_cast<uint32_t *>(Vb + (size_t)tg * DH);
+        kg[w1] = k1; kg[w2] = k2;
+        vg[w1] = v1; vg[w2] = v2;
+      }
+      filled = in_base + g.q_len;
     }
-    for (int i = g.q_len * (DH / 2) + lane; i < G::CHUNK * (DH / 2); i += 32) vs[i] = 0u;
-    __syncwarp();
-    const uint32_t st32 = ring32 + (uint32_t)((G::STAGES - 1) * G::STAGE_BYTES);
-    chunk(st32, st32 + G::TILE_BYTES, p0, p0 + g.q_len);
-    // the first refill of this stage follows the warp barrier at the top of the loop below
+    // (zero up to the end of the last 32-row block that holds a key)
+    for (int i = filled * (DH / 2) + lane; i < ((filled + G::CHUNK - 1) & ~(G::CHUNK - 1)) * (DH / 2); i += 32) vs[i] = 0u;
+    if (single) {
+      flash_wait<0>();
+      __syncwarp();
+      const int t_lim = own_pass_keys ? p0 + g.q_len : t_end;
+#pragma unroll
+      for (int blk = 0; blk < NB; ++blk)
+        if (filled > blk * G::CHUNK)
+          chunk(ring32 + (uint32_t)(blk * G::TILE_BYTES), ring32 + (uint32_t)(S_TILE + blk * G::TILE_BYTES),
+                t_beg + blk * G::CHUNK, t_lim);
+    } else if (own_pass_keys) {
+      __syncwarp();
+      const uint32_t st32 = ring32 + (uint32_t)((G::STAGES - 1) * G::STAGE_BYTES);
+      chunk(st32, st32 + G::TILE_BYTES, p0, p0 + g.q_len);
+      // the first refill of this stage follows the warp barrier at the top of the loop below
+    }
   }
-
 
   for (int c = 0; c < nch; ++c) {
     flash_wait<G::STAGES - 2>();
@@ -307,11 +343,11 @@ attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__
     float m = -INFINITY;
 #pragma unroll
     for (int ww = 0; ww < 4; ++ww)
-      m = fmaxf(m, reinterpret_cast<const float *>(flash_smem + (size_t)ww * G::WARP_BYTES)[16 * DH + i]);
+      m = fmaxf(m, reinterpret_cast<const float *>(flash_smem + (size_t)ww * warp_bytes)[16 * DH + i]);
     float l = 0.f, ox = 0.f, oy = 0.f;
 #pragma unroll
     for (int ww = 0; ww < 4; ++ww) {
-      const float *wb = reinterpret_cast<const float *>(flash_smem + (size_t)ww * G::WARP_BYTES);
+      const float *wb = reinterpret_cast<const float *>(flash_smem + (size_t)ww * warp_bytes);
       const float mw = wb[16 * DH + i];
       if (mw == -INFINITY) continue;                           // that range held no visible key
       const float sc = exp2f(mw - m);
@@ -323,6 +359,23 @@ attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__
     const float inv = 1.f / l;
     *reinterpret_cast<uint32_t *>(out + (row0 + jq + i) * d + h * DH + c) = pack_bf16x2(ox * inv, oy * inv);
   }
+}
+
+// The ring variant (three stages per warp) and the single-stage variant; the latter is compiled
+// for four CTAs per SM where the head size allows it.
+template <int DH>
+__global__ void __launch_bounds__(128)
+attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
+                  const float2 *__restrict__ rope, PassGeom g, int n_heads, int n_pairs, int mode,
+                  bf16 *__restrict__ out) {
+  attn_flash_body<DH, 0>(qkv, Kc, Vc, rope, g, n_heads, n_pairs, mode, out);
+}
+template <int DH, int NB>
+__global__ void __launch_bounds__(128, DH <= 64 ? (NB == 1 ? 4 : 3) : 1)
+attn_flash_single_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
+                         const float2 *__restrict__ rope, PassGeom g, int n_heads, int n_pairs, int mode,
+                         bf16 *__restrict__ out) {
+  attn_flash_body<DH, NB>(qkv, Kc, Vc, rope, g, n_heads, n_pairs, mode, out);
 }
 
 }  // namespace tsfm

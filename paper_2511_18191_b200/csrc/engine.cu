@@ -309,6 +309,8 @@ int attn_set_attr(size_t bytes) {
 constexpr int kFlashWarpMaxCap = 64, kFlashWarpMinPairs = 8 * 148;
 template <int DH> int flash_set_attr() {
   CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::SMEM_BYTES));
+  CU_TRY(cudaFuncSetAttribute(attn_flash_single_kernel<DH, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::single_bytes(1)));
+  CU_TRY(cudaFuncSetAttribute(attn_flash_single_kernel<DH, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::single_bytes(2)));
   return TSFM_OK;
 }
 template <typename T>
@@ -361,6 +363,12 @@ void prefer_max_smem_all() {
   prefer_max_smem(attn_flash_kernel<32>);
   prefer_max_smem(attn_flash_kernel<64>);
   prefer_max_smem(attn_flash_kernel<128>);
+  prefer_max_smem(attn_flash_single_kernel<32, 1>);
+  prefer_max_smem(attn_flash_single_kernel<32, 2>);
+  prefer_max_smem(attn_flash_single_kernel<64, 1>);
+  prefer_max_smem(attn_flash_single_kernel<64, 2>);
+  prefer_max_smem(attn_flash_single_kernel<128, 1>);
+  prefer_max_smem(attn_flash_single_kernel<128, 2>);
   cudaGetLastError();
 }
 
@@ -452,8 +460,17 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
                          : (h->cap <= kFlashWarpMaxCap && pairs >= kFlashWarpMinPairs) ? FLASH_WARP : FLASH_SPLIT;
     const dim3 grid = mode == FLASH_WARP ? dim3((pairs + 3) / 4)
                                          : dim3(m.arch.n_heads, B, pre ? (g.q_len + 4 * ATTN_QT - 1) / (4 * ATTN_QT) : 1);
-    launch_ex(h->ls, h->pdl, attn_flash_kernel<DH>, grid, dim3(128), (size_t)FlashGeom<DH>::SMEM_BYTES, h->qkv,
-              (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
+    // short caches: one stage of 32 or 64 rows per warp instead of the ring, more warps per SM
+    const int nb = pre ? 0 : h->cap <= FlashGeom<DH>::CHUNK ? 1 : h->cap <= 2 * FlashGeom<DH>::CHUNK ? 2 : 0;
+    if (nb == 1)
+      launch_ex(h->ls, h->pdl, attn_flash_single_kernel<DH, 1>, grid, dim3(128), (size_t)FlashGeom<DH>::single_bytes(1),
+                h->qkv, (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
+    else if (nb == 2)
+      launch_ex(h->ls, h->pdl, attn_flash_single_kernel<DH, 2>, grid, dim3(128), (size_t)FlashGeom<DH>::single_bytes(2),
+                h->qkv, (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
+    else
+      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH>, grid, dim3(128), (size_t)FlashGeom<DH>::SMEM_BYTES, h->qkv,
+                (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
   } else {
     const int QT = g.q_len <= ATTN_QT ? g.q_len : ATTN_QT;
     const int skv = attn_key_split(h->cap);
