@@ -261,7 +261,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const float sq = warp_sum(v[j]);
-            if (lane == 0 && t0 + cc + j < M) nm.ssq_out[(size_t)(t0 + cc + j) * (N >> 5) + (f >> 5)] = sq;
+            if (lane == 0 && f < N && t0 + cc + j < M) nm.ssq_out[(size_t)(t0 + cc + j) * (N >> 5) + (f >> 5)] = sq;
           }
         }
       }
@@ -354,10 +354,14 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
               pk.x = *reinterpret_cast<const uint32_t *>(&lo);
               pk.y = *reinterpret_cast<const uint32_t *>(&hi);
               *reinterpret_cast<uint2 *>(nm.a_out + o) = pk;
-              float sq = old.x * old.x + old.y * old.y + old.z * old.z + old.w * old.w;   // 8 lanes = one 32-feature slice
-              sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-              sq += __shfl_xor_sync(0xffffffffu, sq, 2);
-              sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+              // 8 lanes = one 32-feature slice.  N is a multiple of 32 here, so a slice is inside N
+              // or outside it as a whole: only its own 8 lanes are named in the shuffles (the lanes
+              // of a feature tile's slices beyond N never get here).
+              const unsigned grp = 0xffu << (threadIdx.x & 24);
+              float sq = old.x * old.x + old.y * old.y + old.z * old.z + old.w * old.w;
+              sq += __shfl_xor_sync(grp, sq, 1);
+              sq += __shfl_xor_sync(grp, sq, 2);
+              sq += __shfl_xor_sync(grp, sq, 4);
               if ((threadIdx.x & 7) == 0) nm.ssq_out[(size_t)t * (N >> 5) + (f >> 5)] = sq;
             }
           } else {

@@ -19,6 +19,12 @@ def pytest_collection_modifyitems(config, items):
     except Exception:
         has_gpu = False
     if has_gpu:
+        # a GPU test that stalls (a device-side wait that keeps expiring) must not hold the device
+        # for the rest of the session: bound every one of them where pytest-timeout is installed
+        if config.pluginmanager.hasplugin("timeout"):
+            for item in items:
+                if "gpu" in item.keywords and item.get_closest_marker("timeout") is None:
+                    item.add_marker(pytest.mark.timeout(900))
         return
     skip = pytest.mark.skip(reason="no CUDA device")
     for item in items:

@@ -156,6 +156,14 @@ def test_long_rows_small_models_bf16(target, draft):
     run_and_compare(wl, 3, 2.0, 3, [0, 1, 2], exec_mode=1)
 
 
+def test_many_series_short_rows_one_warp_per_series_and_head_bf16():
+    """Enough (series, head) pairs on short rows for the attention mode that gives each warp a pair
+    of its own, with a pair count that is not a multiple of the four warps of a CTA (199 x 6)."""
+    wl = workload("C1", batch=199, horizon=96 * 3, target=Arch(2, 192, 6, 384), draft=Arch(1, 192, 6, 384),
+                  draft_mode="layer_skip")
+    run_and_compare(wl, 3, 1.0, 9, [0, 100, 198])
+
+
 @pytest.mark.parametrize("name,ids", [("C0", [0]), ("C1", [0, 7, 31]), ("C2", [3, 200])])
 def test_draft_only_forecast_matches_oracle(name, ids):
     """Third arm of the matched three-way protocol: the draft model decoding on its own (Eq. 1)."""
