@@ -336,6 +336,9 @@ template <typename T> void prefer_max_smem_typed() {
   prefer_max_smem(embed_kernel<T>);
   prefer_max_smem(rmsnorm_kernel<T>);
   prefer_max_smem(head_kernel<T>);
+  prefer_max_smem(embed_rows_kernel<T>);
+  prefer_max_smem(head_rows_kernel<T>);
+  cudaFuncSetAttribute(head_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
   prefer_max_smem(gemm_simt_kernel<T, EPI_F32>);
   prefer_max_smem(gemm_simt_kernel<T, EPI_T>);
   prefer_max_smem(gemm_simt_kernel<T, EPI_GELU_T>);
@@ -487,6 +490,9 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
 }
 
 enum { HEAD_NONE = 0, HEAD_LAST_TO_HIST = 1, HEAD_ALL_TO_VOUT = 2 };
+// Passes of at least this many rows take the embedding and head kernels that share each weight
+// load between 8 rows; below it there are too few rows to fill the SMs that way.
+constexpr int kManyRows = 1024;
 
 // Draft step i of a round (k_pos = i - 1): lets the head kernel turn its mean into a sampled
 // proposal when the call asks for one (Sec. 3.3); target and prefill passes carry none.
@@ -508,9 +514,13 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   const int L = m.arch.n_layers;
   {
     KTimer kt(h, KC_EMBED, (double)M * P * 4 + (double)d * P * sizeof(T) + (double)M * d * 4, 2.0 * M * P * d);
-    launch_ex(s, h->pdl, embed_kernel<T>, dim3(M, (d + 127) / 128), dim3(128), P * sizeof(float), h->hist, g, P, d,
-              (const T *)m.W_emb, h->x, stamp, fold ? m.layers[0].g1 : (const float *)nullptr,
-              fold ? (T *)h->a : (T *)nullptr, fold ? h->ssq : (float *)nullptr);
+    if (!fold && M >= kManyRows)
+      launch_ex(s, h->pdl, embed_rows_kernel<T>, dim3((M + 7) / 8, (d + 127) / 128), dim3(128), 8 * P * sizeof(float),
+                h->hist, g, M, P, d, (const T *)m.W_emb, h->x, stamp);
+    else
+      launch_ex(s, h->pdl, embed_kernel<T>, dim3(M, (d + 127) / 128), dim3(128), P * sizeof(float), h->hist, g, P, d,
+                (const T *)m.W_emb, h->x, stamp, fold ? m.layers[0].g1 : (const float *)nullptr,
+                fold ? (T *)h->a : (T *)nullptr, fold ? h->ssq : (float *)nullptr);
   }
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
   SkNorm consume{};                 // scale the result rows by rstd of the input rows
@@ -522,7 +532,7 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     LayerDev &ly = m.layers[l];
     if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3(M), dim3(128), 0, h->x, ly.g1, d, eps, (T *)h->a, nullptr, 0);
+      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g1, M, d, eps, (T *)h->a);
     }
     gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
@@ -536,7 +546,7 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, fold ? &produce : nullptr);
     if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3(M), dim3(128), 0, h->x, ly.g2, d, eps, (T *)h->a, nullptr, 0);
+      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g2, M, d, eps, (T *)h->a);
     }
     gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, fold ? &consume : nullptr);
     produce.gain = l + 1 < L ? m.layers[l + 1].g1 : nullptr;
@@ -550,6 +560,9 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     launch_ex(s, h->pdl, head_kernel<T>, dim3(B, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
               (const T *)m.W_head, d, P, eps, g, 1, h->hist, (float *)nullptr,
               ds.k_pos >= 0 ? (const DevState *)h->st : (const DevState *)nullptr, h->muq, ds.k_pos, ds.K);
+  } else if (head_mode == HEAD_ALL_TO_VOUT && M >= kManyRows && (size_t)8 * d * sizeof(float) <= 200 * 1024) {
+    launch_ex(s, h->pdl, head_rows_kernel<T>, dim3((M + 7) / 8, (P + 31) / 32), dim3(256), (size_t)8 * d * sizeof(float),
+              h->x, m.g_f, (const T *)m.W_head, M, d, P, eps, vout);
   } else if (head_mode == HEAD_ALL_TO_VOUT) {
     launch_ex(s, h->pdl, head_kernel<T>, dim3(M, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
               (const T *)m.W_head, d, P, eps, g, 0, (float *)nullptr, vout, (const DevState *)nullptr, (float *)nullptr, 0, 0);

@@ -127,37 +127,104 @@ embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *
   }
 }
 
-// ----------------------------------------------------------------------------------
-// RMSNorm: a[row, :] = g * x / sqrt(mean(x^2) + eps), rounded to T.  grid = M, block 128.
-// Optionally clears zero_cols floats of row `row` of a scratch matrix (the accumulator of
-// a following split-K contraction).
-// ----------------------------------------------------------------------------------
+// The same embedding for passes of many rows: 8 rows per CTA share every weight load.
+// grid = (ceil(M / 8), ceil(d / 128)), block = 128, dynamic shared memory 8 * P floats.
 template <typename T>
 __global__ void __launch_bounds__(128)
-rmsnorm_kernel(const float *__restrict__ x, const float *__restrict__ gain, int d, float eps,
-               T *__restrict__ a, float *__restrict__ zero, int zero_cols) {
-  __shared__ float red[32];
+embed_rows_kernel(const float *__restrict__ hist, PassGeom g, int M, int P, int d, const T *__restrict__ W,
+                  float *__restrict__ x, unsigned long long *__restrict__ stamp) {
+  constexpr int R = 8;
+  extern __shared__ float zs[];                               // [R][P]
   pdl_sync();
-  const size_t row = blockIdx.x;
+  const int row0 = blockIdx.x * R;
+  if (stamp && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *stamp = globaltimer_ns();
+  for (int i = threadIdx.x; i < R * P; i += blockDim.x) {
+    const int row = row0 + i / P;
+    float v = 0.f;
+    if (row < M) {
+      const int b = row / g.q_len, j = row % g.q_len;
+      v = hist[((size_t)b * g.cap + pos0_of(g, b) + j) * P + i % P];
+    }
+    zs[i] = v;
+  }
+  __syncthreads();
+  const int f = blockIdx.y * 128 + threadIdx.x;
+  if (f >= d) return;
+  const T *wr = W + (size_t)f * P;
+  constexpr int V = Vec16<T>::N;
+  float acc[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) acc[r] = 0.f;
+#pragma unroll 2
+  for (int i = 0; i < P; i += V) {
+    float w[V];
+    Vec16<T>::load(wr + i, w);
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int c = 0; c < V; ++c) acc[r] = fmaf(w[c], zs[r * P + i + c], acc[r]);
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+    if (row0 + r < M) x[(size_t)(row0 + r) * d + f] = acc[r];
+}
+
+// ----------------------------------------------------------------------------------
+// RMSNorm: a[row, :] = g * x / sqrt(mean(x^2) + eps), rounded to T.  One warp per row, 8 rows
+// per CTA (grid = ceil(M / 8), block = 256): the row is read once with 16-byte loads and kept in
+// registers (rows of up to 2048 features; longer rows are read a second time), reduced with
+// shuffles only, and written with 16-byte (fp32) or 8-byte (bf16) stores.  d is a multiple of 4.
+// ----------------------------------------------------------------------------------
+__device__ __forceinline__ void store4(float *o, float a, float b, float c, float d4) {
+  *reinterpret_cast<float4 *>(o) = make_float4(a, b, c, d4);
+}
+__device__ __forceinline__ void store4(bf16 *o, float a, float b, float c, float d4) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d4);
+  uint2 pk;
+  pk.x = *reinterpret_cast<const uint32_t *>(&lo);
+  pk.y = *reinterpret_cast<const uint32_t *>(&hi);
+  *reinterpret_cast<uint2 *>(o) = pk;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(const float *__restrict__ x, const float *__restrict__ gain, int M, int d, float eps,
+               T *__restrict__ a) {
+  constexpr int CACHE = 16;                                   // float4 per lane kept in registers
+  pdl_sync();
+  const int lane = threadIdx.x & 31;
+  const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= (size_t)M) return;
   const float4 *xr = reinterpret_cast<const float4 *>(x + row * d);
   const float4 *gr = reinterpret_cast<const float4 *>(gain);
+  const int nv = d / 4;
+  float4 v[CACHE];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
-    const float4 v = xr[i];
-    ss = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, ss))));
+#pragma unroll
+  for (int k = 0; k < CACHE; ++k) {
+    const int i = lane + 32 * k;
+    if (i < nv) {
+      v[k] = xr[i];
+      ss = fmaf(v[k].x, v[k].x, fmaf(v[k].y, v[k].y, fmaf(v[k].z, v[k].z, fmaf(v[k].w, v[k].w, ss))));
+    }
   }
-  if (zero) {
-    float4 *zr = reinterpret_cast<float4 *>(zero + row * zero_cols);
-    for (int i = threadIdx.x; i < zero_cols / 4; i += blockDim.x) zr[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int i = lane + 32 * CACHE; i < nv; i += 32) {
+    const float4 u = xr[i];
+    ss = fmaf(u.x, u.x, fmaf(u.y, u.y, fmaf(u.z, u.z, fmaf(u.w, u.w, ss))));
   }
-  const float rstd = rsqrtf(block_sum(ss, red) / d + eps);
-  for (int i = threadIdx.x; i < d / 4; i += blockDim.x) {
-    const float4 v = xr[i], gg = gr[i];
-    T *o = a + row * d + 4 * i;
-    o[0] = from_f32<T>(gg.x * v.x * rstd);
-    o[1] = from_f32<T>(gg.y * v.y * rstd);
-    o[2] = from_f32<T>(gg.z * v.z * rstd);
-    o[3] = from_f32<T>(gg.w * v.w * rstd);
+  const float rstd = rsqrtf(warp_sum(ss) / d + eps);
+  T *ar = a + row * d;
+#pragma unroll
+  for (int k = 0; k < CACHE; ++k) {
+    const int i = lane + 32 * k;
+    if (i < nv) {
+      const float4 gg = gr[i];
+      store4(ar + 4 * i, gg.x * v[k].x * rstd, gg.y * v[k].y * rstd, gg.z * v[k].z * rstd, gg.w * v[k].w * rstd);
+    }
+  }
+  for (int i = lane + 32 * CACHE; i < nv; i += 32) {
+    const float4 u = xr[i], gg = gr[i];
+    store4(ar + 4 * i, gg.x * u.x * rstd, gg.y * u.y * rstd, gg.z * u.z * rstd, gg.w * u.w * rstd);
   }
 }
 
@@ -650,6 +717,61 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
       acc += st->sigma_q * head_normal(st, b, k_pos, p);
     }
     dst[p] = acc;
+  }
+}
+
+// The head for every token of a pass of many rows (verification: vout[b, j, :]): 8 rows per CTA
+// (one warp normalises one row into shared memory), then each warp produces 4 of the CTA's 32
+// outputs for all 8 rows, so that a weight vector is loaded once per 8 rows.
+// grid = (ceil(M / 8), ceil(P / 32)), block = 256, dynamic shared memory 8 * d floats.
+template <typename T>
+__global__ void __launch_bounds__(256)
+head_rows_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T *__restrict__ Wh, int M,
+                 int d, int P, float eps, float *__restrict__ vout) {
+  constexpr int R = 8;
+  extern __shared__ __align__(16) float xs[];                  // [R][d] normalised rows
+  pdl_sync();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int row0 = blockIdx.x * R;
+  {
+    const int row = row0 + w;
+    float *xw = xs + (size_t)w * d;
+    float ss = 0.f;
+    if (row < M) {
+      const float *xr = x + (size_t)row * d;
+      for (int i = lane; i < d; i += 32) {
+        const float v = xr[i];
+        xw[i] = v;
+        ss = fmaf(v, v, ss);
+      }
+    } else {
+      for (int i = lane; i < d; i += 32) xw[i] = 0.f;
+    }
+    const float rstd = rsqrtf(warp_sum(ss) / d + eps);
+    for (int i = lane; i < d; i += 32) xw[i] = gain[i] * xw[i] * rstd;   // each lane rewrites what it wrote
+  }
+  __syncthreads();
+  constexpr int V = Vec16<T>::N;
+  for (int q = 0; q < 4; ++q) {
+    const int p = blockIdx.y * 32 + q * 8 + w;
+    if (p >= P) break;
+    const T *wr = Wh + (size_t)p * d;
+    float acc[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) acc[r] = 0.f;
+    for (int i = lane * V; i < d; i += 32 * V) {
+      float wv[V];
+      Vec16<T>::load(wr + i, wv);
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int c = 0; c < V; ++c) acc[r] = fmaf(wv[c], xs[(size_t)r * d + i + c], acc[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const float o = warp_sum(acc[r]);
+      if (lane == 0 && row0 + r < M) vout[(size_t)(row0 + r) * P + p] = o;
+    }
   }
 }
 
