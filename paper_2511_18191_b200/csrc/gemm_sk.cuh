@@ -136,6 +136,12 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
   // (Measured: spreading the K steps of a stage over several accumulators does not help a narrow
   // tile -- one MMA of 128 x BN x 16 takes ~90 ns whatever BN is -- so one accumulator per tile.)
 
+  if (warp == 4 && lane == 0) {
+    // descriptor fetches off the critical path of the first loads (and of the output copy)
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&mapA) : "memory");
+    if (tma_c) asm volatile("prefetch.tensormap [%0];" ::"l"(&mapC) : "memory");
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(full0 + 8 * s, 1);
