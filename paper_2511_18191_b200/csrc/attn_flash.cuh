@@ -33,9 +33,9 @@ namespace tsfm {
 
 enum { FLASH_WARP = 0, FLASH_TILES = 1, FLASH_SPLIT = 4 };
 
-template <int DH> struct FlashGeom {
+template <int DH, int ST = 3> struct FlashGeom {
   static constexpr int CHUNK = 32;                              // keys per stage
-  static constexpr int STAGES = 3;
+  static constexpr int STAGES = ST;                             // ring depth (3: prefill tiles; 2: one-tile passes)
   static constexpr int ROW_BYTES = DH * 2;
   static constexpr int TILE_BYTES = CHUNK * ROW_BYTES;          // keys (or values) of one stage
   static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
@@ -65,13 +65,13 @@ __device__ __forceinline__ void flash_cp16(uint32_t dst, const void *src) {
 __device__ __forceinline__ void flash_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void flash_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <int DH, int NB>
+template <int DH, int NB, int ST>
 __device__ __forceinline__ void
 attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
                 const float2 *__restrict__ rope, const PassGeom &g, int n_heads, int n_pairs, int mode,
                 bf16 *__restrict__ out) {
   constexpr bool single = NB > 0;
-  using G = FlashGeom<DH>;
+  using G = FlashGeom<DH, ST>;
   constexpr int S_TILE = (NB > 0 ? NB : 1) * G::TILE_BYTES;     // key (or value) rows of the single stage
   constexpr int HALF = DH / 2, KS = DH / 16, CPR = DH / 8;     // k-steps of Q K^T, 16-byte chunks per row
   extern __shared__ __align__(128) unsigned char flash_smem[];
@@ -361,21 +361,21 @@ attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__re
   }
 }
 
-// The ring variant (three stages per warp) and the single-stage variant; the latter is compiled
+// The ring variant (ST stages per warp) and the single-stage variant; the latter is compiled
 // for four CTAs per SM where the head size allows it.
-template <int DH>
+template <int DH, int ST>
 __global__ void __launch_bounds__(128)
 attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
                   const float2 *__restrict__ rope, PassGeom g, int n_heads, int n_pairs, int mode,
                   bf16 *__restrict__ out) {
-  attn_flash_body<DH, 0>(qkv, Kc, Vc, rope, g, n_heads, n_pairs, mode, out);
+  attn_flash_body<DH, 0, ST>(qkv, Kc, Vc, rope, g, n_heads, n_pairs, mode, out);
 }
 template <int DH, int NB>
 __global__ void __launch_bounds__(128, DH <= 64 ? (NB == 1 ? 4 : 3) : 1)
 attn_flash_single_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
                          const float2 *__restrict__ rope, PassGeom g, int n_heads, int n_pairs, int mode,
                          bf16 *__restrict__ out) {
-  attn_flash_body<DH, NB>(qkv, Kc, Vc, rope, g, n_heads, n_pairs, mode, out);
+  attn_flash_body<DH, NB, 3>(qkv, Kc, Vc, rope, g, n_heads, n_pairs, mode, out);
 }
 
 }  // namespace tsfm

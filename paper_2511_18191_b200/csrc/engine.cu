@@ -307,8 +307,13 @@ int attn_set_attr(size_t bytes) {
 // bf16 caches take the running-softmax kernel (attn_flash_kernel), fp32 caches attn_kernel.
 // Short rows with at least this many (series, head) pairs: one warp per pair instead of four.
 constexpr int kFlashWarpMaxCap = 64, kFlashWarpMinPairs = 8 * 148;
+#ifndef FLASH_ST_SHORT
+#define FLASH_ST_SHORT 2
+#endif
 template <int DH> int flash_set_attr() {
-  CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::SMEM_BYTES));
+  CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH, 3>::SMEM_BYTES));
+  CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH, FLASH_ST_SHORT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              FlashGeom<DH, FLASH_ST_SHORT>::SMEM_BYTES));
   CU_TRY(cudaFuncSetAttribute(attn_flash_single_kernel<DH, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::single_bytes(1)));
   CU_TRY(cudaFuncSetAttribute(attn_flash_single_kernel<DH, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::single_bytes(2)));
   return TSFM_OK;
@@ -363,9 +368,12 @@ void prefer_max_smem_all() {
   prefer_max_smem(gemm_sk_kernel<1, true>);
   prefer_max_smem(gemm_sk_kernel<2, false>);
   prefer_max_smem(pass_cluster_kernel);
-  prefer_max_smem(attn_flash_kernel<32>);
-  prefer_max_smem(attn_flash_kernel<64>);
-  prefer_max_smem(attn_flash_kernel<128>);
+  prefer_max_smem(attn_flash_kernel<32, 3>);
+  prefer_max_smem(attn_flash_kernel<32, FLASH_ST_SHORT>);
+  prefer_max_smem(attn_flash_kernel<64, 3>);
+  prefer_max_smem(attn_flash_kernel<64, FLASH_ST_SHORT>);
+  prefer_max_smem(attn_flash_kernel<128, 3>);
+  prefer_max_smem(attn_flash_kernel<128, FLASH_ST_SHORT>);
   prefer_max_smem(attn_flash_single_kernel<32, 1>);
   prefer_max_smem(attn_flash_single_kernel<32, 2>);
   prefer_max_smem(attn_flash_single_kernel<64, 1>);
@@ -471,9 +479,13 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
     else if (nb == 2)
       launch_ex(h->ls, h->pdl, attn_flash_single_kernel<DH, 2>, grid, dim3(128), (size_t)FlashGeom<DH>::single_bytes(2),
                 h->qkv, (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
-    else
-      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH>, grid, dim3(128), (size_t)FlashGeom<DH>::SMEM_BYTES, h->qkv,
+    else if (pre)
+      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH, 3>, grid, dim3(128), (size_t)FlashGeom<DH, 3>::SMEM_BYTES, h->qkv,
                 (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
+    else      // one query tile: each warp has a few chunks only, a two-stage ring lets a third CTA onto the SM
+      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH, FLASH_ST_SHORT>, grid, dim3(128),
+                (size_t)FlashGeom<DH, FLASH_ST_SHORT>::SMEM_BYTES, h->qkv, (bf16 *)Kc, (bf16 *)Vc, m.rope, g,
+                m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
   } else {
     const int QT = g.q_len <= ATTN_QT ? g.q_len : ATTN_QT;
     const int skv = attn_key_split(h->cap);

@@ -156,6 +156,15 @@ def test_long_rows_small_models_bf16(target, draft):
     run_and_compare(wl, 3, 2.0, 3, [0, 1, 2], exec_mode=1)
 
 
+def test_long_rows_fp32_keys_split_over_a_cluster():
+    """fp32 caches of 200+ rows: the keys of a (series, head) are split over a cluster of four CTAs
+    whose partial softmax results are merged through distributed shared memory, in prefill (13
+    query tiles), verification (4 queries) and one-token steps alike."""
+    wl = workload("C0", batch=2, series_recipe="c1", ctx_len=96 * 200, horizon=96 * 4 + 10)
+    for mode in (1, 0):
+        run_and_compare(wl, 3, 2.0, 4, [0, 1], exec_mode=mode)
+
+
 def test_many_series_short_rows_one_warp_per_series_and_head_bf16():
     """Enough (series, head) pairs on short rows for the attention mode that gives each warp a pair
     of its own, with a pair count that is not a multiple of the four warps of a CTA (199 x 6)."""
