@@ -165,6 +165,15 @@ def test_long_rows_fp32_keys_split_over_a_cluster():
         run_and_compare(wl, 3, 2.0, 4, [0, 1], exec_mode=mode)
 
 
+def test_block_size_beyond_one_query_tile_bf16():
+    """K = 20: the verification pass has 21 tokens per series, more than one 16-query tile, so its
+    keys go to the cache through the append kernel and the attention runs in its multi-tile mode at
+    ragged per-series positions, round after round (rows of rejected proposals are overwritten)."""
+    wl = workload("C1", batch=4, horizon=96 * 6)
+    for mode in (1, 0):
+        run_and_compare(wl, 20, 2.0, 17, [0, 1, 2, 3], exec_mode=mode)
+
+
 def test_many_series_short_rows_one_warp_per_series_and_head_bf16():
     """Enough (series, head) pairs on short rows for the attention mode that gives each warp a pair
     of its own, with a pair count that is not a multiple of the four warps of a CTA (199 x 6)."""
