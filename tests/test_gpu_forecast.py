@@ -246,6 +246,24 @@ def test_general_rule_variants_match_oracle(wl_name, name, kw):
         assert d["proposals_accepted"] == 0                     # acceptance collapses without the 1/d
 
 
+def test_sampled_proposals_with_many_series_bf16():
+    """Sampled proposals and fallback noise at 1024 series (C3 shape, small models): the draft head
+    of such passes shares its weight loads between 8 series and adds the proposal noise itself."""
+    import paper_2511_18191_b200 as tsfm
+    wl = workload("C3", draft_eps=1e-2, horizon=96 * 4, target=Arch(2, 256, 4, 512), draft=Arch(2, 256, 4, 512))
+    K, tau, seed, ids = 3, 1.5, 23, [0, 511, 1023]
+    dec, tw, dw = make_decoder(wl, batch=wl.batch)
+    s, ctx = series_on_device(wl, wl.batch)
+    v = tsfm.tsfm_variant(0.8, 0.2, 1, 0)
+    out, st = dec.forecast(ctx, wl.horizon, K, tau, seed, variant=v)
+    check_stats(st, wl.batch, wl.n_patches, K)
+    nacc, ell, logu = dec.last_trace(wl.batch, K)
+    dec.close()
+    tm, dm = parity.oracle_models(wl, tw, dw)
+    var = orc.Variant(sigma_q=0.8, sample_proposals=True, fallback_noise=0.2, tempering=True)
+    parity.compare_forecast(wl, tm, dm, s, wl.horizon, K, tau, seed, out.cpu().numpy(), nacc, ids, variant=var)
+
+
 def test_tiny_tau_recovers_target_only_and_result_is_independent_of_batch_composition():
     wl = workload("C1")
     dec, tw, dw = make_decoder(wl)
