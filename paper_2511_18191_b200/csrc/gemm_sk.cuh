@@ -490,6 +490,19 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
     *S = 1;
     return;
   }
+  if (M > 512) {
+    // The same token counts with a long K loop: K split 2 or 4 ways; of the measured combinations
+    // (96 tokens x 2, 128 x 2, 128 x 4) the one with the most CTAs within one wave.
+    const int cand[3][2] = {{96, 2}, {128, 2}, {128, 4}};
+    int bb = 128, bs = 2, best_ctas = 0;
+    for (const auto &c : cand) {
+      const int ctas = FT * ((M + c[0] - 1) / c[0]) * c[1];
+      if (ctas <= 296 && ctas > best_ctas) { bb = c[0]; bs = c[1]; best_ctas = ctas; }
+    }
+    *BN = bb;
+    *S = bs;
+    return;
+  }
   int bn = M <= 16 ? 16 : M <= 512 ? 32 : 128;
   const int tiles = FT * ((M + bn - 1) / bn);
   int s = 1;
