@@ -1,15 +1,22 @@
 #!/usr/bin/env python
-"""Benchmark of the speculative patch decoder: committed patches/s on workload C1.
+"""Benchmark of the speculative patch decoder: committed patches/s.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C1]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C4]
 
 One "step" is one whole speculative forecast (instance norm, prefill of both models, the
 round loop draft -> verify -> accept -> rollback until T patches are committed, de-normalise)
-over one batch of synthetic series.  `value` = committed patches per second with the inputs
-resident in HBM; `e2e` = the same through the host-buffer entry point (pinned host input and
-output, copies inside the timed region).  With N > 1 (torchrun) every rank decodes its own
-batch on its own GPU (the path shards by series with no exchange step: weak scaling, no
-collective); times are CUDA-event times, max over ranks.
+over one batch of synthetic series.  The headline workload is C4, the largest single-GPU
+configuration (64 series, 256 context tokens, 64 patches to commit, a 472 M-parameter target):
+`value` = committed patches per second with the inputs resident in HBM; `e2e` = the same
+through the host-buffer entry point (pinned host input and output, copies inside the timed
+region).  With N > 1 (torchrun) every rank decodes its own batch on its own GPU (the path
+shards by series with no exchange step: weak scaling, no collective); times are CUDA-event
+times, max over ranks.
+
+On one GPU the line also carries, under `workloads`, the same measurement (fewer steps) of
+C2 (tensor-bound verification), C1 at its three temperatures and four cells of C3's
+K x eps grid, each with target-only and draft-only decoding, phase times, and the speedup
+Eq. 8 predicts from the measured acceptance rate and cost ratios beside the measured one.
 
 `--impl reference` times the CPU oracle (fp64, as it stands) on a bounded sample of the same
 workload on the host cores, rank 0 only.
@@ -18,6 +25,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import multiprocessing as mp
 import os
 import subprocess
 import sys
@@ -33,6 +41,18 @@ if ROOT not in sys.path:
 METRIC = "committed_patches_per_s"
 UNIT = "patches/s"
 
+# DRAM traffic of the dominant kernels relative to their algorithmic bytes, from ncu captures of
+# small cases of the same kernels (dram__bytes_read.sum + dram__bytes_write.sum per launch over the
+# operands-once bytes of that launch; traffic grows in proportion to the units a launch processes).
+# A kernel that has changed since its capture is listed with None.
+NCU_TRAFFIC_RATIO = {
+    "gemm_sk_small_M": None,
+    "gemm_sk_mid_M": None,
+    "gemm_sk_large_M": None,
+    "attn": None,
+}
+NCU_TRAFFIC_SOURCE = {}
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -40,12 +60,12 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="C1")
+    ap.add_argument("--workload", default="C4")
     ap.add_argument("--tau", type=float, default=None)
     ap.add_argument("--K", type=int, default=None)
     ap.add_argument("--cpu-series", type=int, default=None, help="series per oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--others", default="C2,C4", help="comma list of further workloads to profile briefly ('' = none)")
+    ap.add_argument("--others", default="C2,C1,C3", help="comma list of further workloads measured on one GPU ('' = none)")
     return ap.parse_args()
 
 
@@ -103,81 +123,115 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ CPU oracle leg
-def oracle_sample(wl, K, tau, n_series, repeats):
-    """Time the oracle's speculative forecast on the first `n_series` series; returns patches/s."""
-    import torch
+# Series are independent.  Small models: the oracle decodes one series per worker process (fork; one
+# BLAS thread each), as many at a time as the host has cores.  Large models (every token step streams
+# gigabytes of fp64 weights, so processes only compete for memory bandwidth): one series after the
+# other, the BLAS library using its threads.  The oracle itself is untouched.
+_ORACLE_JOB = {}
+
+
+def _heavy(wl):
+    return wl.target.n_layers * wl.target.d_model ** 2 >= 24 * 1024 ** 2
+
+
+def _oracle_one(b):
     from oracle import tsfm_oracle as orc
-    from tests import parity
-    from tsfm_inputs import build_models, make_series
-    tw, dw = build_models(wl)
-    tm, dm = parity.oracle_models(wl, tw, dw)
-    s = make_series(wl, n_series)
-    times = []
-    for r in range(repeats):
+    lim = None
+    if _ORACLE_JOB["pooled"]:
+        try:
+            from threadpoolctl import threadpool_limits
+            lim = threadpool_limits(limits=1)
+        except Exception:
+            pass
+    j = _ORACLE_JOB
+    t0 = time.perf_counter()
+    orc.forecast_speculative(j["tm"], j["dm"], j["s"][b:b + 1], j["ctx"], j["H"], j["K"], j["tau"], j["seed"],
+                             series_index0=b)
+    del lim
+    return time.perf_counter() - t0
+
+
+class OracleSample:
+    """The oracle's speculative forecast on the first `n_series` series of a workload, optionally
+    on the first `patches` patches of the horizon only (a bounded sample of the same workload)."""
+
+    def __init__(self, wl, K, tau, n_series, patches=None):
+        from tests import parity
+        from tsfm_inputs import build_models, make_series
+        tw, dw = build_models(wl)
+        tm, dm = parity.oracle_models(wl, tw, dw)
+        self.wl, self.n = wl, n_series
+        self.T = min(patches or wl.n_patches, wl.n_patches)
+        H = wl.horizon if self.T == wl.n_patches else self.T * wl.patch_len
+        self.job = dict(tm=tm, dm=dm, s=make_series(wl, n_series), ctx=wl.ctx_len, H=H, K=K, tau=tau,
+                        seed=wl.forecast_seed)
+        self.workers = 1 if _heavy(wl) else max(1, min(n_series, os.cpu_count() or 1))
+        self.job["pooled"] = self.workers > 1
+        self.cores = self.workers if self.workers > 1 else (os.cpu_count() or 1)
+
+    def run(self, seed_offset=0):
+        """One pass over the sample; returns wall seconds."""
+        global _ORACLE_JOB
+        _ORACLE_JOB = dict(self.job, seed=self.job["seed"] + seed_offset)
         t0 = time.perf_counter()
-        orc.forecast_speculative(tm, dm, s, wl.ctx_len, wl.horizon, K, tau, wl.forecast_seed + r)
-        times.append(time.perf_counter() - t0)
-    total = float(np.sum(times))
-    return n_series * wl.n_patches * repeats / total, total, torch.get_num_threads()
+        if self.workers == 1:
+            for b in range(self.n):
+                _oracle_one(b)
+        else:
+            with mp.get_context("fork").Pool(self.workers) as pool:
+                pool.map(_oracle_one, range(self.n), chunksize=1)
+        return time.perf_counter() - t0
+
+    def describe(self):
+        wl = self.wl
+        part = "full forecast" if self.T == wl.n_patches else f"first {self.T} of {wl.n_patches} patches"
+        how = "one series per worker process" if self.workers > 1 else "series one after the other, threaded BLAS"
+        return (f"{self.n} of {wl.batch} series of {wl.name}, {part}, {how}; patches/s of the sample "
+                f"(series are independent, so the whole batch takes B / {self.n} times as long: extrapolated)")
+
+
+def cpu_baseline(wl, K, tau, n_series):
+    """Bounded oracle sample for the bench line: one pass, about 10-30 s of CPU work."""
+    smp = OracleSample(wl, K, tau, n_series)
+    secs = smp.run()
+    return {"value": smp.n * smp.T / secs, "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+            "sample": smp.describe() + f"; {secs:.1f} s"}
+
+
+def bench_config(wl, K, tau):
+    """The `config` object of the JSON line: the same for both arms."""
+    return {"workload": wl.name, "B": wl.batch, "ctx_len": wl.ctx_len, "P": wl.patch_len, "H": wl.horizon, "K": K,
+            "tau": tau, "series_per_gpu": wl.batch, "l2": "flushed between steps (256 MB write)",
+            "sharding": "by series, no collective"}
+
+
+def reference_sample_shape(wl, args):
+    """Series and patches per reference step: small enough that steps + warm-ups end within minutes."""
+    if _heavy(wl):
+        return args.cpu_series or 1, min(wl.n_patches, 8)
+    return args.cpu_series or min(wl.batch, os.cpu_count() or 1, 16), wl.n_patches
 
 
 def run_reference(args, wl, K, tau):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    n_series = args.cpu_series or min(wl.batch, 8)
-    # warm-up steps and timed steps, each one bounded sample
-    for _ in range(args.warmup):
-        oracle_sample(wl, K, tau, n_series, 1)
-    t0 = time.perf_counter()
-    val, total, cores = oracle_sample(wl, K, tau, n_series, args.steps)
-    ms = (time.perf_counter() - t0) * 1e3 / args.steps
-    sample = f"{n_series} of {wl.batch} series of {wl.name} per step, full forecast (T={wl.n_patches})"
+    n_series, patches = reference_sample_shape(wl, args)
+    smp = OracleSample(wl, K, tau, n_series, patches)
+    for i in range(args.warmup):
+        smp.run(i)
+    secs = [smp.run(i) for i in range(args.steps)]
+    total = float(np.sum(secs))
+    val = smp.n * smp.T * args.steps / total
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total * 1e3 / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "B": wl.batch, "ctx_len": wl.ctx_len, "P": wl.patch_len,
-                   "H": wl.horizon, "K": K, "tau": tau},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": bench_config(wl, K, tau),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+                         "sample": smp.describe() + " per step"},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
-
-
-# ------------------------------------------------------------------ other workloads (informational)
-def profile_workload(name, hbm_peak, tf_peak):
-    """One warm speculative and target-only forecast of another workload plus one profiled forecast:
-    where the tensor-bound verification GEMMs (C2) and the KV-bound attention (C4) stand against the
-    measured peaks.  Not part of the headline metric."""
-    import torch
-    import paper_2511_18191_b200 as tsfm
-    from tsfm_inputs import build_models, make_series, workload
-    wl = workload(name)
-    tw, dw = build_models(wl)
-    dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=wl.K)
-    s = make_series(wl)
-    ctx = torch.from_numpy(np.ascontiguousarray(s[:, :wl.ctx_len])).cuda()
-    for _ in range(2):
-        _, st = dec.forecast(ctx, wl.horizon, wl.K, wl.tau, wl.forecast_seed)
-        _, st_t = dec.target_only(ctx, wl.horizon)
-    d, dt = st.as_dict(), st_t.as_dict()
-    tsfm.tsfm_spec_set_profiling(dec.h, True)
-    dec.forecast(ctx, wl.horizon, wl.K, wl.tau, wl.forecast_seed, stats=False)
-    prof = tsfm.tsfm_spec_kernel_profile(dec.h)
-    tsfm.tsfm_spec_set_profiling(dec.h, False)
-    dec.close()
-    tot = sum(v["ms_total"] for v in prof.values())
-    kernels = {}
-    for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms_total"])[:3]:
-        gbs, tfs = v["bytes"] / v["ms_total"] / 1e6, v["flops"] / v["ms_total"] / 1e9
-        kernels[k] = {"share": round(v["ms_total"] / tot, 3), "avg_launch_us": round(v["ms_total"] * 1e3 / v["launches"], 2),
-                      "GB/s": round(gbs, 1), "frac_hbm": round(gbs / hbm_peak, 4),
-                      "TFLOP/s": round(tfs, 1), "frac_tensor": round(tfs / tf_peak, 4)}
-    return {"ms_per_forecast": d["ms_total"], "ms_target_only": dt["ms_total"],
-            "phases_ms": {k: d[k] for k in ("ms_prefill", "ms_draft", "ms_verify", "ms_accept")},
-            "rounds": d["rounds"], "accepted_over_tested": d["proposals_accepted"] / max(d["proposals_tested"], 1),
-            "B": wl.batch, "patches_per_s": wl.batch * wl.n_patches / (d["ms_total"] * 1e-3),
-            "kernels_event_timed": kernels}
 
 
 # ------------------------------------------------------------------ multi-rank host logic
@@ -205,7 +259,9 @@ def whole_job_value(world: int, series_per_rank: int, patches: int, steps: int, 
 def throughput_law(stats, to_stats, K, T):
     """Predicted speedup S(K) = E[L] / (c K + v) of the paper's Eq. 8 from this run's own measurements:
     acceptance rate alpha = accepted / tested, c = draft step time / target step time, v = verification
-    pass time / target step time (phase clocks of the decoder), E[L] of Eq. 7."""
+    pass time / target step time (phase clocks of the decoder), E[L] of Eq. 7.  Eq. 8 leaves out what
+    both arms pay once (prefill) and what only the speculative arm pays (the draft's prefill, the
+    accept step): `with_fixed_costs` is the same ratio with those terms put back, from the same clocks."""
     rounds = max(stats["rounds"], 1)
     step = to_stats["ms_verify"] / T
     if step <= 0:
@@ -216,20 +272,192 @@ def throughput_law(stats, to_stats, K, T):
     e_l = float(K + 1) if alpha >= 1.0 else (1.0 - alpha ** (K + 1)) / (1.0 - alpha)
     import paper_2511_18191_b200 as tsfm
     k_star, s_star = tsfm.tsfm_advise_block_size(alpha, c, v, 32)
+    spec_ms = stats["ms_prefill"] + stats["ms_draft"] + stats["ms_verify"] + stats["ms_accept"]
+    tonly_ms = to_stats["ms_prefill"] + to_stats["ms_verify"]
     return {"alpha": alpha, "c": c, "v": v, "E_L": e_l, "predicted_speedup": e_l / (c * K + v),
+            "rounds": rounds, "rounds_if_all_series_had_mean_yield": T / e_l,
+            "with_fixed_costs": {"predicted_speedup": tonly_ms / spec_ms if spec_ms > 0 else None,
+                                 "target_prefill_ms": to_stats["ms_prefill"],
+                                 "draft_prefill_ms": stats["ms_prefill"] - to_stats["ms_prefill"],
+                                 "accept_ms": stats["ms_accept"],
+                                 "note": "rounds run until the slowest series is done; Eq. 8 counts T / E[L] of them"},
             "advised_K": k_star, "predicted_speedup_at_advised_K": s_star}
+
+
+# ------------------------------------------------------------------ one fully timed workload
+def measure(wl, K, tau, steps, warmup, peaks, *, rank=0, world=1, local=0, e2e=True, clocks=False, barrier=None):
+    """Times speculative, target-only and draft-only forecasts of one workload (L2 flushed between
+    steps, CUDA events on the decoder's stream, max over ranks) and profiles one forecast per kernel."""
+    import torch
+    import paper_2511_18191_b200 as tsfm
+    from tsfm_inputs import build_models, make_series
+
+    barrier = barrier or (lambda: torch.cuda.synchronize())
+    tw, dw = build_models(wl)
+    dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=K, device=f"cuda:{local}")
+    s = make_series(rank_workload(wl, rank))
+    ctx_host = torch.from_numpy(np.ascontiguousarray(s[:, :wl.ctx_len])).pin_memory()
+    ctx = ctx_host.cuda()
+    B, H, T = wl.batch, wl.horizon, wl.n_patches
+    out = torch.empty((B, H), device="cuda")
+    out_host = torch.empty((B, H)).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > 126 MB of L2
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, n, seed0):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        barrier()
+        for i in range(n):
+            flush.fill_(i & 0xFF)
+            ev[i][0].record(stream)
+            fn(seed0 + i)
+            ev[i][1].record(stream)
+        barrier()
+        return max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), world)
+
+    spec = lambda seed: tsfm.tsfm_spec_forecast(dec.h, ctx, B, wl.ctx_len, H, K, tau, seed, out, None)
+    tonly = lambda seed: tsfm.tsfm_target_only_forecast(dec.h, ctx, B, wl.ctx_len, H, out, None)
+    donly = lambda seed: tsfm.tsfm_draft_only_forecast(dec.h, ctx, B, wl.ctx_len, H, out, None)
+    spec_host = lambda seed: tsfm.tsfm_spec_forecast_host(dec.h, ctx_host, B, wl.ctx_len, H, K, tau, seed, out_host, None)
+
+    seed0 = wl.forecast_seed
+    for i in range(warmup):
+        spec(seed0 + i)
+        tonly(0)
+        donly(0)
+        if e2e:
+            spec_host(seed0 + i)
+    sampler = ClockSampler(local) if clocks and rank == 0 else None
+    if sampler:
+        sampler.start()
+    launches0 = tsfm.tsfm_launch_count()
+    ms_spec = timed(spec, steps, seed0)
+    launches = tsfm.tsfm_launch_count() - launches0
+    clk = sampler.stop() if sampler else None
+    ms_tonly = timed(tonly, steps, 0)
+    ms_donly = timed(donly, steps, 0)
+    # accuracy of the three arms against the synthetic ground-truth tail (normalised series: plain MSE)
+    truth = torch.from_numpy(np.ascontiguousarray(s[:, wl.ctx_len:wl.ctx_len + H])).cuda()
+    mse = {}
+    for name, fn in (("target_only", tonly), ("draft_only", donly), ("speculative", spec)):
+        fn(seed0)
+        mse[name] = float(((out - truth) ** 2).mean().item())
+    ms_e2e = timed(spec_host, steps, seed0) if e2e else None
+
+    # counters and phase clocks averaged over the timed seeds, then one profiled forecast per kernel
+    acc = None
+    for i in range(min(steps, 5)):
+        _, st = dec.forecast(ctx, H, K, tau, seed0 + i)
+        d = st.as_dict()
+        if acc is None:
+            acc = {k: (list(v) if isinstance(v, list) else v) for k, v in d.items()}
+        else:
+            for k, v in d.items():
+                acc[k] = [a + b for a, b in zip(acc[k], v)] if isinstance(v, list) else acc[k] + v
+    n_avg = min(steps, 5)
+    stats = {k: ([x / n_avg for x in v] if isinstance(v, list) else v / n_avg) for k, v in acc.items()}
+    _, st_t = dec.target_only(ctx, H)
+    to_stats = st_t.as_dict()
+    tsfm.tsfm_spec_set_profiling(dec.h, True)
+    flush.fill_(1)
+    spec(seed0)
+    prof = tsfm.tsfm_spec_kernel_profile(dec.h)
+    tsfm.tsfm_spec_set_profiling(dec.h, False)
+    dec.close()
+    del flush
+
+    step_ms = ms_spec / steps
+    total_ms = sum(v["ms_total"] for v in prof.values())
+    hbm_peak, tf_peak = peaks["hbm"], peaks["tf_sustained"]
+    kernels = {}
+    for name, p in sorted(prof.items(), key=lambda kv: -kv[1]["ms_total"]):
+        share = p["ms_total"] / total_ms
+        # The per-kernel events bracket launches made one by one from the host (they carry the launch
+        # gaps); the timed region replays a graph.  A kernel's time inside a step is therefore taken as
+        # its share of the profiled kernel time x the step time, which cannot exceed the step.
+        in_step_ms = share * step_ms
+        kernels[name] = {
+            "share": round(share, 4), "launches_per_step": int(p["launches"]), "ms_per_step": in_step_ms,
+            "avg_launch_us": in_step_ms * 1e3 / p["launches"],
+            "bytes_per_launch": p["bytes"] / p["launches"], "flops_per_launch": p["flops"] / p["launches"],
+            "GB/s": p["bytes"] / (in_step_ms * 1e-3) / 1e9, "TFLOP/s": p["flops"] / (in_step_ms * 1e-3) / 1e12,
+        }
+        kernels[name]["frac_hbm"] = kernels[name]["GB/s"] / hbm_peak
+        kernels[name]["frac_tensor"] = kernels[name]["TFLOP/s"] / tf_peak
+    tested, accd = stats["proposals_tested"], stats["proposals_accepted"]
+    lh = stats["L_hist"]
+    res = {
+        "workload": wl.name, "B": B, "K": K, "tau": tau, "steps": steps,
+        "ms_per_step": step_ms, "patches_per_s": whole_job_value(world, B, T, steps, ms_spec),
+        "target_only": {"ms_per_step": ms_tonly / steps, "patches_per_s": whole_job_value(world, B, T, steps, ms_tonly)},
+        "draft_only": {"ms_per_step": ms_donly / steps, "patches_per_s": whole_job_value(world, B, T, steps, ms_donly)},
+        "speedup_vs_target_only": ms_tonly / ms_spec,
+        "phases_ms": {k: stats[k] for k in ("ms_prefill", "ms_draft", "ms_verify", "ms_accept")},
+        "target_only_phases_ms": {"ms_prefill": to_stats["ms_prefill"], "ms_decode": to_stats["ms_verify"]},
+        "throughput_law": throughput_law(stats, to_stats, K, T),
+        "acceptance": {"accepted_over_tested": accd / max(tested, 1), "rounds": stats["rounds"],
+                       "mean_yield": sum(l * c for l, c in enumerate(lh)) / max(sum(lh), 1)},
+        "mse_vs_truth": mse,
+        "kernels": kernels,
+        "_raw": {"ms_spec": ms_spec, "ms_e2e": ms_e2e, "launches": int(launches), "clocks": clk},
+    }
+    return res
+
+
+def roofline_of(m, peaks):
+    """The roofline object of a measured workload: its dominant kernel against the bound that binds it."""
+    name, k = next(iter(m["kernels"].items()))            # sorted by time: the first is the dominant one
+    # arithmetic intensity of the launches decides the bound: the ridge is peak flops / peak bytes
+    ridge = peaks["tf_sustained"] * 1e12 / (peaks["hbm"] * 1e9)
+    tensor = k["flops_per_launch"] / max(k["bytes_per_launch"], 1.0) > ridge
+    ratio = NCU_TRAFFIC_RATIO.get(name)
+    r = {"kernel": name, "bound": "tensor" if tensor else "hbm",
+         "achieved": k["TFLOP/s"] if tensor else k["GB/s"],
+         "peak": peaks["tf_sustained"] if tensor else peaks["hbm"],
+         "unit": "TFLOP/s" if tensor else "GB/s",
+         "frac": k["frac_tensor"] if tensor else k["frac_hbm"],
+         "peak_source": peaks["source"] + (" (sustained cuBLAS bf16: the kernel runs inside a long step)" if tensor else " (copy)"),
+         "traffic": ratio * k["bytes_per_launch"] if ratio is not None else None,
+         "traffic_source": NCU_TRAFFIC_SOURCE.get(name),
+         "algorithmic_bytes_per_launch": k["bytes_per_launch"], "flops_per_launch": k["flops_per_launch"],
+         "avg_launch_us": k["avg_launch_us"], "launches_per_step": k["launches_per_step"],
+         "share_of_step": k["share"], "ms_per_step": k["ms_per_step"],
+         "timing": "share of the per-kernel event profile (stream mode) x CUDA-event time of the graph-replayed step",
+         "frac_hbm": k["frac_hbm"], "frac_tensor": k["frac_tensor"]}
+    return r
+
+
+def other_workloads(names):
+    """(label, workload, K, tau) of the further entries: C2, C1 at its temperatures, cells of C3's grid."""
+    from tsfm_inputs import workload
+    out = []
+    for n in names:
+        if n == "C1":
+            wl = workload("C1")
+            out += [(f"C1_tau{t:g}", wl, wl.K, t) for t in wl.tau_sweep]
+        elif n == "C3":
+            for eps in (0.0, 1e-3):
+                wl = workload("C3", draft_eps=eps)
+                out += [(f"C3_K{k}_eps{eps:g}", wl, k, wl.tau) for k in (1, 4)]
+        else:
+            wl = workload(n)
+            out.append((n, wl, wl.K, wl.tau))
+    return out
 
 
 # ------------------------------------------------------------------ our arm
 def run_ours(args, wl, K, tau):
-    import torch
-    import torch.distributed as dist
-    import paper_2511_18191_b200 as tsfm
-    from tsfm_inputs import build_models, make_series
-
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    # the CPU leg first: its worker processes are forked before this process touches CUDA
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        cpu = cpu_baseline(wl, K, tau, args.cpu_series or (1 if _heavy(wl) else min(wl.batch, 16)))
+
+    import torch
+    import torch.distributed as dist
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the decoder has no CPU path")
     torch.cuda.set_device(local)
@@ -241,140 +469,50 @@ def run_ours(args, wl, K, tau):
             dist.barrier()
         torch.cuda.synchronize()
 
-    peaks = {}
+    pk = {}
     try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        pk = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
     except Exception:
         pass
-    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
-    peak_src = "measured" if "hbm_gbs" in peaks else "fallback"
+    peaks = {"hbm": float(pk.get("hbm_gbs", 6650.0)), "tf_sustained": float(pk.get("bf16_tflops_sustained", 1400.0)),
+             "tf_burst": float(pk.get("bf16_tflops", 1590.0)), "source": "measured" if "hbm_gbs" in pk else "fallback"}
 
-    tw, dw = build_models(wl)
-    dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=K, device=f"cuda:{local}")
-    # every rank decodes its own batch of B series (different series per rank)
-    s = make_series(rank_workload(wl, rank))
-    ctx_host = torch.from_numpy(np.ascontiguousarray(s[:, :wl.ctx_len])).pin_memory()
-    ctx = ctx_host.cuda()
-    B, H, T = wl.batch, wl.horizon, wl.n_patches
-    out = torch.empty((B, H), device="cuda")
-    out_host = torch.empty((B, H)).pin_memory()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > 126 MB of L2
-    stream = torch.cuda.current_stream()
-
-    def timed(fn, steps, seeds0):
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        barrier()
-        for i in range(steps):
-            flush.fill_(i & 0xFF)
-            ev[i][0].record(stream)
-            fn(seeds0 + i)
-            ev[i][1].record(stream)
-        barrier()
-        return max_over_ranks(sum(a.elapsed_time(b) for a, b in ev), world)
-
-    spec = lambda seed: tsfm.tsfm_spec_forecast(dec.h, ctx, B, wl.ctx_len, H, K, tau, seed, out, None)
-    tonly = lambda seed: tsfm.tsfm_target_only_forecast(dec.h, ctx, B, wl.ctx_len, H, out, None)
-    donly = lambda seed: tsfm.tsfm_draft_only_forecast(dec.h, ctx, B, wl.ctx_len, H, out, None)
-    spec_host = lambda seed: tsfm.tsfm_spec_forecast_host(dec.h, ctx_host, B, wl.ctx_len, H, K, tau, seed, out_host, None)
-
-    seed0 = wl.forecast_seed
-    for i in range(args.warmup):
-        spec(seed0 + i)
-        tonly(0)
-        donly(0)
-        spec_host(seed0 + i)
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    launches0 = tsfm.tsfm_launch_count()
-    ms_spec = timed(spec, args.steps, seed0)
-    launches = tsfm.tsfm_launch_count() - launches0
-    clocks = sampler.stop() if rank == 0 else None
-    ms_tonly = timed(tonly, args.steps, 0)
-    ms_donly = timed(donly, args.steps, 0)
-    # accuracy of the three arms against the synthetic ground-truth tail (normalised series: plain MSE)
-    truth = torch.from_numpy(np.ascontiguousarray(s[:, wl.ctx_len:wl.ctx_len + H])).cuda()
-    mse = {}
-    for name, fn in (("target_only", tonly), ("draft_only", donly), ("speculative", spec)):
-        fn(seed0)
-        mse[name] = float(((out - truth) ** 2).mean().item())
-    ms_e2e = timed(spec_host, args.steps, seed0)
-
-    # one forecast for the acceptance counters, then one profiled forecast for per-kernel times
-    _, st = dec.forecast(ctx, H, K, tau, seed0)
-    stats = st.as_dict()
-    _, st_t = dec.target_only(ctx, H)
-    to_stats = st_t.as_dict()
-    tsfm.tsfm_spec_set_profiling(dec.h, True)
-    flush.fill_(1)
-    n_prof = 3
-    for i in range(n_prof):
-        spec(seed0 + i)
-    prof = tsfm.tsfm_spec_kernel_profile(dec.h)
-    tsfm.tsfm_spec_set_profiling(dec.h, False)
-
-    units = world * B * T * args.steps
-    value = whole_job_value(world, B, T, args.steps, ms_spec)
+    m = measure(wl, K, tau, args.steps, args.warmup, peaks, rank=rank, world=world, local=local, e2e=True,
+                clocks=True, barrier=barrier)
+    raw = m.pop("_raw")
     result = None
     if rank == 0:
-        total_ms = sum(v["ms_total"] for v in prof.values())
-        top = max(prof.items(), key=lambda kv: kv[1]["ms_total"])
-        name, p = top
-        achieved = p["bytes"] / (p["ms_total"] * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                    "frac": achieved / hbm_peak, "peak_source": peak_src, "traffic": None,
-                    "launches_per_step": p["launches"] / n_prof,
-                    "avg_launch_us": p["ms_total"] * 1e3 / p["launches"],
-                    "share_of_kernel_time": p["ms_total"] / total_ms,
-                    "achieved_tflops": p["flops"] / (p["ms_total"] * 1e-3) / 1e12,
-                    "kernel_shares": {k: round(v["ms_total"] / total_ms, 4) for k, v in prof.items()}}
-        # The per-kernel events above bracket launches made one by one from the host, so each
-        # duration carries the launch gap around it.  The timed region itself replays a graph with
-        # programmatic dependent launches; this kernel's time inside it is estimated as its share
-        # of the profiled kernel time x the graph's step time (an estimate, reported beside the
-        # directly measured figure, not instead of it).
-        in_graph_us = roofline["share_of_kernel_time"] * (ms_spec / args.steps) * 1e3 / roofline["launches_per_step"]
-        bytes_per_launch = p["bytes"] / p["launches"]
-        roofline["in_graph_estimate"] = {"avg_launch_us": in_graph_us,
-                                         "achieved": bytes_per_launch / (in_graph_us * 1e-6) / 1e9,
-                                         "frac": bytes_per_launch / (in_graph_us * 1e-6) / 1e9 / hbm_peak}
-        tested, acc = stats["proposals_tested"], stats["proposals_accepted"]
+        B, H, T = wl.batch, wl.horizon, wl.n_patches
+        units = world * B * T * args.steps
         result = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_spec / args.steps, "higher_is_better": True,
+            "metric": METRIC, "value": m["patches_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": m["ms_per_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-            "config": {"workload": wl.name, "B": B, "ctx_len": wl.ctx_len, "P": wl.patch_len, "H": H, "K": K,
-                       "tau": tau, "series_per_gpu": B, "l2": "flushed between steps (256 MB write)",
-                       "sharding": "by series, no collective"},
-            "e2e": {"value": units / (ms_e2e * 1e-3), "unit": UNIT,
+            "config": bench_config(wl, K, tau),
+            "e2e": {"value": units / (raw["ms_e2e"] * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": B * wl.ctx_len * 4, "d2h_bytes_per_step": B * H * 4},
-            "gpu_launches": int(launches),
-            "clocks": clocks,
-            "roofline": roofline,
-            "target_only": {"value": units / (ms_tonly * 1e-3), "unit": UNIT, "ms_per_step": ms_tonly / args.steps},
-            "draft_only": {"value": units / (ms_donly * 1e-3), "unit": UNIT, "ms_per_step": ms_donly / args.steps},
-            "speedup_vs_target_only": ms_tonly / ms_spec,
-            "mse_vs_truth": mse,
-            "throughput_law": throughput_law(stats, to_stats, K, T),
-            "acceptance": {"accepted_over_tested": acc / max(tested, 1), "rounds": stats["rounds"],
-                           "mean_yield": (sum(l * c for l, c in enumerate(stats["L_hist"])) /
-                                          max(sum(stats["L_hist"]), 1))},
+            "gpu_launches": raw["launches"],
+            "clocks": raw["clocks"],
+            "roofline": roofline_of(m, peaks),
+            "peaks": peaks,
         }
-        if not args.no_cpu_baseline and world == 1:
-            n_series = args.cpu_series or min(B, 32)
-            val, total, cores = oracle_sample(wl, K, tau, n_series, 3)
-            result["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                      "sample": f"{n_series} of {B} series of {wl.name}, full forecast, 3 repeats, "
-                                                f"{total:.1f} s"}
-    dec.close()
-    if result is not None and world == 1 and args.others:
-        tf_peak = float(peaks.get("bf16_tflops_sustained", 1400.0))
-        result["other_workloads"] = {"peaks": {"hbm_gbs": hbm_peak, "bf16_tflops_sustained": tf_peak, "source": peak_src}}
-        for name in [n for n in args.others.split(",") if n]:
+        for k in ("target_only", "draft_only", "speedup_vs_target_only", "phases_ms", "target_only_phases_ms",
+                  "throughput_law", "acceptance", "mse_vs_truth", "kernels"):
+            result[k] = m[k]
+        if cpu is not None:
+            result["cpu_baseline"] = cpu
+    if world == 1 and args.others:
+        result["workloads"] = {}
+        for label, owl, oK, otau in other_workloads([n for n in args.others.split(",") if n and n != wl.name]):
             try:
-                result["other_workloads"][name] = profile_workload(name, hbm_peak, tf_peak)
-            except Exception as e:          # informational: never lose the headline line
-                result["other_workloads"][name] = {"error": repr(e)}
+                om = measure(owl, oK, otau, max(3, min(args.steps, 10)), max(3, min(args.warmup, 3)), peaks, e2e=False)
+                om.pop("_raw")
+                om["roofline"] = roofline_of(om, peaks)
+                om["kernels"] = {k: {kk: v[kk] for kk in ("share", "avg_launch_us", "GB/s", "TFLOP/s", "frac_hbm", "frac_tensor")}
+                                 for k, v in list(om["kernels"].items())[:4]}
+                result["workloads"][label] = om
+            except Exception as e:          # further entries never cost the headline line
+                result["workloads"][label] = {"error": repr(e)}
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()

@@ -39,9 +39,10 @@ extern "C" {
 #endif
 
 #define TSFM_OK            0
-#define TSFM_ERR_ARG      (-1)  /* null pointer, B < 1, K < 1 or > max_K, tau not finite or <= 0, H < 1 */
-#define TSFM_ERR_SHAPE    (-2)  /* ctx_len % P != 0, fewer than 2 context patches, capacity exceeded,
-                                   d_model % n_heads != 0, unsupported head size, bad weight blob   */
+#define TSFM_ERR_ARG      (-1)  /* null pointer, B < 1, K < 1, tau not finite or <= 0, H < 1           */
+#define TSFM_ERR_SHAPE    (-2)  /* ctx_len % P != 0, fewer than 2 context patches, capacity exceeded
+                                   (B, N, T or K beyond the handle's max_*), d_model % n_heads != 0,
+                                   unsupported head size, bad weight blob                           */
 #define TSFM_ERR_ARCH     (-3)  /* current device is not compute capability 10.x                   */
 #define TSFM_ERR_CUDA     (-4)  /* a CUDA runtime/driver call failed (see tsfm_last_cuda_error)     */
 #define TSFM_ERR_TIMEOUT  (-5)  /* a bounded device-side wait expired                               */
@@ -56,11 +57,6 @@ extern "C" {
 
 #define TSFM_GEMM_AUTO  0       /* bf16 contractions on tcgen05 tensor cores where shapes allow     */
 #define TSFM_GEMM_SIMT  1       /* force the plain FMA kernels everywhere (differential reference)  */
-#define TSFM_GEMM_FUSED_PASS 3  /* as AUTO, but a pass over at most 32 tokens per series group runs as
-                                   ONE cluster kernel (embedding to mean head) when the model has
-                                   head size 64 and at most 8 heads; measured slower than AUTO on
-                                   B200 (one CTA per head cannot stream its weight share fast
-                                   enough), kept as an alternative and a differential target        */
 
 #define TSFM_EXEC_GRAPH   0       /* a forecast is one CUDA-graph launch: prologue, a device-side WHILE
                                    over the rounds, de-normalisation; no host round trip             */
@@ -173,7 +169,7 @@ int tsfm_spec_forecast(tsfm_spec *h, const float *series, int32_t B, int32_t ctx
  * eps are standard normals from the same Philox key: Box-Muller on the words of counter
  * (series, round, position, stream | element / 2), stream 0x10000000 for proposals and 0x20000000
  * for the fallback, cosine branch for even elements, sine for odd.  variant == NULL is the deployed
- * scheme.  Noise is not available with TSFM_GEMM_FUSED_PASS (TSFM_ERR_ARG). */
+ * scheme. */
 typedef struct {
   float   sigma_q;
   float   fallback_noise;
@@ -234,7 +230,7 @@ int tsfm_accept_round(void *stream, const float *x, const float *mu_q, const flo
 /* Full causal forward of one of the handle's models over fresh sequences (positions
  * 0..n-1), for numerics checks: tokens dev [B, n, P] fp32 (already normalised), out dev
  * [B, n, P] fp32 = next-patch mean at every position.  which: 0 target, 1 draft.
- * n <= max_ctx_tokens + max_horizon_patches + max_K.  Overwrites the KV cache. */
+ * n <= max_ctx_tokens (TSFM_ERR_SHAPE beyond it).  Overwrites the KV cache; synchronises the stream. */
 int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t B, int32_t n,
                        float *out);
 

@@ -158,7 +158,7 @@ __global__ void __launch_bounds__(128) accept_kernel(AcceptArgs a) {
     else u = uniform_from_word(philox4x32_10(
                  make_uint4((uint32_t)(a.series0 + b), (uint32_t)a.round_idx, (uint32_t)lane, 0u), a.key).x);
     lu = logf(u);
-    ok = lu <= fminf(l, 0.f);
+    ok = (lu <= l) && (lu <= 0.f);                   // log u <= min(l, 0); a NaN statistic compares false: rejected
     if (a.ell) a.ell[(size_t)b * K + lane] = l;
     if (a.log_u) a.log_u[(size_t)b * K + lane] = lu;
   }

@@ -21,7 +21,6 @@
 #include "accept.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_sk.cuh"
-#include "pass_cluster.cuh"
 
 using namespace tsfm;
 
@@ -103,7 +102,6 @@ struct ModelDev {
   void *Kc = nullptr, *Vc = nullptr;     // [L][B][heads][cap][dh]
   size_t kv_layer_elems = 0;
   float2 *rope = nullptr;                // [cap][dh/2] (cos, sin)
-  ClPlan cl;                             // whole-pass cluster kernel (small batches), if the shape allows
 };
 
 }  // namespace
@@ -130,7 +128,6 @@ struct tsfm_spec {
   DevState *st = nullptr;
   int cap = 0;
   bool use_tc = false;
-  bool use_cluster = false;              // whole-pass cluster kernel where eligible
   bool pdl = false;                      // launches carry the programmatic-serialization attribute
   ModelDev tgt, drf;
   // activations (sized for M_max rows)
@@ -149,6 +146,7 @@ struct tsfm_spec {
   float *tr_ell = nullptr, *tr_logu = nullptr;   // [max_T][B][K]
   float *stage_in = nullptr, *stage_out = nullptr;   // device staging for the *_host entry points
   int last_B = 0, last_K = 0;
+  int enqueue_err = TSFM_OK;             // first failure while enqueuing work (a launch that was refused)
   // optional per-launch timing (tsfm_spec_set_profiling)
   bool profiling = false;
   struct ProfRec { int cls; cudaEvent_t e0, e1; double bytes, flops; };
@@ -162,10 +160,12 @@ struct tsfm_spec {
 namespace {
 
 // Kernel classes for per-launch timing.
-enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_TC, KC_GEMM_SIMT, KC_ATTN, KC_HEAD, KC_ACCEPT, KC_DENORM,
-       KC_PASS, KC_COUNT };
-const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_sk", "gemm_simt", "attn",
-                                            "head", "accept", "denorm", "pass_cluster"};
+// The tensor-core contraction is one kernel in three regimes: up to 512 tokens it streams weights
+// (HBM / latency bound), from 4096 tokens it is tensor bound, between them it is one wave of tiles.
+enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_TC_SMALL, KC_GEMM_TC_MID, KC_GEMM_TC_LARGE, KC_GEMM_SIMT,
+       KC_ATTN, KC_HEAD, KC_ACCEPT, KC_DENORM, KC_COUNT };
+const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_sk_small_M", "gemm_sk_mid_M",
+                                            "gemm_sk_large_M", "gemm_simt", "attn", "head", "accept", "denorm"};
 
 // Brackets one launch with two events when profiling is on (no-op otherwise).
 struct KTimer {
@@ -252,40 +252,6 @@ int make_rope(tsfm_spec *h, ModelDev &m) {
   return TSFM_OK;
 }
 
-// Device-resident descriptors of a model for the whole-pass cluster kernel (tensor maps of
-// every weight matrix, gains, cache pointers).  Leaves the plan invalid when the shape is
-// outside that kernel's domain.
-int make_cluster_plan(tsfm_spec *h, ModelDev &m) {
-  const int d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len, L = m.arch.n_layers;
-  m.cl.valid = false;
-  if (m.dh != 64 || !cl_model_ok(m.arch.n_heads, d, f, P)) return TSFM_OK;
-  std::vector<ClLayer> ls(L);
-  ClModel cm{};
-  for (int l = 0; l < L; ++l) {
-    const LayerDev &ly = m.layers[l];
-    if (tc_encode(&ls[l].qkv, ly.Wqkv, 3 * d, d, 64) || tc_encode(&ls[l].wo, ly.Wo, d, d, 128) ||
-        tc_encode(&ls[l].w1, ly.W1, f, d, 128) || tc_encode(&ls[l].w2, ly.W2, d, f, 128))
-      return TSFM_ERR_CUDA;
-    ls[l].g1 = ly.g1;
-    ls[l].g2 = ly.g2;
-    ls[l].Kc = (bf16 *)m.Kc + (size_t)l * m.kv_layer_elems;
-    ls[l].Vc = (bf16 *)m.Vc + (size_t)l * m.kv_layer_elems;
-  }
-  if (tc_encode(&cm.head, m.W_head, P, d, 128)) return TSFM_ERR_CUDA;
-  cm.W_emb = (const bf16 *)m.W_emb;
-  cm.g_f = m.g_f;
-  cm.rope = m.rope;
-  cm.n_layers = L; cm.d = d; cm.heads = m.arch.n_heads; cm.ff = f; cm.P = P;
-  if (int rc = dev_alloc(h, &m.cl.layers, (size_t)L)) return rc;
-  if (int rc = dev_alloc(h, &m.cl.model, 1)) return rc;
-  CU_TRY(cudaMemcpyAsync(m.cl.layers, ls.data(), sizeof(ClLayer) * L, cudaMemcpyHostToDevice, h->stream));
-  CU_TRY(cudaMemcpyAsync(m.cl.model, &cm, sizeof(ClModel), cudaMemcpyHostToDevice, h->stream));
-  CU_TRY(cudaStreamSynchronize(h->stream));
-  m.cl.R = m.arch.n_heads; m.cl.d = d; m.cl.ff = f; m.cl.P = P; m.cl.L = L;
-  m.cl.valid = true;
-  return TSFM_OK;
-}
-
 template <typename T> size_t attn_smem_bytes(int dh, int nk) {
   const int vw = AttnWords<T>::per_row(dh);
   return (size_t)nk * (2 * vw + 1) * 4 + (size_t)ATTN_QT * nk * sizeof(float) + (size_t)5 * ATTN_QT * dh * sizeof(float) +
@@ -308,13 +274,12 @@ int attn_set_attr(size_t bytes) {
 // Short rows with at least this many (series, head) pairs: one warp per pair instead of four
 // (measured: C2's draft, 1024 pairs, 15 % faster that way; no difference at 256 pairs).
 constexpr int kFlashWarpMaxCap = 64, kFlashWarpMinPairs = 512;
-#ifndef FLASH_ST_SHORT
-#define FLASH_ST_SHORT 2
-#endif
+// one-tile passes: a two-stage ring (each warp has a few chunks only, and a third CTA fits on the SM)
+constexpr int kFlashStShort = 2;
 template <int DH> int flash_set_attr() {
   CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH, 3>::SMEM_BYTES));
-  CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH, FLASH_ST_SHORT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              FlashGeom<DH, FLASH_ST_SHORT>::SMEM_BYTES));
+  CU_TRY(cudaFuncSetAttribute(attn_flash_kernel<DH, kFlashStShort>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              FlashGeom<DH, kFlashStShort>::SMEM_BYTES));
   CU_TRY(cudaFuncSetAttribute(attn_flash_single_kernel<DH, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::single_bytes(1)));
   CU_TRY(cudaFuncSetAttribute(attn_flash_single_kernel<DH, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, FlashGeom<DH>::single_bytes(2)));
   return TSFM_OK;
@@ -368,13 +333,12 @@ void prefer_max_smem_all() {
   prefer_max_smem(gemm_sk_kernel<1, false>);
   prefer_max_smem(gemm_sk_kernel<1, true>);
   prefer_max_smem(gemm_sk_kernel<2, false>);
-  prefer_max_smem(pass_cluster_kernel);
   prefer_max_smem(attn_flash_kernel<32, 3>);
-  prefer_max_smem(attn_flash_kernel<32, FLASH_ST_SHORT>);
+  prefer_max_smem(attn_flash_kernel<32, kFlashStShort>);
   prefer_max_smem(attn_flash_kernel<64, 3>);
-  prefer_max_smem(attn_flash_kernel<64, FLASH_ST_SHORT>);
+  prefer_max_smem(attn_flash_kernel<64, kFlashStShort>);
   prefer_max_smem(attn_flash_kernel<128, 3>);
-  prefer_max_smem(attn_flash_kernel<128, FLASH_ST_SHORT>);
+  prefer_max_smem(attn_flash_kernel<128, kFlashStShort>);
   prefer_max_smem(attn_flash_single_kernel<32, 1>);
   prefer_max_smem(attn_flash_single_kernel<32, 2>);
   prefer_max_smem(attn_flash_single_kernel<64, 1>);
@@ -445,8 +409,16 @@ void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C,
   const double bytes = ((double)N * K + (double)M * K) * e + (double)M * N * out_b;
   const double flops = 2.0 * M * N * K;
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
-    KTimer kt(h, KC_GEMM_TC, bytes, flops);
-    if (gemm_sk_launch(h->ls, h->pdl, *plan, C, M, epi, h->dev_status, norm)) { LAUNCHED(); return; }
+    KTimer kt(h, M <= 512 ? KC_GEMM_TC_SMALL : M < 4096 ? KC_GEMM_TC_MID : KC_GEMM_TC_LARGE, bytes, flops);
+    if (gemm_sk_launch(h->ls, h->pdl, *plan, C, M, epi, h->dev_status, norm)) {
+      LAUNCHED();
+    } else if (h->enqueue_err == TSFM_OK) {
+      // No silent fallback: the FMA kernel knows nothing of a folded norm, and a pass that mixes
+      // the two would be wrong without saying so.  The call that enqueued this reports the error.
+      h->enqueue_err = TSFM_ERR_CUDA;
+      g_cuda_err = std::string("tensor-core contraction could not be launched: ") + cudaGetErrorString(cudaGetLastError());
+    }
+    return;
   }
   KTimer kt(h, KC_GEMM_SIMT, bytes, flops);
   launch_gemm_simt<T>(h->ls, h->pdl, (const T *)A, (const T *)W, C, M, N, K, epi);
@@ -484,8 +456,8 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
       launch_ex(h->ls, h->pdl, attn_flash_kernel<DH, 3>, grid, dim3(128), (size_t)FlashGeom<DH, 3>::SMEM_BYTES, h->qkv,
                 (bf16 *)Kc, (bf16 *)Vc, m.rope, g, m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
     else      // one query tile: each warp has a few chunks only, a two-stage ring lets a third CTA onto the SM
-      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH, FLASH_ST_SHORT>, grid, dim3(128),
-                (size_t)FlashGeom<DH, FLASH_ST_SHORT>::SMEM_BYTES, h->qkv, (bf16 *)Kc, (bf16 *)Vc, m.rope, g,
+      launch_ex(h->ls, h->pdl, attn_flash_kernel<DH, kFlashStShort>, grid, dim3(128),
+                (size_t)FlashGeom<DH, kFlashStShort>::SMEM_BYTES, h->qkv, (bf16 *)Kc, (bf16 *)Vc, m.rope, g,
                 m.arch.n_heads, pairs, mode, (bf16 *)h->ao);
   } else {
     const int QT = g.q_len <= ATTN_QT ? g.q_len : ATTN_QT;
@@ -582,41 +554,9 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   }
 }
 
-// The whole pass as one cluster kernel, when the model and the token count allow it.
-bool pass_fused(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout,
-                unsigned long long *stamp) {
-  if (!h->use_cluster || head_mode == HEAD_NONE) return false;
-  int Bg, BN, G, stages, smem;
-  if (!cl_geometry(m.cl, B, g.q_len, h->cap, &Bg, &BN, &G, &stages, &smem)) return false;
-  ClArgs a{};
-  a.model = m.cl.model;
-  a.layers = m.cl.layers;
-  a.hist_in = h->hist;
-  a.hist_out = h->hist;
-  a.vout = vout;
-  a.g = g;
-  a.B = B; a.Bg = Bg; a.BN = BN; a.stages = stages;
-  a.head_all = head_mode == HEAD_ALL_TO_VOUT;
-  a.eps = h->cfg.rms_eps;
-  a.status = h->dev_status;
-  a.stamp = stamp;
-  // algorithmic bytes: every weight once + the cached keys and values + tokens in, predictions out
-  const int d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len, L = m.arch.n_layers;
-  const double M = (double)B * g.q_len;
-  const double wbytes = 2.0 * ((double)d * P * 2 + (double)L * (4.0 * d * d + 2.0 * d * f));
-  const double kv = (double)L * B * (std::max(g.base, 0) + g.q_len) * 2.0 * d * 2;
-  const double flops = 2.0 * M * ((double)d * P * 2 + (double)L * (4.0 * d * d + 2.0 * d * f)) +
-                       4.0 * M * (std::max(g.base, 0) + 0.5 * g.q_len) * d * L;
-  KTimer kt(h, KC_PASS, wbytes + kv + 2.0 * M * P * 4, flops);
-  if (!cl_launch(h->ls, h->pdl, m.cl, a, G, smem)) return false;
-  LAUNCHED();
-  return true;
-}
-
 void pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout = nullptr,
           unsigned long long *stamp = nullptr, DraftStep ds = DraftStep{}) {
   if (g.q_len < 1) return;
-  if (pass_fused(h, m, B, g, head_mode, vout, stamp)) return;
   if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout, stamp, ds);
   else run_pass<float>(h, m, B, g, head_mode, vout, stamp, ds);
 }
@@ -720,6 +660,13 @@ void enqueue_single_model(tsfm_spec *h, ModelDev &m, int B, int N, int T, int H)
   enqueue_denorm(h, B, N, H);
 }
 
+// The first error met while enqueuing (and clears it).
+int take_enqueue_err(tsfm_spec *h) {
+  const int rc = h->enqueue_err;
+  h->enqueue_err = TSFM_OK;
+  return rc;
+}
+
 // ---------------------------------------------------------------- graph capture
 // A forecast of a given geometry is captured once into a CUDA graph and replayed: the
 // prologue, a WHILE node whose body is one round (the round-end kernel sets the condition),
@@ -783,6 +730,7 @@ int capture_graph(tsfm_spec *h, const GraphKey &k, int slot, GraphInfo *out) {
   out->n_fixed = g_launches.load() - launches0 - n_body;
   g_launches.store(launches0);                     // captured launches have not run
   if (rc == TSFM_OK) step(cudaGetLastError(), "capture");
+  if (rc == TSFM_OK) rc = take_enqueue_err(h);
   if (rc == TSFM_OK) step(cudaGraphInstantiate(&out->exec, graph, 0), "cudaGraphInstantiate");
   if (graph) cudaGraphDestroy(graph);
   if (rc == TSFM_OK) {
@@ -915,9 +863,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   const int P = cfg->patch_len;
   if (cfg->dtype != TSFM_F32 && cfg->dtype != TSFM_BF16) return TSFM_ERR_ARG;
   if (cfg->exec_mode & ~(TSFM_EXEC_STREAM | TSFM_EXEC_NO_PDL)) return TSFM_ERR_ARG;
-  if (cfg->gemm_backend != TSFM_GEMM_AUTO && cfg->gemm_backend != TSFM_GEMM_SIMT &&
-      cfg->gemm_backend != TSFM_GEMM_FUSED_PASS)
-    return TSFM_ERR_ARG;
+  if (cfg->gemm_backend != TSFM_GEMM_AUTO && cfg->gemm_backend != TSFM_GEMM_SIMT) return TSFM_ERR_ARG;
   if (cfg->draft_mode != TSFM_DRAFT_SEPARATE && cfg->draft_mode != TSFM_DRAFT_LAYER_SKIP) return TSFM_ERR_ARG;
   if (cfg->max_batch < 1 || cfg->max_ctx_tokens < 2 || cfg->max_horizon_patches < 1 || cfg->max_K < 1 ||
       cfg->max_K > TSFM_MAX_K)
@@ -944,7 +890,6 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   h->stream = h->ls = (cudaStream_t)cfg->stream;
   h->cap = cfg->max_ctx_tokens + cfg->max_horizon_patches + cfg->max_K + 1;
   h->use_tc = cfg->dtype == TSFM_BF16 && cfg->gemm_backend != TSFM_GEMM_SIMT;
-  h->use_cluster = cfg->dtype == TSFM_BF16 && cfg->gemm_backend == TSFM_GEMM_FUSED_PASS;
   h->pdl = (cfg->exec_mode & TSFM_EXEC_NO_PDL) == 0;
   int rc = TSFM_OK;
   auto fail = [&](int code) { tsfm_spec_destroy(h); return code; };
@@ -1024,11 +969,6 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
       }
     }
   }
-  if (h->use_cluster) {
-    if ((rc = cl_init())) return fail(rc);
-    for (ModelDev *m : {&h->tgt, &h->drf})
-      if ((rc = make_cluster_plan(h, *m))) return fail(rc);
-  }
   if (cudaStreamSynchronize(h->stream) != cudaSuccess) return fail(TSFM_ERR_CUDA);
   {
     std::lock_guard<std::mutex> lock(g_handles_mu);
@@ -1055,6 +995,7 @@ static int single_model_forecast(tsfm_spec *h, int mode, const float *series, in
     enqueue_single_model(h, mode == 1 ? h->tgt : h->drf, B, N, T, H);
   }
   CU_TRY(cudaGetLastError());
+  if (int rc = take_enqueue_err(h)) return rc;
   if (stats) {
     std::memset(stats, 0, sizeof(*stats));
     DevState st;
@@ -1092,8 +1033,6 @@ int tsfm_spec_forecast_variant(tsfm_spec *h, const float *series, int32_t B, int
     if (!std::isfinite(variant->sigma_q) || variant->sigma_q < 0.f || !std::isfinite(variant->fallback_noise) ||
         variant->fallback_noise < 0.f)
       return TSFM_ERR_ARG;
-    if (h && h->use_cluster && (variant->sample_proposals || variant->fallback_noise != 0.f))
-      return TSFM_ERR_ARG;             // the whole-pass cluster kernel has no noise path
   }
   if (int rc = check_call(h, series, B, ctx_len, H, out, K)) return rc;
   const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
@@ -1119,6 +1058,7 @@ int tsfm_spec_forecast_variant(tsfm_spec *h, const float *series, int32_t B, int
   }
   h->last_B = B; h->last_K = K;
   CU_TRY(cudaGetLastError());
+  if (int rc = take_enqueue_err(h)) return rc;
   if (stats) {
     std::memset(stats, 0, sizeof(*stats));
     AcceptCounters c;
@@ -1220,6 +1160,7 @@ int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t
   h->ls = h->stream;
   pass(h, which == 0 ? h->tgt : h->drf, B, PassGeom{nullptr, 0, n, h->cap}, HEAD_ALL_TO_VOUT, out);
   CU_TRY(cudaGetLastError());
+  if (int rc = take_enqueue_err(h)) return rc;
   int status = 0;
   CU_TRY(cudaMemcpyAsync(&status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
   CU_TRY(cudaStreamSynchronize(h->stream));
@@ -1243,7 +1184,10 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t
   if (!plan.valid) return TSFM_ERR_SHAPE;
   int *status = nullptr;
   CU_TRY(cudaMalloc((void **)&status, sizeof(int)));
-  CU_TRY(cudaMemsetAsync(status, 0, sizeof(int), s));
+  if (cudaError_t e0 = cudaMemsetAsync(status, 0, sizeof(int), s)) {
+    cudaFree(status);
+    CU_TRY(e0);
+  }
   const bool ok = gemm_sk_launch(s, false, plan, C, M, EPI_F32, status);
   if (ok) LAUNCHED();
   int hs = 0;
@@ -1307,14 +1251,14 @@ int tsfm_gemm_bf16_static(void *stream, const void *A, const void *W, float *C, 
   // accumulator this call adds into must start at zero
   CU_TRY(cudaMemsetAsync(status, 0, 256, s));
   CU_TRY(cudaMemsetAsync(acc, 0, out_bytes, s));
-  const bool ok = gemm_tc_launch(s, plan, A, acc, M, EPI_ATOMIC, status);
-  if (ok) LAUNCHED();
+  if (!gemm_tc_launch(s, plan, A, acc, M, EPI_ATOMIC, status)) return TSFM_ERR_INTERNAL;
+  CU_TRY(cudaGetLastError());            // a refused launch: C is left untouched
+  LAUNCHED();
   int hs = 0;
   CU_TRY(cudaMemcpyAsync(C, acc, out_bytes, cudaMemcpyDeviceToDevice, s));
   CU_TRY(cudaMemcpyAsync(&hs, status, sizeof(int), cudaMemcpyDeviceToHost, s));
   CU_TRY(cudaStreamSynchronize(s));
   CU_TRY(cudaGetLastError());
-  if (!ok) return TSFM_ERR_INTERNAL;
   return hs ? TSFM_ERR_TIMEOUT : TSFM_OK;
 }
 

@@ -54,7 +54,6 @@ struct SkNorm {
   float inv_d, eps;
 };
 
-static int g_sk_force_stages = 0;   // experiment override
 struct SkShape {
   int BN, stages, tmem_cols, smem_bytes;
 };
@@ -65,7 +64,6 @@ static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1) {
   s.BN = BN;
   const int stage = TC_W_BYTES * wt + BN * TC_BK * 2;
   int stages = wt == 2 ? 3 : BN > 160 ? 4 : BN > 64 ? 3 : 4;
-  if (g_sk_force_stages) stages = g_sk_force_stages;
   if (stages > kb_per_cta) stages = kb_per_cta < 1 ? 1 : kb_per_cta;
   int bytes = stages * stage;
   if (split && bytes < BN * TC_BM * 4) bytes = BN * TC_BM * 4;
@@ -425,13 +423,16 @@ static int sk_encode_c(CUtensorMap *map, const void *base, int rows, int N, int 
 
 static int gemm_sk_init() {
   if (int rc = gemm_tc_init()) return rc;
-  static bool done = false;
-  if (done) return 0;
+  static bool dev_done[TC_MAX_DEVICES] = {false};       // per device, like gemm_tc_init
+  std::lock_guard<std::mutex> lock(g_tc_init_mu);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TC_MAX_DEVICES) return -4;
+  if (dev_done[dev]) return 0;
   if (cudaFuncSetAttribute(gemm_sk_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_sk_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_sk_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
     return -4;
-  done = true;
+  dev_done[dev] = true;
   return 0;
 }
 
@@ -451,15 +452,8 @@ static int gemm_sk_plan(GemmSkPlan *plan, const void *W, int N, int K, const voi
 // Tile and split choice for M tokens: one token tile up to 256 rows (rounded up to 16), and
 // as many K splits (a power of two, at most 8, at most the number of K blocks) as it takes to
 // put the grid on most of the 148 SMs.
-static int g_sk_force_wt = 0;
-static int g_sk_force_bn = 0, g_sk_force_s = 0;   // experiment overrides (0 = automatic)
 static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
   *WT = 1;
-  if (g_sk_force_bn && g_sk_force_s) {
-    *BN = g_sk_force_bn; *S = g_sk_force_s;
-    if (g_sk_force_wt) *WT = g_sk_force_wt;
-    return;
-  }
   // Measured on B200 (graph replay, dependent launches): up to a few hundred tokens a 32-token
   // tile with K split until the grid has ~150-250 CTAs is fastest (the partial-tile exchange
   // grows with the tile, the latency chain does not shrink); large M takes 128/256-token tiles.

@@ -16,6 +16,7 @@
 // still frees its tensor memory and returns.
 #pragma once
 #include <cuda.h>
+#include <mutex>
 #include "common.cuh"
 #include "kernels_simt.cuh"   // EPI_* codes
 
@@ -24,7 +25,10 @@ namespace tsfm {
 constexpr int TC_BM = 128;         // output features per CTA (MMA M)
 constexpr int TC_BK = 64;          // K elements per pipeline stage (one 128-byte swizzle row)
 constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
-constexpr unsigned long long TC_WAIT_NS = 2000000000ull;
+// Bound of every mbarrier wait.  The longest legitimate wait is an epilogue warp waiting for its
+// own CTA's main loop (tens of microseconds); 100 ms is far beyond that and short enough that a
+// wedged pipeline gives the device back at once.
+constexpr unsigned long long TC_WAIT_NS = 100000000ull;
 
 struct GemmTcPlan {
   bool valid = false;
@@ -231,18 +235,29 @@ template <int BN> static int gemm_tc_set_attr() {
                               TcShape<BN>::SMEM_BYTES) == cudaSuccess ? 0 : -4;
 }
 
-// Resolve the driver's tensor-map encoder and opt the kernels into large shared memory.
+// Resolve the driver's tensor-map encoder (once per process) and opt the kernels into large
+// shared memory (once per device: function attributes belong to the current device).  Calls from
+// several threads are serialised.
+constexpr int TC_MAX_DEVICES = 64;
+static std::mutex g_tc_init_mu;
 static int gemm_tc_init() {
-  if (g_encode) return 0;
-  void *fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-      qres != cudaDriverEntryPointSuccess || !fn)
-    return -4;
+  static bool dev_done[TC_MAX_DEVICES] = {false};
+  std::lock_guard<std::mutex> lock(g_tc_init_mu);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= TC_MAX_DEVICES) return -4;
+  if (!g_encode) {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn)
+      return -4;
+    g_encode = (PFN_encodeTiled)fn;
+  }
+  if (dev_done[dev]) return 0;
   if (gemm_tc_set_attr<16>() || gemm_tc_set_attr<32>() || gemm_tc_set_attr<64>() || gemm_tc_set_attr<128>() ||
       gemm_tc_set_attr<256>())
     return -4;
-  g_encode = (PFN_encodeTiled)fn;
+  dev_done[dev] = true;
   return 0;
 }
 

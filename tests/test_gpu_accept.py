@@ -117,3 +117,32 @@ def test_general_statistic_with_unequal_scales():
     for b in range(B):
         for i in range(K):
             assert ell[b, i] == pytest.approx(orc.log_ratio(x[b, i], mu_p[b, i], mu_q[b, i], sp, sq), rel=3e-5, abs=2e-6)
+
+
+def test_non_finite_proposals_are_rejected_and_the_target_corrects():
+    """A NaN or infinite proposal makes Eq. 5's statistic NaN (with mean proposals the draft term is
+    inf - inf).  A NaN never passes the test: the position is a rejection, and the committed patch
+    there is the target's own prediction -- on the GPU as in the oracle."""
+    B, K, P = 5, 3, 32
+    rng = np.random.default_rng(3)
+    mu_p = rng.standard_normal((B, K + 1, P)).astype(np.float32)
+    x = (mu_p[:, :K] + 0.1 * rng.standard_normal((B, K, P))).astype(np.float32)
+    x[0, 1, 5] = np.nan
+    x[1, 0, :] = np.inf
+    x[2, 2, 3] = -np.inf
+    mu_q = x.copy()
+    mu_q[3] = mu_p[3, :K]                                     # series 3: finite draft mean, infinite proposal
+    x[3, 1, 0] = np.inf
+    u = np.full((B, K), 2.0 ** -24, dtype=np.float32)         # accepts every finite statistic
+    commit, nacc, ell, logu, done = run_accept(x, mu_q, mu_p, 100, 1.0, 1.0, 0, 0, 0, u, np.zeros(B, np.int32))
+    want_n = [1, 0, 2, 1, 3]
+    for b in range(B):
+        n = 0
+        for i in range(K):                                    # the oracle's decisions on the same inputs
+            if not orc.accept(orc.log_ratio(x[b, i], mu_p[b, i], mu_q[b, i], 1.0, 1.0), float(u[b, i])):
+                break
+            n += 1
+        assert n == want_n[b] == nacc[b], (b, n, nacc[b])
+        assert done[b] == n + 1
+        np.testing.assert_array_equal(commit[b, n], mu_p[b, n])     # the target's mean replaces the rejected patch
+        np.testing.assert_array_equal(commit[b, :n], x[b, :n])

@@ -34,6 +34,7 @@ def check_stats(st, B, T, K):
 def run_and_compare(wl, K, tau, seed, ids, backend=0, batch=None, H=None, exec_mode=0):
     H = H or wl.horizon
     B = batch or wl.batch
+    ids = list(ids)
     dec, tw, dw = make_decoder(wl, backend=backend, max_K=max(K, wl.K), batch=B, exec_mode=exec_mode)
     s, ctx = series_on_device(wl, B)
     out, st = dec.forecast(ctx, H, K, tau, seed)
@@ -41,20 +42,28 @@ def run_and_compare(wl, K, tau, seed, ids, backend=0, batch=None, H=None, exec_m
     d = check_stats(st, B, T, K)
     nacc, ell, logu = dec.last_trace(B, K)
     assert nacc.shape[0] == d["rounds"]
+    # the decoder's near-margin counter is the count over its own trace
+    assert d["near_margin_decisions"] == parity.gpu_near_margin_total(nacc, ell, logu, K, parity.MARGIN[wl.dtype])
     ref, st0 = dec.target_only(ctx, H)
     got = out.cpu().numpy()
     tgt_only = ref.cpu().numpy()
     dec.close()
     tm, dm = parity.oracle_models(wl, tw, dw)
-    res = parity.compare_forecast(wl, tm, dm, s, H, K, tau, seed, got, nacc, ids)
-    want_t = orc.forecast_target_only(tm, s[list(ids)], wl.ctx_len, H)
+    res = parity.compare_forecast(wl, tm, dm, s, H, K, tau, seed, got, nacc, ids, gpu_ell=ell, gpu_logu=logu)
+    want_t = parity.oracle_target_only(tm, s, wl.ctx_len, H, ids)
     kind, tol = parity.VALUE_TOL[wl.dtype]
-    res["target_only_error"] = parity.value_error(kind, tgt_only[list(ids)], want_t)
-    assert res["target_only_error"] <= tol
+    each = parity.per_series_errors(kind, tgt_only[ids], want_t)
+    res["target_only_error"] = float(each.max())
+    assert each.max() <= tol, f"target-only, series {ids[int(each.argmax())]}: {kind} error {each.max():.4g} > {tol}"
     res["stats"] = d
     print(wl.name, K, tau, {k: v for k, v in res.items() if k != "stats"},
           "acc", d["proposals_accepted"], "/", d["proposals_tested"], "rounds", d["rounds"])
     return res
+
+
+def spread(B, n):
+    """n series ids spread over a batch of B (first, last and evenly spaced ones between)."""
+    return sorted(set(int(round(i * (B - 1) / (n - 1))) for i in range(n)))
 
 
 EXEC = pytest.mark.parametrize("exec_mode", [1, 0], ids=["stream", "graph"])
@@ -74,8 +83,8 @@ def test_c0_shape_ragged_batch_fp32(K, tau, H, exec_mode):
     run_and_compare(wl, K, tau, 7, range(6), exec_mode=exec_mode)
 
 
-@pytest.mark.parametrize("backend,exec_mode", [(1, 1), (0, 1), (0, 0), (3, 0)],
-                         ids=["simt-stream", "tcgen05-stream", "tcgen05-graph", "fused_pass-graph"])
+@pytest.mark.parametrize("backend,exec_mode", [(1, 1), (0, 1), (0, 0)],
+                         ids=["simt-stream", "tcgen05-stream", "tcgen05-graph"])
 @pytest.mark.parametrize("tau", [0.5, 1.0, 2.0])
 def test_c1_full(tau, backend, exec_mode):
     wl = workload("C1")
@@ -124,24 +133,43 @@ def test_launch_counter_counts_replayed_rounds():
     assert counts[0] == counts[1] and counts[0] > 0
 
 
-def test_c2_subset():
+def test_c2_sixteen_series():
     wl = workload("C2")
-    run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, [0, 1, 100, 255])
+    res = run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, spread(wl.batch, 16))
+    assert res["series"] == 16
 
 
-@pytest.mark.parametrize("K,eps", [(1, 1e-2), (2, 1e-1), (4, 1e-2), (8, 1e-3), (4, 0.0)])
-def test_c3_sweep_subset(K, eps):
+@pytest.mark.parametrize("K", [1, 2, 4, 8])            # (the upper decorator varies fastest: weights are reused)
+@pytest.mark.parametrize("eps", [0.0, 1e-3, 1e-2, 1e-1])
+def test_c3_whole_sweep(K, eps):
+    """Every cell of the K x eps grid, 16 series each.  eps = 0 is a draft that is the target:
+    everything is accepted and every round yields K + 1.  With this build's perturbation recipe
+    (eps x the tensor's standard deviation) eps = 1e-1 still accepts about nine proposals in ten at
+    tau = 1; the low end of the acceptance range is reached through tau (next test)."""
     wl = workload("C3", draft_eps=eps)
-    res = run_and_compare(wl, K, wl.tau, wl.forecast_seed, [0, 513, 1023])
+    res = run_and_compare(wl, K, wl.tau, wl.forecast_seed, spread(wl.batch, 16))
     d = res["stats"]
     if eps == 0.0:                       # draft == target: everything accepted, every round yields K+1
         assert d["proposals_accepted"] == d["proposals_tested"]
         assert d["rounds"] == -(-wl.n_patches // (K + 1))
+    else:
+        assert d["proposals_accepted"] < d["proposals_tested"] or eps < 1e-1
 
 
-def test_c4_subset():
+@pytest.mark.parametrize("tau,lo,hi", [(0.3, 0.05, 0.9), (0.1, 0.0, 0.1)])
+def test_c3_low_acceptance_end(tau, lo, hi):
+    """The most perturbed draft of the sweep at small acceptance temperatures: ragged per-series
+    acceptance in the middle of the range, then hardly any (every round yields one patch)."""
+    wl = workload("C3", draft_eps=1e-1)
+    res = run_and_compare(wl, 4, tau, wl.forecast_seed, spread(wl.batch, 16))
+    d = res["stats"]
+    assert lo <= d["proposals_accepted"] / d["proposals_tested"] <= hi
+
+
+def test_c4_sixteen_series():
     wl = workload("C4")
-    run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, [0, 63])
+    res = run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, spread(wl.batch, 16))
+    assert res["series"] == 16
 
 
 @pytest.mark.parametrize("target,draft", [
@@ -195,7 +223,7 @@ def test_draft_only_forecast_matches_oracle(name, ids):
     tm, dm = parity.oracle_models(wl, tw, dw)
     want = orc.forecast_target_only(dm, s[list(ids)], wl.ctx_len, wl.horizon)
     kind, tol = parity.VALUE_TOL[wl.dtype]
-    assert parity.value_error(kind, out.cpu().numpy()[list(ids)], want) <= tol
+    assert parity.per_series_errors(kind, out.cpu().numpy()[list(ids)], want).max() <= tol
 
 
 @pytest.mark.parametrize("K,H,ctx_patches,B", [(32, 96 * 3, 2, 2), (1, 50, 2, 1), (5, 96, 3, 7), (8, 96 * 9 + 1, 7, 3)])

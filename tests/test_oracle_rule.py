@@ -92,6 +92,23 @@ def test_accept_is_u_le_alpha():
     assert orc.accept(800.0, 0.999)                   # overflow-safe
 
 
+def test_a_non_finite_statistic_is_a_rejection():
+    """A NaN (or -inf) statistic never passes the test u <= min(1, e^l): the comparison is false, the
+    proposal is rejected and the target's own prediction takes its place."""
+    for ell in (float("nan"), float("-inf")):
+        for u in (2.0 ** -24, 0.5, 1.0 - 2.0 ** -24):
+            assert not orc.accept(ell, u)
+    # an infinite or NaN proposal makes the statistic non-finite whatever the draft mean is
+    mu = np.zeros(8)
+    for bad in (np.inf, -np.inf, np.nan):
+        x = mu.copy()
+        x[3] = bad
+        for mu_q in (x, mu):                              # mean proposal (x = mu_q) and a finite draft mean
+            l = orc.log_ratio(x, mu, mu_q, 1.0, 1.0)
+            assert not l > -np.inf or math.isnan(l)
+            assert not orc.accept(l, 2.0 ** -24)
+
+
 # ------------------------------------------- Algorithm 1 / Figure 1 example ----
 def _scripted_round(decisions, K=4):
     """Drive one round with uniforms chosen to realise a given accept/reject script."""
@@ -327,6 +344,23 @@ def test_standard_normals_are_standard_and_streams_differ():
     b = orc.standard_normals(7, 1, 2, 3, orc.NOISE_FALLBACK, 8)
     assert not np.allclose(a, b)
     np.testing.assert_array_equal(a[:5], orc.standard_normals(7, 1, 2, 3, orc.NOISE_PROPOSAL, 5))   # prefix-stable
+
+
+def test_standard_normals_invert_to_the_philox_words_they_were_made_from():
+    """Box-Muller is invertible: an (even, odd) element pair gives back its two uniforms,
+    z0^2 + z1^2 = -2 ln u1 and atan2(z1, z0) = 2 pi u2.  That fixes which Philox word feeds the
+    radius and which the angle, the cosine branch on even and the sine branch on odd elements, and
+    the counter layout (series, round, position, stream | pair index)."""
+    seed, series, rnd, pos = 0x1234567800000009, 5, 2, 3
+    key = (seed & 0xFFFFFFFF, seed >> 32)
+    for stream in (orc.NOISE_PROPOSAL, orc.NOISE_FALLBACK):
+        z = orc.standard_normals(seed, series, rnd, pos, stream, 10)
+        for j in range(5):
+            w = orc.philox4x32_10((series, rnd, pos, stream | j), key)
+            u1, u2 = orc.uniform_from_word(w[0]), orc.uniform_from_word(w[1])
+            assert z[2 * j] ** 2 + z[2 * j + 1] ** 2 == pytest.approx(-2.0 * math.log(u1), rel=1e-12)
+            ang = math.atan2(z[2 * j + 1], z[2 * j]) % (2.0 * math.pi)
+            assert ang == pytest.approx(2.0 * math.pi * u2, abs=1e-9)
 
 
 def test_sampled_proposals_accept_at_the_equal_covariance_rate_in_one_dimension():
