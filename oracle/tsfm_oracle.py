@@ -21,6 +21,11 @@ What follows the paper, and where:
   index N-1+i, appendix B "Per-Family Boundary Indexing")  -> speculative_round
 * capped-geometric block length and dependence band (Eq. 7; appendix
   propositions on block length and dependence)             -> capped_geometric_*
+* input tokens shorter than the predicted patch (the point-token family of
+  appendix B: input patch length P_in, a horizon head of P steps): a patch is
+  P / P_in tokens and the boundary of prefix i sits at token
+  N - 1 + i (P / P_in) (appendix B "Per-Family Boundary Indexing")
+                                                           -> speculative_round, boundary_indices
 
 The paper fixes the decoding rule but not the network: it says only
 "decoder-only Transformer / point head".  The transformer below (pre-norm,
@@ -130,18 +135,27 @@ class Model:
     d_model: int
     n_heads: int
     d_ff: int
-    patch_len: int
+    patch_len: int                # P: steps predicted per forward (length of a committed patch)
     w: Dict[str, np.ndarray]
 
     @property
     def d_head(self) -> int:
         return self.d_model // self.n_heads
 
+    @property
+    def patch_in(self) -> int:
+        """P_in: steps per input token (= P for the patch-token families, 1 for point tokens)."""
+        return self.w["W_emb"].shape[1]
+
+    @property
+    def tokens_per_patch(self) -> int:
+        return self.patch_len // self.patch_in
+
 
 def make_model(weights: Dict[str, np.ndarray], n_layers: int, d_model: int, n_heads: int,
                d_ff: int, patch_len: int) -> Model:
     w = {k: np.asarray(v, dtype=np.float64) for k, v in weights.items()}
-    assert w["W_emb"].shape == (d_model, patch_len)
+    assert w["W_emb"].shape[0] == d_model and patch_len % w["W_emb"].shape[1] == 0
     assert w["W_head"].shape == (patch_len, d_model)
     return Model(n_layers, d_model, n_heads, d_ff, patch_len, w)
 
@@ -192,8 +206,8 @@ class KVCache:
 def forward(model: Model, z: np.ndarray, cache: Optional[KVCache] = None) -> np.ndarray:
     """Next-patch means at every input position.
 
-    z: [n, P] patch tokens.  Row t of the result is the model's mean for the
-    patch that follows tokens 0..t (of the cache plus ``z``).  With a cache the
+    z: [n, P_in] input tokens.  Row t of the result is the model's mean for the
+    P steps that follow tokens 0..t (of the cache plus ``z``).  With a cache the
     new tokens sit at positions cache.length .. cache.length + n - 1 and their
     keys/values are appended; without one this is the full recomputation.
     """
@@ -285,13 +299,18 @@ def speculative_round(hist: np.ndarray, target: Model, draft: Model, K: int, sig
     hist: [n, P] context + committed patches (normalised space).  ``uniforms``
     supplies u_1..u_K.  ``forced`` (optional) overrides the decisions, used to
     replay another implementation's accept/reject sequence.  ``caches`` is an
-    optional (target KVCache, draft KVCache) pair holding a prefix of ``hist``;
-    without it both models recompute from scratch.
+    optional (target KVCache, draft KVCache) pair holding a prefix of ``hist``
+    (their lengths count tokens); without it both models recompute from scratch.
+
+    The models read the sequence as tokens of P_in steps (P / P_in of them per
+    patch); the target's prediction after prefix i is read at token index
+    N - 1 + i (P / P_in), N the token count of ``hist``.
     """
     n = hist.shape[0]
     tc, dc = caches if caches is not None else (None, None)
 
-    def run(model, cache, tokens):
+    def run(model, cache, patches):
+        tokens = patches.reshape(-1, model.patch_in)
         if cache is None:
             return forward(model, tokens)
         out = forward(model, tokens[cache.length:], cache)
@@ -309,13 +328,14 @@ def speculative_round(hist: np.ndarray, target: Model, draft: Model, K: int, sig
     x = np.stack(props, axis=0)                           # x_i = mu_q^(i) (+ sigma_q eps)
     mu_q = np.stack(means, axis=0)
     o = run(target, tc, np.concatenate([hist, x], axis=0))
-    mu_p = o[n - 1: n + K]                                # boundaries N-1+i, i = 0..K
+    at = boundary_indices(n * target.tokens_per_patch, K, target.tokens_per_patch)
+    mu_p = o[at]                                          # boundaries N-1+i(P/P_in), i = 0..K
     if var.fallback_noise != 0.0:
         mu_p = mu_p + var.fallback_noise * np.asarray(fallback_eps, dtype=np.float64)
     ell, log_u, dec = [], [], []
     n_acc = 0
     for i in range(K):
-        mp_i = o[n - 1 + i]                               # the statistic uses the noise-free target mean
+        mp_i = o[at[i]]                                   # the statistic uses the noise-free target mean
         l_i = log_ratio(x[i], mp_i, mu_q[i], sigma, sigma_q)
         if not var.tempering:
             l_i *= x.shape[1]                             # l_i is (1/d) log p/q: undo the 1/d
@@ -327,6 +347,12 @@ def speculative_round(hist: np.ndarray, target: Model, draft: Model, K: int, sig
             break
         n_acc += 1
     return RoundRecord(n_acc, n_acc + 1, n_acc + 1, ell, log_u, dec, x, mu_p)
+
+
+def boundary_indices(n_tokens: int, K: int, tokens_per_patch: int = 1) -> np.ndarray:
+    """Token indices at which the target's predictions mu_p^(1..K+1) are read in the pass over
+    [h, x_1..x_K]: N - 1 + i (P / P_in), i = 0..K, with N the token count of h."""
+    return n_tokens - 1 + tokens_per_patch * np.arange(K + 1)
 
 
 def committed_patches(rec: RoundRecord) -> np.ndarray:
@@ -353,10 +379,11 @@ def forecast_target_only(target: Model, series: np.ndarray, ctx_len: int, H: int
         hist = _patches((series[b, :ctx_len].astype(np.float64) - m) / sd, P)
         cache = KVCache.empty(target) if use_cache else None
         for _ in range(T):
+            tokens = hist.reshape(-1, target.patch_in)
             if cache is None:
-                mu = forward(target, hist)[-1]
+                mu = forward(target, tokens)[-1]
             else:
-                mu = forward(target, hist[cache.length:], cache)[-1]
+                mu = forward(target, tokens[cache.length:], cache)[-1]
             hist = np.concatenate([hist, mu[None, :]], axis=0)
         out[b] = (hist[-T:].reshape(-1) * sd + m)[:H]
     return out
@@ -419,8 +446,8 @@ def forecast_speculative(target: Model, draft: Model, series: np.ndarray, ctx_le
             recs.append(rec)
             if caches is not None:                       # roll both caches back
                 keep = hist.shape[0] - 1                 # everything but the newest patch
-                for c in caches:
-                    c.truncate(min(c.length, keep))
+                for c, mdl in zip(caches, (target, draft)):
+                    c.truncate(min(c.length, keep * mdl.tokens_per_patch))
         trace.rounds.append(recs)
         out[b] = (hist[-T:].reshape(-1) * sd + m)[:H]
     return out, trace

@@ -199,6 +199,67 @@ def test_sigma_to_zero_recovers_target_only_with_zero_acceptance():
     assert all(len(recs) == 6 for recs in tr.rounds)
 
 
+# ------------------------------- point tokens: P_in < P, strided boundaries ----
+def point_token_models(P=8, P_in=2, seed=5, same=False):
+    ta, da = Arch(2, 32, 4, 64), Arch(1, 16, 2, 32)
+    tw = make_weights(ta, P, seed, "f32", stream=0, patch_in=P_in)
+    target = orc.make_model(tw, ta.n_layers, ta.d_model, ta.n_heads, ta.d_ff, P)
+    if same:
+        return target, target
+    dw = make_weights(da, P, seed, "f32", stream=1, patch_in=P_in)
+    return target, orc.make_model(dw, da.n_layers, da.d_model, da.n_heads, da.d_ff, P)
+
+
+def test_boundary_indices_follow_the_per_family_rule():
+    """Prefix i is read at token N - 1 + i (P / P_in): with patch tokens that is N - 1 + i; with
+    point tokens and a 64-step head, 64 tokens further per prefix."""
+    assert list(orc.boundary_indices(30, 4)) == [29, 30, 31, 32, 33]
+    assert list(orc.boundary_indices(3072, 3, 64)) == [3071, 3135, 3199, 3263]
+    t, _ = point_token_models(P=8, P_in=2)
+    assert t.patch_in == 2 and t.tokens_per_patch == 4
+
+
+@pytest.mark.parametrize("P_in", [1, 2, 4, 8])
+def test_strided_boundaries_are_prefix_forwards(P_in):
+    """The single-pass property with input tokens shorter than a patch: the prediction read at
+    token N - 1 + i (P / P_in) of the one causal pass over [h, x_1..x_K] is what a forward over
+    h + x_{1:i} alone gives at its last token -- for the draft rollout as for the verification."""
+    P, K = 8, 3
+    target, draft = point_token_models(P, P_in)
+    hist = toy_series(1, 48, seed=7)[0].reshape(-1, P)
+    rec = orc.speculative_round(hist, target, draft, K, 1.0, [0.5] * K)
+    seq = hist
+    for i in range(K):
+        np.testing.assert_allclose(rec.mu_q[i], orc.forward(draft, seq.reshape(-1, P_in))[-1], atol=1e-12)
+        np.testing.assert_allclose(rec.mu_p[i], orc.forward(target, seq.reshape(-1, P_in))[-1], atol=1e-12)
+        seq = np.concatenate([seq, rec.mu_q[i][None]], axis=0)
+    np.testing.assert_allclose(rec.mu_p[K], orc.forward(target, seq.reshape(-1, P_in))[-1], atol=1e-12)
+    # a wrong stride would read a prediction made from an incomplete patch: those differ
+    o = orc.forward(target, np.concatenate([hist, rec.mu_q], axis=0).reshape(-1, P_in))
+    if P_in < P:
+        assert not np.allclose(o[hist.shape[0] * (P // P_in) - 1 + 1], rec.mu_p[1])
+
+
+def test_point_token_forecasts_keep_the_rule_level_invariants():
+    """draft == target accepts everything and reproduces target-only decoding; the KV-cached and the
+    full-recompute forecasts agree; every round commits between 1 and K + 1 patches, T in total."""
+    P, P_in, K, H = 8, 2, 3, 44
+    target, draft = point_token_models(P, P_in)
+    s = toy_series(3, 40 + H, seed=2)
+    same, _ = point_token_models(P, P_in, same=True)
+    out, tr = orc.forecast_speculative(same, same, s, 40, H, K, 1.0, 3)
+    np.testing.assert_allclose(out, orc.forecast_target_only(same, s, 40, H), atol=1e-10)
+    assert all(r.n_accept == K for recs in tr.rounds for r in recs)
+    a, tra = orc.forecast_speculative(target, draft, s, 40, H, K, 2.0, 9, use_cache=True)
+    b, trb = orc.forecast_speculative(target, draft, s, 40, H, K, 2.0, 9, use_cache=False)
+    np.testing.assert_allclose(a, b, atol=1e-10)
+    T = -(-H // P)
+    for recs in tra.rounds:
+        assert all(1 <= r.L <= K + 1 for r in recs) and sum(r.committed for r in recs) == T
+    np.testing.assert_allclose(orc.forecast_target_only(target, s, 40, H, use_cache=True),
+                               orc.forecast_target_only(target, s, 40, H, use_cache=False), atol=1e-10)
+
+
 @pytest.mark.parametrize("K,tau,H", [(1, 1.0, 40), (2, 2.0, 44), (4, 1.5, 64), (8, 3.0, 50)])
 def test_round_yield_and_total(K, tau, H):
     target, draft = tiny_models()

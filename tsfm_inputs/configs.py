@@ -47,14 +47,20 @@ class Workload:
     tau_sweep: Tuple[float, ...] = ()
     eps_sweep: Tuple[float, ...] = ()
     draft_eps: float = 0.0          # perturbation size for "perturbed" drafts
+    patch_in: int = 0               # steps per input token; 0 = patch_len (patch tokens)
     weight_seed: int = 0
     perturb_seed: int = 1
     series_seed: int = 1000
     forecast_seed: int = 2021
 
     @property
+    def token_len(self) -> int:
+        """P_in: steps per input token."""
+        return self.patch_in or self.patch_len
+
+    @property
     def n_ctx_tokens(self) -> int:
-        return self.ctx_len // self.patch_len
+        return self.ctx_len // self.token_len
 
     @property
     def n_patches(self) -> int:
@@ -81,6 +87,13 @@ WORKLOADS = {
     "C4": Workload("C4", 64, 8192, 32, 2048, 8, 1.0, "bf16",
                    Arch(24, 1280, 20, 5120), Arch(4, 384, 6, 1536), "separate", "c4",
                    series_seed=1004),
+    # The point-token family of the paper's appendix B (its Time-MoE table: input patch 1, a horizon
+    # head of 64 steps, K = 3, bf16, a draft of about a quarter of the target's size): tokens are
+    # single points, a committed patch is 64 of them.  Context, horizon and model sizes are scaled
+    # down from the table's 3072 / 1536 / 453 M so that the oracle decodes a series in seconds.
+    "C5": Workload("C5", 16, 768, 64, 384, 3, 1.0, "bf16",
+                   Arch(6, 512, 8, 2048), Arch(2, 256, 4, 1024), "separate", "c1",
+                   patch_in=1, series_seed=1005),
 }
 
 

@@ -39,20 +39,21 @@ def tensor_names(n_layers: int) -> List[str]:
     return names
 
 
-def _shape(name: str, arch: Arch, patch_len: int):
+def _shape(name: str, arch: Arch, patch_len: int, patch_in: int = 0):
     d, f, p = arch.d_model, arch.d_ff, patch_len
     t = name.split(".")[-1]
-    return {"W_emb": (d, p), "g1": (d,), "g2": (d,), "g_f": (d,),
+    return {"W_emb": (d, patch_in or p), "g1": (d,), "g2": (d,), "g_f": (d,),
             "Wq": (d, d), "Wk": (d, d), "Wv": (d, d), "Wo": (d, d),
             "W1": (f, d), "W2": (d, f), "W_head": (p, d)}[t]
 
 
-def make_model(arch: Arch, patch_len: int, seed: int, dtype: str, stream: int = 0) -> Weights:
-    """Xavier-normal weights; ``stream`` separates target (0) and draft (1) draws."""
+def make_model(arch: Arch, patch_len: int, seed: int, dtype: str, stream: int = 0, patch_in: int = 0) -> Weights:
+    """Xavier-normal weights; ``stream`` separates target (0) and draft (1) draws.  ``patch_in``
+    (0 = patch_len) is the length of an input token: the embedding is [d, patch_in]."""
     rng = np.random.default_rng([int(seed), int(stream), 0x7511])
     w: Weights = {}
     for name in tensor_names(arch.n_layers):
-        shape = _shape(name, arch, patch_len)
+        shape = _shape(name, arch, patch_len, patch_in)
         if len(shape) == 1:
             w[name] = np.ones(shape, dtype=np.float32)
             continue
@@ -95,11 +96,11 @@ def perturbed_draft(target: Weights, n_layers: int, eps: float, seed: int, dtype
 
 def build_models(wl: Workload):
     """(target weights, draft weights) for a workload."""
-    tgt = make_model(wl.target, wl.patch_len, wl.weight_seed, wl.dtype, stream=0)
+    tgt = make_model(wl.target, wl.patch_len, wl.weight_seed, wl.dtype, stream=0, patch_in=wl.patch_in)
     if wl.draft_mode == "layer_skip":
         drf = layer_skip_draft(tgt, wl.draft.n_layers)
     elif wl.draft_mode == "perturbed":
         drf = perturbed_draft(tgt, wl.draft.n_layers, wl.draft_eps, wl.perturb_seed, wl.dtype)
     else:
-        drf = make_model(wl.draft, wl.patch_len, wl.weight_seed, wl.dtype, stream=1)
+        drf = make_model(wl.draft, wl.patch_len, wl.weight_seed, wl.dtype, stream=1, patch_in=wl.patch_in)
     return tgt, drf
