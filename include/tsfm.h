@@ -66,6 +66,19 @@ extern "C" {
 #define TSFM_EXEC_NO_PDL  2       /* flag, may be OR-ed in: launch without programmatic dependent launch,
                                    i.e. every kernel starts only after its predecessor has finished   */
 
+#define TSFM_EXEC_NO_COMPACT 4     /* flag, may be OR-ed in: every round runs its passes over all B series, finished
+                                   or not (by default only the series that still have patches to commit take
+                                   part: the batch desynchronises as per-series first rejections differ, the
+                                   paper's "Batch Size" sensitivity paragraph); same results either way  */
+
+#define TSFM_EXEC_CHECK_BOUNDS 8   /* flag, may be OR-ed in: bounds-checking mode.  Every device buffer of the handle
+                                   gets guard bytes behind it, every (layer, series, head) block of the KV
+                                   caches and every series' history one spare token that nothing may write;
+                                   after each call a kernel inspects them all, and a damaged guard makes a
+                                   call that reads its status (stats != NULL) return TSFM_ERR_INTERNAL with
+                                   the buffer's name in tsfm_last_cuda_error().  Costs memory and a launch
+                                   per call; for test runs                                               */
+
 #define TSFM_MAX_K 32           /* hard upper bound on the block size K                             */
 
 typedef struct tsfm_spec tsfm_spec;   /* opaque decoder handle */
@@ -84,24 +97,30 @@ typedef struct {
   int32_t dtype;                /* TSFM_F32 | TSFM_BF16                                          */
   int32_t draft_mode;           /* TSFM_DRAFT_*                                                  */
   int32_t max_batch;            /* capacity: series per call                                     */
-  int32_t max_ctx_tokens;       /* capacity: context patches N = ctx_len / P                     */
+  int32_t max_ctx_tokens;       /* capacity: context tokens N = ctx_len / P_in (>= 2 patches' worth) */
   int32_t max_horizon_patches;  /* capacity: T = ceil(H / P)                                     */
   int32_t max_K;                /* capacity: block size, <= TSFM_MAX_K                           */
   int32_t gemm_backend;         /* TSFM_GEMM_*                                                   */
   float   rms_eps;              /* RMSNorm epsilon (1e-6)                                        */
   float   norm_eps;             /* instance-norm variance epsilon (1e-5)                         */
   float   rope_base;            /* RoPE base (1e4)                                               */
-  int32_t exec_mode;            /* TSFM_EXEC_GRAPH or TSFM_EXEC_STREAM, optionally | TSFM_EXEC_NO_PDL */
+  int32_t exec_mode;            /* TSFM_EXEC_GRAPH or TSFM_EXEC_STREAM, optionally | TSFM_EXEC_NO_PDL | TSFM_EXEC_NO_COMPACT */
+  int32_t patch_in;             /* P_in: steps per INPUT token; 0 = patch_len (a token is a whole patch).
+                                   Must divide patch_len.  With P_in < P (the point-token family of the
+                                   paper's appendix B: P_in = 1, a horizon head of P steps) a committed
+                                   patch is P / P_in tokens, the embedding is [d, P_in], and the target's
+                                   prediction after prefix i is read at token N - 1 + i (P / P_in) of the
+                                   verification pass (appendix B, "Per-Family Boundary Indexing")        */
   void   *stream;               /* cudaStream_t, borrowed for the handle's lifetime              */
 } tsfm_cfg;
 
 /* A weight blob in DEVICE memory, borrowed for the handle's lifetime (never copied, never
  * written).  Layout: a 256-byte header of int32 words
  *     [0] magic 0x4D465354 ("TSFM")  [1] version 1  [2] dtype  [3] n_layers  [4] d_model
- *     [5] n_heads  [6] d_ff  [7] patch_len            (remaining words zero)
+ *     [5] n_heads  [6] d_ff  [7] patch_len  [8] patch_in (0 = patch_len)   (remaining words zero)
  * followed by the tensors, each starting on a 256-byte boundary, every linear stored
  * [out_features, in_features] row-major in `dtype`, gains in fp32, in this order:
- *     W_emb[d,P];  per layer: g1[d], Wq[d,d], Wk[d,d], Wv[d,d], Wo[d,d], g2[d],
+ *     W_emb[d,P_in];  per layer: g1[d], Wq[d,d], Wk[d,d], Wv[d,d], Wo[d,d], g2[d],
  *     W1[d_ff,d], W2[d,d_ff];  g_f[d];  W_head[P,d].
  * tsfm_weights_bytes() gives the total size. */
 typedef struct {
@@ -136,9 +155,15 @@ size_t tsfm_weights_bytes(const tsfm_arch *arch, int32_t patch_len, int32_t dtyp
 size_t tsfm_weights_offset(const tsfm_arch *arch, int32_t patch_len, int32_t dtype,
                            int32_t layer, const char *name);
 
+/* The same two queries for a model whose input tokens are patch_in steps long (0 = patch_len):
+ * only W_emb [d, patch_in] differs.  Return 0 if patch_in does not divide patch_len. */
+size_t tsfm_weights_bytes_io(const tsfm_arch *arch, int32_t patch_in, int32_t patch_len, int32_t dtype);
+size_t tsfm_weights_offset_io(const tsfm_arch *arch, int32_t patch_in, int32_t patch_len, int32_t dtype,
+                              int32_t layer, const char *name);
+
 /* Create a decoder (Algorithm 1's inputs "target p, draft q").  Validates shapes and blob
  * headers, allocates both KV caches ([layer][series][head][token][d_head], capacity
- * max_ctx_tokens + max_horizon_patches + max_K + 1 tokens per series), activation workspaces
+ * max_ctx_tokens + (max_horizon_patches + max_K + 1) * (P / P_in) tokens per series), activation workspaces
  * and TMA descriptors.  target_w, cfg, out_h: host pointers to structs; blobs: dev.
  * draft_w may be NULL only with TSFM_DRAFT_LAYER_SKIP.  *out_h is owned by the caller and
  * released with tsfm_spec_destroy. */
@@ -149,7 +174,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w,
  *   series  dev  [B, ctx_len] fp32 row-major, raw (un-normalised) context values
  *   out     dev  [B, H] fp32 row-major, forecast in the series' own scale
  *   stats   host, nullable; when non-NULL the call synchronises the stream and fills it
- * ctx_len must be a multiple of P with at least 2 patches; T = ceil(H / P) patches are
+ * ctx_len must be a multiple of P (hence of P_in) with at least 2 patches; T = ceil(H / P) patches are
  * committed per series, the last one truncated to H on output.  Each round drafts K patches
  * with the draft model, verifies them in one causal target pass, accepts left to right with
  * uniforms Philox4x32-10(key = seed, counter = (series, round, position, 0)), commits the
@@ -228,7 +253,7 @@ int tsfm_accept_round(void *stream, const float *x, const float *mu_q, const flo
                       int32_t *done, float *commit, int32_t *n_accept, float *ell, float *log_u);
 
 /* Full causal forward of one of the handle's models over fresh sequences (positions
- * 0..n-1), for numerics checks: tokens dev [B, n, P] fp32 (already normalised), out dev
+ * 0..n-1), for numerics checks: tokens dev [B, n, P_in] fp32 (already normalised), out dev
  * [B, n, P] fp32 = next-patch mean at every position.  which: 0 target, 1 draft.
  * n <= max_ctx_tokens (TSFM_ERR_SHAPE beyond it).  Overwrites the KV cache; synchronises the stream. */
 int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t B, int32_t n,
@@ -262,6 +287,12 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C,
 #define TSFM_STATIC_GEMM_MAX_ELEMS (1 << 20)
 int tsfm_gemm_bf16_static(void *stream, const void *A, const void *W, float *C,
                           int32_t M, int32_t N, int32_t Kd);
+
+/* Bounds-checking mode only (TSFM_EXEC_CHECK_BOUNDS): *n_regions (nullable) receives the number of
+ * guard regions of the handle.  region >= 0 additionally overwrites (damage != 0) or restores
+ * (damage == 0) one byte of that guard region -- a write inside the library's own allocation --
+ * so that a test can see the checker report it.  region < 0: query only. */
+int tsfm_spec_debug_guard(tsfm_spec *h, int32_t region, int32_t damage, int32_t *n_regions);
 
 /* Per-launch timing, for roofline accounting.  While enabled, every kernel launch of the handle
  * is bracketed by two CUDA events on the handle's stream (this perturbs end-to-end time: do not

@@ -19,14 +19,14 @@ TSFM_ERR_ARG, TSFM_ERR_SHAPE, TSFM_ERR_ARCH, TSFM_ERR_CUDA, TSFM_ERR_TIMEOUT, TS
 TSFM_F32, TSFM_BF16 = 0, 1
 TSFM_DRAFT_SEPARATE, TSFM_DRAFT_LAYER_SKIP = 0, 1
 TSFM_GEMM_AUTO, TSFM_GEMM_SIMT = 0, 1
-TSFM_EXEC_GRAPH, TSFM_EXEC_STREAM, TSFM_EXEC_NO_PDL = 0, 1, 2
+TSFM_EXEC_GRAPH, TSFM_EXEC_STREAM, TSFM_EXEC_NO_PDL, TSFM_EXEC_NO_COMPACT, TSFM_EXEC_CHECK_BOUNDS = 0, 1, 2, 4, 8
 TSFM_MAX_K = 32
 
 EXPORTS = [
-    "tsfm_weights_bytes", "tsfm_weights_offset", "tsfm_spec_create", "tsfm_spec_forecast", "tsfm_spec_forecast_variant",
+    "tsfm_weights_bytes", "tsfm_weights_offset", "tsfm_weights_bytes_io", "tsfm_weights_offset_io", "tsfm_spec_create", "tsfm_spec_forecast", "tsfm_spec_forecast_variant",
     "tsfm_target_only_forecast", "tsfm_draft_only_forecast", "tsfm_spec_forecast_host", "tsfm_target_only_forecast_host",
     "tsfm_spec_last_trace", "tsfm_accept_round", "tsfm_model_forward", "tsfm_gemm_bf16", "tsfm_gemm_bf16_static",
-    "tsfm_spec_set_profiling", "tsfm_spec_kernel_profile", "tsfm_advise_block_size", "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
+    "tsfm_spec_debug_guard", "tsfm_spec_set_profiling", "tsfm_spec_kernel_profile", "tsfm_advise_block_size", "tsfm_spec_destroy", "tsfm_launch_count", "tsfm_strerror", "tsfm_last_cuda_error",
 ]
 
 
@@ -40,7 +40,7 @@ class tsfm_cfg(C.Structure):
                 ("max_batch", C.c_int32), ("max_ctx_tokens", C.c_int32),
                 ("max_horizon_patches", C.c_int32), ("max_K", C.c_int32), ("gemm_backend", C.c_int32),
                 ("rms_eps", C.c_float), ("norm_eps", C.c_float), ("rope_base", C.c_float),
-                ("exec_mode", C.c_int32), ("stream", C.c_void_p)]
+                ("exec_mode", C.c_int32), ("patch_in", C.c_int32), ("stream", C.c_void_p)]
 
 
 class tsfm_weights(C.Structure):
@@ -86,6 +86,10 @@ def _load() -> C.CDLL:
     lib.tsfm_weights_bytes.argtypes = [C.POINTER(tsfm_arch), i32, i32]
     lib.tsfm_weights_offset.restype = sz
     lib.tsfm_weights_offset.argtypes = [C.POINTER(tsfm_arch), i32, i32, i32, C.c_char_p]
+    lib.tsfm_weights_bytes_io.restype = sz
+    lib.tsfm_weights_bytes_io.argtypes = [C.POINTER(tsfm_arch), i32, i32, i32]
+    lib.tsfm_weights_offset_io.restype = sz
+    lib.tsfm_weights_offset_io.argtypes = [C.POINTER(tsfm_arch), i32, i32, i32, i32, C.c_char_p]
     lib.tsfm_spec_create.restype = C.c_int
     lib.tsfm_spec_create.argtypes = [C.POINTER(tsfm_weights), C.POINTER(tsfm_weights), C.POINTER(tsfm_cfg), C.POINTER(vp)]
     for name in ("tsfm_spec_forecast", "tsfm_spec_forecast_host"):
@@ -109,6 +113,8 @@ def _load() -> C.CDLL:
     lib.tsfm_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     lib.tsfm_gemm_bf16_static.restype = C.c_int
     lib.tsfm_gemm_bf16_static.argtypes = [vp, vp, vp, vp, i32, i32, i32]
+    lib.tsfm_spec_debug_guard.restype = C.c_int
+    lib.tsfm_spec_debug_guard.argtypes = [vp, i32, i32, C.POINTER(i32)]
     lib.tsfm_spec_set_profiling.restype = C.c_int
     lib.tsfm_spec_set_profiling.argtypes = [vp, i32]
     lib.tsfm_spec_kernel_profile.restype = C.c_int
@@ -133,7 +139,7 @@ class TsfmError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
         msg = lib.tsfm_strerror(code).decode()
-        if code == TSFM_ERR_CUDA:
+        if code in (TSFM_ERR_CUDA, TSFM_ERR_INTERNAL):
             msg += " (" + lib.tsfm_last_cuda_error().decode() + ")"
         super().__init__(f"{where}: {msg} [{code}]")
 
@@ -171,18 +177,29 @@ def tsfm_weights_offset(arch, patch_len: int, dtype: str, layer: int, name: str)
     return int(lib.tsfm_weights_offset(C.byref(a), patch_len, _dtype_code(dtype), layer, name.encode()))
 
 
-def pack_weights(weights: Dict[str, np.ndarray], arch, patch_len: int, dtype: str) -> np.ndarray:
+def tsfm_weights_bytes_io(arch, patch_in: int, patch_len: int, dtype: str) -> int:
+    a = _arch(arch)
+    return int(lib.tsfm_weights_bytes_io(C.byref(a), patch_in, patch_len, _dtype_code(dtype)))
+
+
+def tsfm_weights_offset_io(arch, patch_in: int, patch_len: int, dtype: str, layer: int, name: str) -> int:
+    a = _arch(arch)
+    return int(lib.tsfm_weights_offset_io(C.byref(a), patch_in, patch_len, _dtype_code(dtype), layer, name.encode()))
+
+
+def pack_weights(weights: Dict[str, np.ndarray], arch, patch_len: int, dtype: str, patch_in: int = 0) -> np.ndarray:
     """Serialise a name -> float32 array dict into the blob layout of include/tsfm.h (host bytes)."""
-    total = tsfm_weights_bytes(arch, patch_len, dtype)
+    total = tsfm_weights_bytes_io(arch, patch_in, patch_len, dtype)
     if total == 0:
         raise ValueError("unsupported model shape")
     blob = np.zeros(total, dtype=np.uint8)
-    hdr = blob[:32].view(np.int32)
-    hdr[:] = [0x4D465354, 1, _dtype_code(dtype), arch.n_layers, arch.d_model, arch.n_heads, arch.d_ff, patch_len]
+    hdr = blob[:36].view(np.int32)
+    hdr[:] = [0x4D465354, 1, _dtype_code(dtype), arch.n_layers, arch.d_model, arch.n_heads, arch.d_ff, patch_len,
+              patch_in]
     for name, w in weights.items():
         parts = name.split(".")
         layer, short = (int(parts[1]), parts[2]) if parts[0] == "layers" else (-1, name)
-        off = tsfm_weights_offset(arch, patch_len, dtype, layer, short)
+        off = tsfm_weights_offset_io(arch, patch_in, patch_len, dtype, layer, short)
         if off == 0:
             raise ValueError(f"no slot for tensor {name}")
         w32 = np.ascontiguousarray(w, dtype=np.float32)
@@ -284,6 +301,13 @@ def tsfm_gemm_bf16_static(stream, A, W, Cout, M: int, N: int, Kd: int) -> None:
     _check(code, "tsfm_gemm_bf16_static")
 
 
+def tsfm_spec_debug_guard(h, region: int = -1, damage: bool = False) -> int:
+    """Bounds-checking mode: number of guard regions; region >= 0 damages / restores one byte of it."""
+    n = C.c_int32(0)
+    _check(lib.tsfm_spec_debug_guard(h, region, int(bool(damage)), C.byref(n)), "tsfm_spec_debug_guard")
+    return n.value
+
+
 def tsfm_spec_set_profiling(h, enable: bool) -> None:
     _check(lib.tsfm_spec_set_profiling(h, int(bool(enable))), "tsfm_spec_set_profiling")
 
@@ -314,19 +338,21 @@ class SpecDecoder:
 
     def __init__(self, target_w, draft_w, target_arch, draft_arch, patch_len: int, dtype: str,
                  draft_mode: str, max_batch: int, max_ctx_tokens: int, max_horizon_patches: int, max_K: int,
-                 gemm_backend: int = TSFM_GEMM_AUTO, exec_mode: int = TSFM_EXEC_GRAPH, device: str = "cuda:0"):
+                 gemm_backend: int = TSFM_GEMM_AUTO, exec_mode: int = TSFM_EXEC_GRAPH, device: str = "cuda:0",
+                 patch_in: int = 0):
         import torch
         self.torch = torch
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         self.patch_len, self.dtype = patch_len, dtype
-        self.target_blob = torch.from_numpy(pack_weights(target_w, target_arch, patch_len, dtype)).to(self.device)
+        self.target_blob = torch.from_numpy(pack_weights(target_w, target_arch, patch_len, dtype, patch_in)).to(self.device)
         self.draft_blob = None
         if draft_mode != "layer_skip":
-            self.draft_blob = torch.from_numpy(pack_weights(draft_w, draft_arch, patch_len, dtype)).to(self.device)
+            self.draft_blob = torch.from_numpy(pack_weights(draft_w, draft_arch, patch_len, dtype, patch_in)).to(self.device)
         cfg = tsfm_cfg()
         cfg.target, cfg.draft = _arch(target_arch), _arch(draft_arch)
         cfg.patch_len, cfg.dtype = patch_len, _dtype_code(dtype)
+        cfg.patch_in = patch_in
         cfg.draft_mode = TSFM_DRAFT_LAYER_SKIP if draft_mode == "layer_skip" else TSFM_DRAFT_SEPARATE
         cfg.max_batch, cfg.max_ctx_tokens = max_batch, max_ctx_tokens
         cfg.max_horizon_patches, cfg.max_K = max_horizon_patches, max_K
@@ -343,7 +369,7 @@ class SpecDecoder:
         ks = max(wl.K_sweep) if wl.K_sweep else wl.K
         return cls(target_w, draft_w, wl.target, wl.draft, wl.patch_len, wl.dtype,
                    "layer_skip" if wl.draft_mode == "layer_skip" else "separate",
-                   batch or wl.batch, wl.n_ctx_tokens, wl.n_patches, max_K or ks, **kw)
+                   batch or wl.batch, wl.n_ctx_tokens, wl.n_patches, max_K or ks, patch_in=wl.patch_in, **kw)
 
     def close(self):
         if getattr(self, "h", None):
@@ -389,7 +415,7 @@ class SpecDecoder:
         return tsfm_spec_last_trace(self.h, B, K, self.max_T)
 
     def model_forward(self, which: int, tokens):
-        B, n, P = tokens.shape
-        out = self.torch.empty_like(tokens)
+        B, n, _ = tokens.shape                                # [B, n, P_in]
+        out = self.torch.empty((B, n, self.patch_len), dtype=tokens.dtype, device=tokens.device)
         tsfm_model_forward(self.h, which, tokens, B, n, out)
         return out

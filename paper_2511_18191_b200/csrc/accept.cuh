@@ -80,12 +80,38 @@ struct AcceptArgs {
 };
 
 // Closes a round: accumulates the phase clocks, advances the round counter, adds the round's
-// kernel launches to the device-side launch counter and, inside a captured graph, tells the
-// WHILE node whether another round is needed.  One thread.
-__global__ void round_end_kernel(DevState *st, const int *unfinished, int T,
-                                 cudaGraphConditionalHandle handle, int use_handle,
-                                 const int *body_launches, unsigned long long *launch_ctr) {
+// kernel launches to the device-side launch counter, lists the series that still have patches
+// to commit (ascending, for the next round's compacted passes) and, inside a captured graph, tells
+// the WHILE node whether another round is needed.  One CTA of 256 threads.
+__global__ void __launch_bounds__(256)
+round_end_kernel(DevState *st, const int *unfinished, int T, cudaGraphConditionalHandle handle, int use_handle,
+                 const int *body_launches, unsigned long long *launch_ctr, const int *__restrict__ done, int B,
+                 int *__restrict__ live, int *__restrict__ n_live) {
+  __shared__ int warp_count[8];
+  __shared__ int base;
   pdl_sync();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (int b0 = 0; b0 < B; b0 += 256) {             // ordered compaction, 256 series at a time
+    const int b = b0 + threadIdx.x;
+    const bool alive = b < B && done[b] < T;
+    const unsigned m = __ballot_sync(0xffffffffu, alive);
+    if (lane == 0) warp_count[w] = __popc(m);
+    __syncthreads();
+    int off = base;
+    for (int i = 0; i < w; ++i) off += warp_count[i];
+    if (alive) live[off + __popc(m & ((1u << lane) - 1u))] = b;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int t = 0;
+      for (int i = 0; i < 8; ++i) t += warp_count[i];
+      base += t;
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x != 0) return;
+  *n_live = base;
   const int r = st->round;
   const unsigned long long now = globaltimer_ns();
   if (r == 0) st->ns_prefill = st->t_phase[0] - st->t_call;

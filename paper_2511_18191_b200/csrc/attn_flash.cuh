@@ -78,19 +78,21 @@ attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__re
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int gr = lane >> 2, q4 = lane & 3;                     // fragment row group, column pair
   const int d = n_heads * DH;
-  int h = blockIdx.x, b = blockIdx.y;
+  int h = blockIdx.x, slot = blockIdx.y;
   if (mode == FLASH_WARP) {
     const int pair = blockIdx.x * 4 + w;
     if (pair >= n_pairs) return;                               // no block-wide barrier in this mode
-    b = pair / n_heads;
+    slot = pair / n_heads;
     h = pair % n_heads;
   }
   const int warp_bytes = single ? 2 * S_TILE : G::WARP_BYTES;   // shared memory of one warp
   unsigned char *ring = flash_smem + (size_t)w * warp_bytes;
   const uint32_t ring32 = (uint32_t)__cvta_generic_to_shared(ring);
   pdl_sync();
+  if (slot_dead(g, slot)) return;                              // per warp (FLASH_WARP) or per CTA: no barrier is pending
+  const int b = series_of(g, slot);
   const int p0 = pos0_of(g, b);
-  const size_t row0 = (size_t)b * g.q_len;
+  const size_t row0 = (size_t)slot * g.q_len;
   bf16 *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
   bf16 *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
 

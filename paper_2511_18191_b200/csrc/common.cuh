@@ -9,7 +9,19 @@ namespace tsfm {
 typedef __nv_bfloat16 bf16;
 
 // Device status codes written by kernels whose bounded waits expire (0 = fine).
-enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPILOGUE = 3 };
+// From DEV_GUARD_BASE on: guard region (code - DEV_GUARD_BASE) behind a buffer was overwritten.
+enum : int { DEV_OK = 0, DEV_TIMEOUT_TMA = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPILOGUE = 3, DEV_GUARD_BASE = 16 };
+
+// Guard regions of the bounds-checking mode: n_blocks runs of `len` bytes, `stride` bytes apart, that
+// were filled with GUARD_BYTE when the handle was made and that no kernel may ever write (the bytes
+// behind an allocation; the spare last row of every (layer, series, head) block of a KV cache; the
+// spare last token of every series' history).
+constexpr unsigned char GUARD_BYTE = 0xA5;
+struct GuardRegion {
+  const unsigned char *base;
+  unsigned long long stride;
+  unsigned int n_blocks, len;
+};
 
 // Per-forecast state in device memory.  The first block holds the call's parameters (written
 // by the host before the work is enqueued, so that a captured graph can be replayed with new

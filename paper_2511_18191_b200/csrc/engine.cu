@@ -55,6 +55,9 @@ bool arch_ok(const tsfm_arch &a, int P) {
   if (P < 16 || P > 256 || P % 16) return false;
   return true;
 }
+// Input token length P_in (0 = P): it divides the patch length P (a patch is P / P_in tokens).
+inline int token_len(int P_in, int P) { return P_in > 0 ? P_in : P; }
+bool io_ok(int P_in, int P) { return P_in >= 0 && P % token_len(P_in, P) == 0; }
 
 // Offsets of the tensors of one model inside its blob (canonical order, 256-byte aligned).
 struct BlobLayout {
@@ -63,12 +66,12 @@ struct BlobLayout {
   std::vector<L> layers;
 };
 
-BlobLayout blob_layout(const tsfm_arch &a, int P, int dtype) {
+BlobLayout blob_layout(const tsfm_arch &a, int P, int dtype, int P_in = 0) {
   BlobLayout b;
   const size_t e = elt_bytes(dtype), d = a.d_model, f = a.d_ff;
   size_t off = 256;
   auto take = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return o; };
-  b.W_emb = take(d * P * e);
+  b.W_emb = take(d * token_len(P_in, P) * e);
   for (int l = 0; l < a.n_layers; ++l) {
     BlobLayout::L x;
     x.g1 = take(d * 4);
@@ -126,7 +129,8 @@ struct tsfm_spec {
   unsigned long long *dev_launches = nullptr;   // launches made by replayed round bodies
   int *dev_body_launches = nullptr;             // [kMaxGraphs] launches of one round body, per cached graph
   DevState *st = nullptr;
-  int cap = 0;
+  int P_in = 0, tpp = 1;                 // steps per input token; tokens per patch (P / P_in)
+  int cap = 0;                           // token capacity per series of history and KV caches
   bool use_tc = false;
   bool pdl = false;                      // launches carry the programmatic-serialization attribute
   ModelDev tgt, drf;
@@ -138,6 +142,8 @@ struct tsfm_spec {
   float *hist = nullptr, *vout = nullptr, *mean = nullptr, *sd = nullptr;
   float *muq = nullptr;                  // [B][max_K][P] draft means of the round (sampled proposals)
   int *done = nullptr;
+  int *live = nullptr, *n_live = nullptr;   // [B] slot -> unfinished series, and their number (round_end_kernel)
+  bool compact = true;                   // rounds run over the unfinished series only
   AcceptCounters *ctr = nullptr;
   int *unfinished = nullptr;             // [max_T + 1]
   int *h_unfinished = nullptr;           // pinned
@@ -155,6 +161,11 @@ struct tsfm_spec {
   size_t prof_pool_used = 0;
   std::vector<cudaEvent_t> ev;
   std::vector<void *> owned;
+  // bounds-checking mode (TSFM_EXEC_CHECK_BOUNDS): guard regions, their names, the device copy
+  bool check = false;
+  std::vector<GuardRegion> guards;
+  std::vector<std::string> guard_names;
+  GuardRegion *dev_guards = nullptr;
 };
 
 namespace {
@@ -194,22 +205,36 @@ struct KTimer {
   }
 };
 
-template <typename T>
-int dev_alloc(tsfm_spec *h, T **p, size_t count) {
-  void *q = nullptr;
-  CU_TRY(cudaMalloc(&q, count * sizeof(T) ? count * sizeof(T) : 256));
-  h->owned.push_back(q);
-  *p = (T *)q;
+constexpr size_t kGuardTail = 256;       // guard bytes behind every allocation in bounds-checking mode
+
+// Registers (and fills) a guard region: n_blocks runs of len bytes, stride bytes apart.
+int add_guard(tsfm_spec *h, const char *name, void *base, size_t stride, size_t n_blocks, size_t len) {
+  if (n_blocks == 1) CU_TRY(cudaMemsetAsync(base, GUARD_BYTE, len, h->stream));
+  else CU_TRY(cudaMemset2DAsync(base, stride, GUARD_BYTE, len, n_blocks, h->stream));
+  h->guards.push_back(GuardRegion{(const unsigned char *)base, (unsigned long long)stride, (unsigned)n_blocks, (unsigned)len});
+  h->guard_names.push_back(name);
   return TSFM_OK;
 }
 
-int read_header(const tsfm_weights *w, const tsfm_arch &a, int P, int dtype, cudaStream_t s) {
+template <typename T>
+int dev_alloc(tsfm_spec *h, T **p, size_t count, const char *name = "buffer") {
+  void *q = nullptr;
+  const size_t bytes = count * sizeof(T) ? count * sizeof(T) : 256;
+  CU_TRY(cudaMalloc(&q, bytes + (h->check ? kGuardTail : 0)));
+  h->owned.push_back(q);
+  *p = (T *)q;
+  if (h->check) return add_guard(h, name, (char *)q + bytes, 0, 1, kGuardTail);
+  return TSFM_OK;
+}
+
+int read_header(const tsfm_weights *w, const tsfm_arch &a, int P, int P_in, int dtype, cudaStream_t s) {
   if (!w || !w->blob) return TSFM_ERR_ARG;
-  int32_t hd[8];
+  int32_t hd[9];
   CU_TRY(cudaMemcpyAsync(hd, w->blob, sizeof(hd), cudaMemcpyDeviceToHost, s));
   CU_TRY(cudaStreamSynchronize(s));
   if (hd[0] != 0x4D465354 || hd[1] != 1 || hd[2] != dtype || hd[3] < a.n_layers ||
-      hd[4] != a.d_model || hd[5] != a.n_heads || hd[6] != a.d_ff || hd[7] != P)
+      hd[4] != a.d_model || hd[5] != a.n_heads || hd[6] != a.d_ff || hd[7] != P ||
+      token_len(hd[8], P) != token_len(P_in, P))
     return TSFM_ERR_SHAPE;
   return TSFM_OK;
 }
@@ -217,8 +242,8 @@ int read_header(const tsfm_weights *w, const tsfm_arch &a, int P, int dtype, cud
 // Wire a model's tensor pointers.  `blob_arch` is the shape the blob was written for (a
 // layer-skip draft reads the first layers of the target's blob).
 void wire_model(ModelDev &m, const tsfm_arch &arch, const tsfm_arch &blob_arch, const void *blob,
-                int P, int dtype) {
-  const BlobLayout lay = blob_layout(blob_arch, P, dtype);
+                int P, int dtype, int P_in) {
+  const BlobLayout lay = blob_layout(blob_arch, P, dtype, P_in);
   const char *base = (const char *)blob;
   m.arch = arch;
   m.dh = arch.d_model / arch.n_heads;
@@ -246,7 +271,7 @@ int make_rope(tsfm_spec *h, ModelDev &m) {
       const double theta = std::pow((double)h->cfg.rope_base, -2.0 * i / m.dh);
       t[(size_t)p * half + i] = make_float2((float)std::cos(p * theta), (float)std::sin(p * theta));
     }
-  if (int rc = dev_alloc(h, &m.rope, t.size())) return rc;
+  if (int rc = dev_alloc(h, &m.rope, t.size(), "rope")) return rc;
   CU_TRY(cudaMemcpyAsync(m.rope, t.data(), t.size() * sizeof(float2), cudaMemcpyHostToDevice, h->stream));
   CU_TRY(cudaStreamSynchronize(h->stream));
   return TSFM_OK;
@@ -403,14 +428,14 @@ void launch_gemm_simt(cudaStream_t s, bool pdl, const T *A, const T *W, void *C,
 // C (op)= A . W^T through the tensor-core kernel when a plan exists, else the FMA kernel.
 template <typename T>
 void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C, int M, int N,
-          int K, int epi, const SkNorm *norm = nullptr) {
+          int K, int epi, const SkNorm *norm = nullptr, LiveRows lr = LiveRows{nullptr, 0}) {
   const double e = sizeof(T);
   const double out_b = (epi == EPI_F32 || epi == EPI_ATOMIC) ? 4.0 : epi == EPI_RESID ? 8.0 : e;
   const double bytes = ((double)N * K + (double)M * K) * e + (double)M * N * out_b;
   const double flops = 2.0 * M * N * K;
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
     KTimer kt(h, M <= 512 ? KC_GEMM_TC_SMALL : M < 4096 ? KC_GEMM_TC_MID : KC_GEMM_TC_LARGE, bytes, flops);
-    if (gemm_sk_launch(h->ls, h->pdl, *plan, C, M, epi, h->dev_status, norm)) {
+    if (gemm_sk_launch(h->ls, h->pdl, *plan, C, M, epi, h->dev_status, norm, lr)) {
       LAUNCHED();
     } else if (h->enqueue_err == TSFM_OK) {
       // No silent fallback: the FMA kernel knows nothing of a folded norm, and a pass that mixes
@@ -487,7 +512,7 @@ struct DraftStep { int k_pos = -1, K = 0; };
 template <typename T>
 void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout,
               unsigned long long *stamp, DraftStep ds) {
-  const int M = B * g.q_len, d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len;
+  const int M = B * g.q_len, d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len, Pi = h->P_in;
   cudaStream_t s = h->ls;
   const float eps = h->cfg.rms_eps;
   // On the tensor-core path the RMSNorms are folded into the contractions around them (SkNorm):
@@ -497,13 +522,14 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   // large tiles the epilogue is the bottleneck and the separate RMSNorm kernel is the cheaper way.)
   const bool fold = sizeof(T) == 2 && h->use_tc && m.layers[0].tc_qkv.valid && M <= 512;
   const int L = m.arch.n_layers;
+  const LiveRows lr{g.n_live, g.q_len};
   {
-    KTimer kt(h, KC_EMBED, (double)M * P * 4 + (double)d * P * sizeof(T) + (double)M * d * 4, 2.0 * M * P * d);
+    KTimer kt(h, KC_EMBED, (double)M * Pi * 4 + (double)d * Pi * sizeof(T) + (double)M * d * 4, 2.0 * M * Pi * d);
     if (!fold && M >= kManyRows)
-      launch_ex(s, h->pdl, embed_rows_kernel<T>, dim3((M + 7) / 8, (d + 127) / 128), dim3(128), 8 * P * sizeof(float),
-                h->hist, g, M, P, d, (const T *)m.W_emb, h->x, stamp);
+      launch_ex(s, h->pdl, embed_rows_kernel<T>, dim3((M + 7) / 8, (d + 127) / 128), dim3(128), 8 * Pi * sizeof(float),
+                h->hist, g, M, Pi, d, (const T *)m.W_emb, h->x, stamp);
     else
-      launch_ex(s, h->pdl, embed_kernel<T>, dim3(M, (d + 127) / 128), dim3(128), P * sizeof(float), h->hist, g, P, d,
+      launch_ex(s, h->pdl, embed_kernel<T>, dim3(M, (d + 127) / 128), dim3(128), Pi * sizeof(float), h->hist, g, Pi, d,
                 (const T *)m.W_emb, h->x, stamp, fold ? m.layers[0].g1 : (const float *)nullptr,
                 fold ? (T *)h->a : (T *)nullptr, fold ? h->ssq : (float *)nullptr);
   }
@@ -517,9 +543,9 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     LayerDev &ly = m.layers[l];
     if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g1, M, d, eps, (T *)h->a);
+      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g1, M, d, eps, (T *)h->a, lr);
     }
-    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr);
+    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr, lr);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
     else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
     else launch_attn<T, 128>(h, m, l, B, g);
@@ -528,29 +554,31 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     produce.ssq_out = h->ssq;
     produce.a_out = (bf16 *)h->a;
     produce.gain = ly.g2;
-    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, fold ? &produce : nullptr);
+    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, fold ? &produce : nullptr, lr);
     if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g2, M, d, eps, (T *)h->a);
+      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g2, M, d, eps, (T *)h->a, lr);
     }
-    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, fold ? &consume : nullptr);
+    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, fold ? &consume : nullptr, lr);
     produce.gain = l + 1 < L ? m.layers[l + 1].g1 : nullptr;
     if (l + 1 == L) produce.a_out = nullptr, produce.ssq_out = nullptr;   // the head kernel norms the final rows itself
-    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID, fold && l + 1 < L ? &produce : nullptr);
+    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID, fold && l + 1 < L ? &produce : nullptr, lr);
   }
-  const double rows = head_mode == HEAD_LAST_TO_HIST ? B : M;
+  const int Mb = B * (g.q_len / g.head_step);          // boundary rows the head reads (verification)
+  const double rows = head_mode == HEAD_LAST_TO_HIST ? B : Mb;
   KTimer kt(h, head_mode == HEAD_NONE ? -1 : KC_HEAD, rows * d * 4 + (double)P * d * sizeof(T) + rows * P * 4,
             2.0 * rows * P * d);
   if (head_mode == HEAD_LAST_TO_HIST) {
     launch_ex(s, h->pdl, head_kernel<T>, dim3(B, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
               (const T *)m.W_head, d, P, eps, g, 1, h->hist, (float *)nullptr,
-              ds.k_pos >= 0 ? (const DevState *)h->st : (const DevState *)nullptr, h->muq, ds.k_pos, ds.K);
-  } else if (head_mode == HEAD_ALL_TO_VOUT && M >= kManyRows && (size_t)8 * d * sizeof(float) <= 200 * 1024) {
-    launch_ex(s, h->pdl, head_rows_kernel<T>, dim3((M + 7) / 8, (P + 31) / 32), dim3(256), (size_t)8 * d * sizeof(float),
-              h->x, m.g_f, (const T *)m.W_head, M, d, P, eps, vout);
+              ds.k_pos >= 0 ? (const DevState *)h->st : (const DevState *)nullptr, h->muq, ds.k_pos, ds.K, Pi);
+  } else if (head_mode == HEAD_ALL_TO_VOUT && Mb >= kManyRows && (size_t)8 * d * sizeof(float) <= 200 * 1024) {
+    launch_ex(s, h->pdl, head_rows_kernel<T>, dim3((Mb + 7) / 8, (P + 31) / 32), dim3(256), (size_t)8 * d * sizeof(float),
+              h->x, m.g_f, (const T *)m.W_head, Mb, d, P, eps, vout, g);
   } else if (head_mode == HEAD_ALL_TO_VOUT) {
-    launch_ex(s, h->pdl, head_kernel<T>, dim3(M, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
-              (const T *)m.W_head, d, P, eps, g, 0, (float *)nullptr, vout, (const DevState *)nullptr, (float *)nullptr, 0, 0);
+    launch_ex(s, h->pdl, head_kernel<T>, dim3(Mb, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
+              (const T *)m.W_head, d, P, eps, g, 0, (float *)nullptr, vout, (const DevState *)nullptr, (float *)nullptr, 0, 0,
+              Pi);
   }
 }
 
@@ -565,9 +593,9 @@ int check_call(tsfm_spec *h, const float *series, int B, int ctx_len, int H, flo
   if (!h || !series || !out) return TSFM_ERR_ARG;
   if (B < 1 || H < 1 || ctx_len < 1) return TSFM_ERR_ARG;
   const int P = h->cfg.patch_len;
-  if (ctx_len % P) return TSFM_ERR_SHAPE;
-  const int N = ctx_len / P, T = (H + P - 1) / P;
-  if (N < 2) return TSFM_ERR_SHAPE;
+  if (ctx_len % P) return TSFM_ERR_SHAPE;                       // the context is a whole number of patches
+  const int N = ctx_len / h->P_in, T = (H + P - 1) / P;         // N counts input tokens
+  if (ctx_len / P < 2) return TSFM_ERR_SHAPE;
   if (B > h->cfg.max_batch || N > h->cfg.max_ctx_tokens || T > h->cfg.max_horizon_patches ||
       K > h->cfg.max_K)
     return TSFM_ERR_SHAPE;
@@ -579,22 +607,33 @@ int check_call(tsfm_spec *h, const float *series, int B, int ctx_len, int H, flo
 // stream capture.
 
 void enqueue_begin(tsfm_spec *h, int B, int ctx_len) {
-  const int P = h->cfg.patch_len;
+  const int hist_stride = h->cap * h->P_in;             // values per series in the history buffer
+  const int hist_len = hist_stride - (h->check ? h->P_in : 0);   // (the spare token stays untouched)
   cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->ls);
-  KTimer kt(h, KC_INSTNORM, (double)B * (ctx_len + (double)h->cap * P) * 4, 4.0 * B * ctx_len);
-  launch_ex(h->ls, h->pdl, instnorm_kernel, dim3(B), dim3(256), 0, h->st, ctx_len, P, h->cap, h->cfg.norm_eps, h->hist,
-            h->mean, h->sd, h->done);
+  KTimer kt(h, KC_INSTNORM, (double)B * (ctx_len + (double)hist_len) * 4, 4.0 * B * ctx_len);
+  launch_ex(h->ls, h->pdl, instnorm_kernel, dim3(B), dim3(256), 0, h->st, ctx_len, hist_stride, hist_len, h->cfg.norm_eps, h->hist,
+            h->mean, h->sd, h->done, h->live, h->n_live);
 }
 
+// Bounds-checking mode: after the work of a call, look at every guard region.
+void enqueue_guard_check(tsfm_spec *h) {
+  if (!h->check || h->guards.empty()) return;
+  launch_ex(h->ls, h->pdl, guard_check_kernel, dim3(64, (unsigned)std::min<size_t>(h->guards.size(), 1024)), dim3(256), 0,
+            (const GuardRegion *)h->dev_guards, (int)h->guards.size(), h->dev_status);
+}
+
+// N = context tokens.
 void enqueue_denorm(tsfm_spec *h, int B, int N, int H) {
   KTimer kt(h, KC_DENORM, 8.0 * B * H, 2.0 * B * H);
-  launch_ex(h->ls, h->pdl, denorm_kernel, dim3(B), dim3(256), 0, h->hist, N, h->cfg.patch_len, h->cap, H, h->mean, h->sd,
+  launch_ex(h->ls, h->pdl, denorm_kernel, dim3(B), dim3(256), 0, h->hist, N * h->P_in, h->cap * h->P_in, H, h->mean, h->sd,
             h->st);
+  enqueue_guard_check(h);
 }
 
 // Everything of a speculative forecast that precedes the round loop: counters, traces,
 // instance norm, and the prefill of both caches (the target ingests the context except its
 // last patch, the draft except its last two: those are re-read by the first round).
+// N counts context tokens; a patch is tpp = P / P_in of them.
 void enqueue_spec_prologue(tsfm_spec *h, int B, int N, int T, int K) {
   cudaStream_t s = h->ls;
   cudaMemsetAsync(h->ctr, 0, sizeof(AcceptCounters), s);
@@ -602,9 +641,10 @@ void enqueue_spec_prologue(tsfm_spec *h, int B, int N, int T, int K) {
   cudaMemsetAsync(h->tr_nacc, 0xff, sizeof(int) * (size_t)T * B, s);
   cudaMemsetAsync(h->tr_ell, 0, sizeof(float) * (size_t)T * B * K, s);
   cudaMemsetAsync(h->tr_logu, 0, sizeof(float) * (size_t)T * B * K, s);
-  enqueue_begin(h, B, N * h->cfg.patch_len);
-  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
-  pass(h, h->drf, B, PassGeom{nullptr, 0, N - 2, h->cap}, HEAD_NONE);
+  const int tpp = h->tpp;
+  enqueue_begin(h, B, N * h->P_in);
+  pass(h, h->tgt, B, PassGeom{nullptr, 0, N - tpp, h->cap}, HEAD_NONE);
+  pass(h, h->drf, B, PassGeom{nullptr, 0, N - 2 * tpp, h->cap}, HEAD_NONE);
 }
 
 // One round of Algorithm 1 for the whole batch: K draft steps, one verification pass over
@@ -612,22 +652,27 @@ void enqueue_spec_prologue(tsfm_spec *h, int B, int N, int T, int K) {
 // the Philox key are read from device state, so the same enqueued work serves every round.
 void enqueue_round(tsfm_spec *h, int B, int N, int T, int K, cudaGraphConditionalHandle handle, int use_handle,
                    const int *body_launches = nullptr) {
-  const int P = h->cfg.patch_len;
+  const int P = h->cfg.patch_len, tpp = h->tpp;
+  // the passes of a round run over the unfinished series only (see PassGeom)
+  const int *live = h->compact ? h->live : nullptr, *n_live = h->compact ? h->n_live : nullptr;
   // step 1 re-ingests the last two committed patches (the draft cache may lack the last
-  // accepted proposal), steps 2..K ingest the previous proposal
-  pass(h, h->drf, B, PassGeom{h->done, N - 2, 2, h->cap}, HEAD_LAST_TO_HIST, nullptr, &h->st->t_phase[0], DraftStep{0, K});
+  // accepted proposal), steps 2..K ingest the previous proposal; a patch is tpp tokens
+  pass(h, h->drf, B, PassGeom{h->done, N - 2 * tpp, 2 * tpp, h->cap, live, n_live, tpp, tpp}, HEAD_LAST_TO_HIST, nullptr,
+       &h->st->t_phase[0], DraftStep{0, K});
   for (int i = 2; i <= K; ++i)
-    pass(h, h->drf, B, PassGeom{h->done, N - 1 + (i - 1), 1, h->cap}, HEAD_LAST_TO_HIST, nullptr, nullptr,
-         DraftStep{i - 1, K});
-  // single-pass verification over [pending, x_1..x_K]
-  pass(h, h->tgt, B, PassGeom{h->done, N - 1, K + 1, h->cap}, HEAD_ALL_TO_VOUT, h->vout, &h->st->t_phase[1]);
+    pass(h, h->drf, B, PassGeom{h->done, N - tpp + (i - 1) * tpp, tpp, h->cap, live, n_live, tpp, tpp}, HEAD_LAST_TO_HIST,
+         nullptr, nullptr, DraftStep{i - 1, K});
+  // single-pass verification over [pending, x_1..x_K], read at the last token of each patch: the
+  // prefix boundaries N - 1 + i (P / P_in), i = 0..K (appendix B, "Per-Family Boundary Indexing")
+  pass(h, h->tgt, B, PassGeom{h->done, N - tpp, (K + 1) * tpp, h->cap, live, n_live, tpp, tpp}, HEAD_ALL_TO_VOUT, h->vout,
+       &h->st->t_phase[1]);
 
   AcceptArgs a{};
-  a.x = a.mu_q = h->hist + (size_t)N * P;       // slot N + done[b] holds x_1
-  a.x_stride_b = (long long)h->cap * P;
+  a.x = a.mu_q = h->hist + (size_t)N * h->P_in;   // patch done[b] behind the context holds x_1
+  a.x_stride_b = (long long)h->cap * h->P_in;
   a.mu_q_alt = h->muq;                          // used only when the call samples its proposals
   a.mu_p = h->vout;
-  a.commit = h->hist + (size_t)N * P;
+  a.commit = h->hist + (size_t)N * h->P_in;
   a.commit_stride_b = a.x_stride_b;
   a.commit_accepted = 0;
   a.commit_follows_done = 1;
@@ -646,16 +691,17 @@ void enqueue_round(tsfm_spec *h, int B, int N, int T, int K, cudaGraphConditiona
     KTimer kt(h, KC_ACCEPT, (double)B * (2 * K + 2) * P * 4, 4.0 * B * K * P);
     launch_ex(h->ls, h->pdl, accept_kernel, dim3((B + 3) / 4), dim3(128), 0, a);
   }
-  launch_ex(h->ls, h->pdl, round_end_kernel, dim3(1), dim3(1), 0, h->st, (const int *)h->unfinished, T, handle,
-            use_handle, body_launches, h->dev_launches);
+  launch_ex(h->ls, h->pdl, round_end_kernel, dim3(1), dim3(256), 0, h->st, (const int *)h->unfinished, T, handle,
+            use_handle, body_launches, h->dev_launches, (const int *)h->done, B, h->live, h->n_live);
 }
 
 // Plain patch-autoregressive decoding with one model (the target, or the draft on its own).
 void enqueue_single_model(tsfm_spec *h, ModelDev &m, int B, int N, int T, int H) {
-  enqueue_begin(h, B, N * h->cfg.patch_len);
-  pass(h, m, B, PassGeom{nullptr, 0, N - 1, h->cap}, HEAD_NONE);
-  for (int t = 0; t < T; ++t)       // Eq. 1: one pass per committed patch
-    pass(h, m, B, PassGeom{nullptr, N - 1 + t, 1, h->cap}, HEAD_LAST_TO_HIST, nullptr,
+  const int tpp = h->tpp;
+  enqueue_begin(h, B, N * h->P_in);
+  pass(h, m, B, PassGeom{nullptr, 0, N - tpp, h->cap}, HEAD_NONE);
+  for (int t = 0; t < T; ++t)       // Eq. 1: one pass per committed patch (its tpp tokens)
+    pass(h, m, B, PassGeom{nullptr, N - tpp + t * tpp, tpp, h->cap}, HEAD_LAST_TO_HIST, nullptr,
          t == 0 ? &h->st->t_phase[0] : nullptr);
   enqueue_denorm(h, B, N, H);
 }
@@ -789,6 +835,16 @@ long long device_launches(tsfm_spec *h) {
 
 bool use_graph(const tsfm_spec *h) { return !(h->cfg.exec_mode & TSFM_EXEC_STREAM) && !h->profiling; }
 
+// What a non-zero device status word means for the caller.
+int status_code(tsfm_spec *h, int status) {
+  if (status == 0) return TSFM_OK;
+  if (status < DEV_GUARD_BASE) return TSFM_ERR_TIMEOUT;
+  const size_t k = (size_t)(status - DEV_GUARD_BASE);
+  g_cuda_err = "bounds check: a kernel wrote past the end of '" +
+               (k < h->guard_names.size() ? h->guard_names[k] : std::string("?")) + "' (guard region " + std::to_string(k) + ")";
+  return TSFM_ERR_INTERNAL;
+}
+
 // Reads status and phase clocks back (synchronises) and fills ms_total.
 int finish_stats(tsfm_spec *h, tsfm_stats *stats, DevState *st_out) {
   cudaStream_t s = h->stream;
@@ -808,14 +864,26 @@ int finish_stats(tsfm_spec *h, tsfm_stats *stats, DevState *st_out) {
 extern "C" {
 
 size_t tsfm_weights_bytes(const tsfm_arch *arch, int32_t patch_len, int32_t dtype) {
-  if (!arch || !arch_ok(*arch, patch_len) || (dtype != TSFM_F32 && dtype != TSFM_BF16)) return 0;
-  return blob_layout(*arch, patch_len, dtype).total;
+  return tsfm_weights_bytes_io(arch, 0, patch_len, dtype);
 }
 
 size_t tsfm_weights_offset(const tsfm_arch *arch, int32_t patch_len, int32_t dtype, int32_t layer,
                            const char *name) {
-  if (!arch || !name || !arch_ok(*arch, patch_len) || (dtype != TSFM_F32 && dtype != TSFM_BF16)) return 0;
-  const BlobLayout b = blob_layout(*arch, patch_len, dtype);
+  return tsfm_weights_offset_io(arch, 0, patch_len, dtype, layer, name);
+}
+
+size_t tsfm_weights_bytes_io(const tsfm_arch *arch, int32_t patch_in, int32_t patch_len, int32_t dtype) {
+  if (!arch || !arch_ok(*arch, patch_len) || !io_ok(patch_in, patch_len) || (dtype != TSFM_F32 && dtype != TSFM_BF16))
+    return 0;
+  return blob_layout(*arch, patch_len, dtype, patch_in).total;
+}
+
+size_t tsfm_weights_offset_io(const tsfm_arch *arch, int32_t patch_in, int32_t patch_len, int32_t dtype, int32_t layer,
+                              const char *name) {
+  if (!arch || !name || !arch_ok(*arch, patch_len) || !io_ok(patch_in, patch_len) ||
+      (dtype != TSFM_F32 && dtype != TSFM_BF16))
+    return 0;
+  const BlobLayout b = blob_layout(*arch, patch_len, dtype, patch_in);
   const std::string n(name);
   if (n == "W_emb") return b.W_emb;
   if (n == "g_f") return b.g_f;
@@ -862,14 +930,15 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   *out_h = nullptr;
   const int P = cfg->patch_len;
   if (cfg->dtype != TSFM_F32 && cfg->dtype != TSFM_BF16) return TSFM_ERR_ARG;
-  if (cfg->exec_mode & ~(TSFM_EXEC_STREAM | TSFM_EXEC_NO_PDL)) return TSFM_ERR_ARG;
+  if (cfg->exec_mode & ~(TSFM_EXEC_STREAM | TSFM_EXEC_NO_PDL | TSFM_EXEC_NO_COMPACT | TSFM_EXEC_CHECK_BOUNDS))
+    return TSFM_ERR_ARG;
   if (cfg->gemm_backend != TSFM_GEMM_AUTO && cfg->gemm_backend != TSFM_GEMM_SIMT) return TSFM_ERR_ARG;
   if (cfg->draft_mode != TSFM_DRAFT_SEPARATE && cfg->draft_mode != TSFM_DRAFT_LAYER_SKIP) return TSFM_ERR_ARG;
   if (cfg->max_batch < 1 || cfg->max_ctx_tokens < 2 || cfg->max_horizon_patches < 1 || cfg->max_K < 1 ||
       cfg->max_K > TSFM_MAX_K)
     return TSFM_ERR_ARG;
   if (!(cfg->rms_eps > 0.f) || !(cfg->norm_eps > 0.f) || !(cfg->rope_base > 1.f)) return TSFM_ERR_ARG;
-  if (!arch_ok(cfg->target, P) || !arch_ok(cfg->draft, P)) return TSFM_ERR_SHAPE;
+  if (!arch_ok(cfg->target, P) || !arch_ok(cfg->draft, P) || !io_ok(cfg->patch_in, P)) return TSFM_ERR_SHAPE;
   if (cfg->draft_mode == TSFM_DRAFT_LAYER_SKIP) {
     if (draft_w && draft_w->blob) return TSFM_ERR_ARG;
     if (cfg->draft.d_model != cfg->target.d_model || cfg->draft.n_heads != cfg->target.n_heads ||
@@ -888,21 +957,28 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   if (!h) return TSFM_ERR_INTERNAL;
   h->cfg = *cfg;
   h->stream = h->ls = (cudaStream_t)cfg->stream;
-  h->cap = cfg->max_ctx_tokens + cfg->max_horizon_patches + cfg->max_K + 1;
+  h->P_in = token_len(cfg->patch_in, P);
+  h->tpp = P / h->P_in;
+  if (cfg->max_ctx_tokens < 2 * h->tpp) { delete h; return TSFM_ERR_ARG; }   // at least two context patches
+  h->check = (cfg->exec_mode & TSFM_EXEC_CHECK_BOUNDS) != 0;
+  // token capacity per series; bounds-checking mode adds one spare token that nothing may write
+  h->cap = cfg->max_ctx_tokens + (cfg->max_horizon_patches + cfg->max_K + 1) * h->tpp + (h->check ? 1 : 0);
   h->use_tc = cfg->dtype == TSFM_BF16 && cfg->gemm_backend != TSFM_GEMM_SIMT;
   h->pdl = (cfg->exec_mode & TSFM_EXEC_NO_PDL) == 0;
+  h->compact = (cfg->exec_mode & TSFM_EXEC_NO_COMPACT) == 0;
   int rc = TSFM_OK;
   auto fail = [&](int code) { tsfm_spec_destroy(h); return code; };
 
-  if (target_w->bytes < blob_layout(cfg->target, P, cfg->dtype).total) return fail(TSFM_ERR_SHAPE);
-  if ((rc = read_header(target_w, cfg->target, P, cfg->dtype, h->stream))) return fail(rc);
-  wire_model(h->tgt, cfg->target, cfg->target, target_w->blob, P, cfg->dtype);
+  const int Pi = cfg->patch_in;
+  if (target_w->bytes < blob_layout(cfg->target, P, cfg->dtype, Pi).total) return fail(TSFM_ERR_SHAPE);
+  if ((rc = read_header(target_w, cfg->target, P, Pi, cfg->dtype, h->stream))) return fail(rc);
+  wire_model(h->tgt, cfg->target, cfg->target, target_w->blob, P, cfg->dtype, Pi);
   if (cfg->draft_mode == TSFM_DRAFT_LAYER_SKIP) {
-    wire_model(h->drf, cfg->draft, cfg->target, target_w->blob, P, cfg->dtype);
+    wire_model(h->drf, cfg->draft, cfg->target, target_w->blob, P, cfg->dtype, Pi);
   } else {
-    if (draft_w->bytes < blob_layout(cfg->draft, P, cfg->dtype).total) return fail(TSFM_ERR_SHAPE);
-    if ((rc = read_header(draft_w, cfg->draft, P, cfg->dtype, h->stream))) return fail(rc);
-    wire_model(h->drf, cfg->draft, cfg->draft, draft_w->blob, P, cfg->dtype);
+    if (draft_w->bytes < blob_layout(cfg->draft, P, cfg->dtype, Pi).total) return fail(TSFM_ERR_SHAPE);
+    if ((rc = read_header(draft_w, cfg->draft, P, Pi, cfg->dtype, h->stream))) return fail(rc);
+    wire_model(h->drf, cfg->draft, cfg->draft, draft_w->blob, P, cfg->dtype, Pi);
   }
 
   const size_t e = elt_bytes(cfg->dtype);
@@ -910,30 +986,42 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   for (ModelDev *m : {&h->tgt, &h->drf}) {
     m->kv_layer_elems = (size_t)Bm * m->arch.d_model * h->cap;
     const size_t bytes = m->kv_layer_elems * m->arch.n_layers * e;
-    if ((rc = dev_alloc(h, (char **)&m->Kc, bytes))) return fail(rc);
-    if ((rc = dev_alloc(h, (char **)&m->Vc, bytes))) return fail(rc);
+    if ((rc = dev_alloc(h, (char **)&m->Kc, bytes, "K cache"))) return fail(rc);
+    if ((rc = dev_alloc(h, (char **)&m->Vc, bytes, "V cache"))) return fail(rc);
+    if (h->check) {                       // the spare last row of every (layer, series, head) block
+      const size_t row = (size_t)m->dh * e, blk = (size_t)h->cap * row;
+      const size_t n_blk = (size_t)m->arch.n_layers * Bm * m->arch.n_heads;
+      if ((rc = add_guard(h, "K cache row past a series' capacity", (char *)m->Kc + blk - row, blk, n_blk, row))) return fail(rc);
+      if ((rc = add_guard(h, "V cache row past a series' capacity", (char *)m->Vc + blk - row, blk, n_blk, row))) return fail(rc);
+    }
     if ((rc = make_rope(h, *m))) return fail(rc);
     rc = cfg->dtype == TSFM_BF16 ? attn_prepare<bf16>(m->dh, h->cap) : attn_prepare<float>(m->dh, h->cap);
     if (rc) return fail(rc);
   }
-  h->M_max = Bm * std::max(std::max(cfg->max_ctx_tokens, cfg->max_K + 1), 2);
+  h->M_max = Bm * std::max(std::max(cfg->max_ctx_tokens, (cfg->max_K + 1) * h->tpp), 2 * h->tpp);
   const int dmax = std::max(cfg->target.d_model, cfg->draft.d_model);
   const int fmax = std::max(cfg->target.d_ff, cfg->draft.d_ff);
   const size_t Mx = h->M_max;
-  if ((rc = dev_alloc(h, &h->x, Mx * dmax))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->qkv, Mx * 3 * dmax))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->ssq, Mx * (dmax / 32 + 1)))) return fail(rc);
-  if ((rc = dev_alloc(h, (char **)&h->a, Mx * dmax * e))) return fail(rc);
-  if ((rc = dev_alloc(h, (char **)&h->ao, Mx * dmax * e))) return fail(rc);
-  if ((rc = dev_alloc(h, (char **)&h->hbuf, Mx * fmax * e))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->hist, (size_t)Bm * h->cap * P))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->vout, (size_t)Bm * (cfg->max_K + 1) * P))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->muq, (size_t)Bm * cfg->max_K * P))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->mean, Bm))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->sd, Bm))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->done, Bm))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->x, Mx * dmax, "x"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->qkv, Mx * 3 * dmax, "qkv"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->ssq, Mx * (dmax / 32 + 1), "ssq"))) return fail(rc);
+  if ((rc = dev_alloc(h, (char **)&h->a, Mx * dmax * e, "a"))) return fail(rc);
+  if ((rc = dev_alloc(h, (char **)&h->ao, Mx * dmax * e, "ao"))) return fail(rc);
+  if ((rc = dev_alloc(h, (char **)&h->hbuf, Mx * fmax * e, "hbuf"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->hist, (size_t)Bm * h->cap * h->P_in, "hist"))) return fail(rc);
+  if (h->check) {                         // the spare last token of every series' history
+    const size_t tok = (size_t)h->P_in * sizeof(float), blk = (size_t)h->cap * tok;
+    if ((rc = add_guard(h, "history token past a series' capacity", (char *)h->hist + blk - tok, blk, Bm, tok))) return fail(rc);
+  }
+  if ((rc = dev_alloc(h, &h->vout, (size_t)Bm * (cfg->max_K + 1) * P, "vout"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->muq, (size_t)Bm * cfg->max_K * P, "muq"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->mean, Bm, "mean"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->sd, Bm, "sd"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->done, Bm, "done"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->live, Bm, "live"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->n_live, 1))) return fail(rc);
   if ((rc = dev_alloc(h, &h->ctr, 1))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->unfinished, cfg->max_horizon_patches + 1))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->unfinished, cfg->max_horizon_patches + 1, "unfinished"))) return fail(rc);
   if ((rc = dev_alloc(h, &h->dev_status, 1))) return fail(rc);
   if ((rc = dev_alloc(h, &h->st, 1))) return fail(rc);
   if ((rc = dev_alloc(h, &h->dev_launches, 1))) return fail(rc);
@@ -945,17 +1033,23 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
       cudaStreamCreateWithFlags(&h->cap_stream2, cudaStreamNonBlocking) != cudaSuccess)
     return fail(TSFM_ERR_CUDA);
   const size_t tr = (size_t)cfg->max_horizon_patches * Bm;
-  if ((rc = dev_alloc(h, &h->tr_nacc, tr))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->tr_ell, tr * cfg->max_K))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->tr_logu, tr * cfg->max_K))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->stage_in, (size_t)Bm * cfg->max_ctx_tokens * P))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->stage_out, (size_t)Bm * cfg->max_horizon_patches * P))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->tr_nacc, tr, "trace n_accept"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->tr_ell, tr * cfg->max_K, "trace ell"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->tr_logu, tr * cfg->max_K, "trace log_u"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->stage_in, (size_t)Bm * cfg->max_ctx_tokens * h->P_in, "stage_in"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->stage_out, (size_t)Bm * cfg->max_horizon_patches * P, "stage_out"))) return fail(rc);
   if (cudaMallocHost((void **)&h->h_unfinished, sizeof(int)) != cudaSuccess) return fail(TSFM_ERR_CUDA);
   h->ev.resize(2 + 4 * (size_t)cfg->max_horizon_patches + 4);
   for (auto &ev : h->ev)
     if (cudaEventCreate(&ev) != cudaSuccess) { ev = nullptr; return fail(TSFM_ERR_CUDA); }
   if (cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream) != cudaSuccess) return fail(TSFM_ERR_CUDA);
 
+  if (h->check) {
+    if ((rc = dev_alloc(h, &h->dev_guards, h->guards.size() + 1, "guard table"))) return fail(rc);
+    if (cudaMemcpyAsync(h->dev_guards, h->guards.data(), sizeof(GuardRegion) * h->guards.size(), cudaMemcpyHostToDevice,
+                        h->stream) != cudaSuccess)
+      return fail(TSFM_ERR_CUDA);
+  }
   prefer_max_smem_all();
   if (h->use_tc) {
     if ((rc = gemm_sk_init())) return fail(rc);
@@ -981,7 +1075,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
 static int single_model_forecast(tsfm_spec *h, int mode, const float *series, int32_t B, int32_t ctx_len, int32_t H,
                                  float *out, tsfm_stats *stats) {
   if (int rc = check_call(h, series, B, ctx_len, H, out, 1)) return rc;
-  const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
+  const int P = h->cfg.patch_len, N = ctx_len / h->P_in, T = (H + P - 1) / P;
   cudaStream_t s = h->stream;
   if (stats) CU_TRY(cudaEventRecord(h->ev[0], s));
   if (int rc = write_call_state(h, series, out, 1.f, 0)) return rc;
@@ -1004,7 +1098,7 @@ static int single_model_forecast(tsfm_spec *h, int mode, const float *series, in
     (mode == 1 ? stats->ms_verify : stats->ms_draft) = (float)((st.t_end - st.t_phase[0]) * 1e-6);
     stats->rounds = T;
     stats->patches_committed = (int64_t)B * T;
-    if (stats->device_status) return TSFM_ERR_TIMEOUT;
+    if (stats->device_status) return status_code(h, stats->device_status);
   }
   return TSFM_OK;
 }
@@ -1035,7 +1129,7 @@ int tsfm_spec_forecast_variant(tsfm_spec *h, const float *series, int32_t B, int
       return TSFM_ERR_ARG;
   }
   if (int rc = check_call(h, series, B, ctx_len, H, out, K)) return rc;
-  const int P = h->cfg.patch_len, N = ctx_len / P, T = (H + P - 1) / P;
+  const int P = h->cfg.patch_len, N = ctx_len / h->P_in, T = (H + P - 1) / P;
   cudaStream_t s = h->stream;
   if (stats) CU_TRY(cudaEventRecord(h->ev[0], s));
   if (int rc = write_call_state(h, series, out, tau, seed, variant)) return rc;
@@ -1080,7 +1174,7 @@ int tsfm_spec_forecast_variant(tsfm_spec *h, const float *series, int32_t B, int
     stats->ms_draft = (float)(st.ns_draft * 1e-6);
     stats->ms_verify = (float)(st.ns_verify * 1e-6);
     stats->ms_accept = (float)(st.ns_accept * 1e-6);
-    if (stats->device_status) return TSFM_ERR_TIMEOUT;
+    if (stats->device_status) return status_code(h, stats->device_status);
   }
   return TSFM_OK;
 }
@@ -1153,18 +1247,19 @@ int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t
   if (!h || !tokens || !out || (which != 0 && which != 1)) return TSFM_ERR_ARG;
   if (B < 1 || n < 1) return TSFM_ERR_ARG;
   if (B > h->cfg.max_batch || n > h->cfg.max_ctx_tokens || B * n > h->M_max) return TSFM_ERR_SHAPE;
-  const int P = h->cfg.patch_len;
-  CU_TRY(cudaMemcpy2DAsync(h->hist, (size_t)h->cap * P * sizeof(float), tokens, (size_t)n * P * sizeof(float),
-                           (size_t)n * P * sizeof(float), B, cudaMemcpyDeviceToDevice, h->stream));
+  const int Pi = h->P_in;
+  CU_TRY(cudaMemcpy2DAsync(h->hist, (size_t)h->cap * Pi * sizeof(float), tokens, (size_t)n * Pi * sizeof(float),
+                           (size_t)n * Pi * sizeof(float), B, cudaMemcpyDeviceToDevice, h->stream));
   CU_TRY(cudaMemsetAsync(h->dev_status, 0, sizeof(int), h->stream));
   h->ls = h->stream;
   pass(h, which == 0 ? h->tgt : h->drf, B, PassGeom{nullptr, 0, n, h->cap}, HEAD_ALL_TO_VOUT, out);
+  enqueue_guard_check(h);
   CU_TRY(cudaGetLastError());
   if (int rc = take_enqueue_err(h)) return rc;
   int status = 0;
   CU_TRY(cudaMemcpyAsync(&status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, h->stream));
   CU_TRY(cudaStreamSynchronize(h->stream));
-  return status ? TSFM_ERR_TIMEOUT : TSFM_OK;
+  return status_code(h, status);
 }
 
 int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t M, int32_t N, int32_t Kd,
@@ -1260,6 +1355,19 @@ int tsfm_gemm_bf16_static(void *stream, const void *A, const void *W, float *C, 
   CU_TRY(cudaStreamSynchronize(s));
   CU_TRY(cudaGetLastError());
   return hs ? TSFM_ERR_TIMEOUT : TSFM_OK;
+}
+
+int tsfm_spec_debug_guard(tsfm_spec *h, int32_t region, int32_t damage, int32_t *n_regions) {
+  if (!h) return TSFM_ERR_ARG;
+  if (n_regions) *n_regions = (int32_t)h->guards.size();
+  if (region < 0) return TSFM_OK;
+  if (!h->check || (size_t)region >= h->guards.size()) return TSFM_ERR_ARG;
+  // one byte of the library's own guard region: an ordinary in-bounds write
+  const GuardRegion &g = h->guards[region];
+  unsigned char *p = const_cast<unsigned char *>(g.base) + (size_t)(g.n_blocks - 1) * g.stride + g.len - 1;
+  CU_TRY(cudaMemsetAsync(p, damage ? 0x00 : GUARD_BYTE, 1, h->stream));
+  CU_TRY(cudaStreamSynchronize(h->stream));
+  return TSFM_OK;
 }
 
 int tsfm_spec_set_profiling(tsfm_spec *h, int32_t enable) {

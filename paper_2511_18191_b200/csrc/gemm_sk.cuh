@@ -110,8 +110,19 @@ __global__ void __launch_bounds__(192, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
                const __grid_constant__ CUtensorMap mapC, void *__restrict__ C, int M, int N, int K, int BN,
                int stages, int tmem_cols, int ring_bytes, int epi, int tma_c, const SkNorm nm,
-               int *__restrict__ status) {
+               int *__restrict__ status, const LiveRows lr) {
   constexpr int wt = WT;
+  // Active-series compaction: only the first n_live * q_len rows are in use.  CTAs (whole clusters:
+  // the split shares the token tile) of token tiles past them leave before touching anything.  The
+  // count is read before the dependency wait on purpose, so that such CTAs cost nothing: it was
+  // written by the kernel that closed the previous round, and every contraction has at least two
+  // kernels of its own pass between itself and that one, so it is complete and visible by the time
+  // this grid may start (a grid starts only after every CTA of its predecessor has passed its own
+  // wait, i.e. after the predecessor's predecessor has finished).
+  if (lr.n_live) {
+    M = min(M, *reinterpret_cast<const volatile int *>(lr.n_live) * lr.q_len);
+    if ((int)blockIdx.y * BN >= M) return;
+  }
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = tiles + (uint32_t)ring_bytes;
@@ -506,7 +517,7 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
 }
 
 static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, int M, int epi, int *status,
-                           const SkNorm *norm = nullptr) {
+                           const SkNorm *norm = nullptr, LiveRows lr = LiveRows{nullptr, 0}) {
   if (!p.valid || M < 1 || M > p.M_max) return false;
   int BN, S, wt;
   gemm_sk_geometry(p.N, p.K, M, &BN, &S, &wt);
@@ -558,12 +569,12 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   int N = p.N, K = p.K, stages = sh.stages, cols = sh.tmem_cols, rb = ring_bytes;
   if (wt == 2)
     return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<2, false>, p.mapW, p.mapA[idx], *mapC, C, M, N, K, BN, stages, cols, rb,
-                              epi, tc, nm, status) == cudaSuccess;
+                              epi, tc, nm, status, lr) == cudaSuccess;
   if (norm)
     return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, true>, p.mapW, p.mapA[idx], *mapC, C, M, N, K, BN, stages, cols, rb,
-                              epi, tc, nm, status) == cudaSuccess;
+                              epi, tc, nm, status, lr) == cudaSuccess;
   return cudaLaunchKernelEx(&cfg, gemm_sk_kernel<1, false>, p.mapW, p.mapA[idx], *mapC, C, M, N, K, BN, stages, cols, rb,
-                            epi, tc, nm, status) == cudaSuccess;
+                            epi, tc, nm, status, lr) == cudaSuccess;
 }
 
 }  // namespace tsfm

@@ -8,28 +8,52 @@
 
 namespace tsfm {
 
-// Where the tokens of one pass sit.  Token j of series b is history slot
-// pos0(b) + j with pos0(b) = done[b] + base (done may be NULL = 0).  Activations are
-// stored row-major with row = b * q_len + j.
+// Where the tokens of one pass sit.  Token j of series b is history token
+// pos0(b) + j with pos0(b) = done[b] * tpp + base (done may be NULL = 0; tpp = tokens per
+// committed patch: 1 when a token is a whole patch, P / P_in for shorter input tokens).
+// Activations are stored row-major with row = b * q_len + j.  The mean head reads every
+// head_step-th token of a pass (the last token of each patch: the prefix boundaries
+// N - 1 + i (P / P_in) of the paper's appendix B, "Per-Family Boundary Indexing").
+//
+// Active-series compaction: inside the round loop only the series that still have patches to
+// commit take part in a pass.  `live` lists them in ascending order and `n_live` counts them (both
+// written by round_end_kernel); the pass works on SLOTS 0 .. n_live-1, slot s standing for series
+// live[s].  Activation rows are compacted (row = slot * q_len + j); history, KV caches, `done` and
+// the verification output stay indexed by series.  Grids are sized for all B series (a captured
+// graph cannot change them): blocks of slots >= n_live return at once.  live == NULL: slot = series.
 struct PassGeom {
   const int *done;   // [B] patches committed so far, or NULL
   int base;          // pos0 = done[b] + base
   int q_len;         // tokens per series in this pass
   int cap;           // token capacity of history / KV cache per series
+  const int *live = nullptr;     // [B] slot -> series, or NULL
+  const int *n_live = nullptr;   // number of live slots, or NULL (all)
+  int tpp = 1;                   // tokens per committed patch
+  int head_step = 1;             // the head reads tokens head_step - 1, 2 head_step - 1, ... of the pass
 };
 __device__ __forceinline__ int pos0_of(const PassGeom &g, int b) {
-  return (g.done ? g.done[b] : 0) + g.base;
+  return (g.done ? g.done[b] * g.tpp : 0) + g.base;
+}
+__device__ __forceinline__ bool slot_dead(const PassGeom &g, int slot) { return g.n_live && slot >= *g.n_live; }
+__device__ __forceinline__ int series_of(const PassGeom &g, int slot) { return g.live ? g.live[slot] : slot; }
+// Rows of a pass that are in use: n_live * q_len of the M the launch was sized for.
+struct LiveRows {
+  const int *n_live;
+  int q_len;
+};
+__device__ __forceinline__ int live_rows(const LiveRows &lr, int M) {
+  return lr.n_live ? min(M, *lr.n_live * lr.q_len) : M;
 }
 
 // ----------------------------------------------------------------------------------
 // Instance statistics frozen on the context (Sec. 3.4) and history initialisation.
-// grid = B, block = 256.  hist[b, t, :] = (series - mean) / sd for the N context
-// patches; the remaining slots are zeroed.  Sums in fp64 (8 K values, one pass each).
+// grid = B, block = 256.  hist[b, :ctx_len] = (series - mean) / sd; the rest of the
+// series' hist_len values is zeroed.  Sums in fp64 (8 K values, one pass each).
 // ----------------------------------------------------------------------------------
-__global__ void instnorm_kernel(DevState *__restrict__ st, int ctx_len, int P, int cap,
+__global__ void instnorm_kernel(DevState *__restrict__ st, int ctx_len, int hist_stride, int hist_len,
                                 float norm_eps, float *__restrict__ hist,
                                 float *__restrict__ mean_out, float *__restrict__ sd_out,
-                                int *__restrict__ done) {
+                                int *__restrict__ done, int *__restrict__ live, int *__restrict__ n_live) {
   __shared__ double red[32];
   const int b = blockIdx.x;
   pdl_sync();
@@ -45,18 +69,20 @@ __global__ void instnorm_kernel(DevState *__restrict__ st, int ctx_len, int P, i
   }
   const double var = block_sum_d(acc, red) / ctx_len;
   const double sd = sqrt(var + (double)norm_eps);
-  float *hb = hist + (size_t)b * cap * P;
-  for (int i = threadIdx.x; i < cap * P; i += blockDim.x)
+  float *hb = hist + (size_t)b * hist_stride;             // (stride > length only in bounds-checking mode)
+  for (int i = threadIdx.x; i < hist_len; i += blockDim.x)
     hb[i] = (i < ctx_len) ? (float)(((double)s[i] - mean) / sd) : 0.f;
   if (threadIdx.x == 0) {
     mean_out[b] = (float)mean;
     sd_out[b] = (float)sd;
     done[b] = 0;
+    live[b] = b;                                  // every series starts unfinished
+    if (b == 0) *n_live = gridDim.x;
   }
 }
 
-// out[b, s] = hist[b, N + s / P, s % P] * sd + mean, s < H.   grid = B.
-__global__ void denorm_kernel(const float *__restrict__ hist, int N, int P, int cap, int H,
+// out[b, s] = hist[b, ctx_len + s] * sd + mean, s < H.   grid = B.
+__global__ void denorm_kernel(const float *__restrict__ hist, int ctx_len, int hist_len, int H,
                               const float *__restrict__ mean, const float *__restrict__ sd,
                               DevState *__restrict__ st) {
   const int b = blockIdx.x;
@@ -64,8 +90,25 @@ __global__ void denorm_kernel(const float *__restrict__ hist, int N, int P, int 
   float *out = st->out;
   if (b == 0 && threadIdx.x == 0) st->t_end = globaltimer_ns();
   const float m = mean[b], s = sd[b];
-  const float *hb = hist + ((size_t)b * cap + N) * P;
+  const float *hb = hist + (size_t)b * hist_len + ctx_len;
   for (int i = threadIdx.x; i < H; i += blockDim.x) out[(size_t)b * H + i] = hb[i] * s + m;
+}
+
+// Bounds-checking mode: every guard byte must still hold GUARD_BYTE after a forecast; the first
+// region found damaged is reported through the status word.  grid = (64, regions), block = 256.
+__global__ void guard_check_kernel(const GuardRegion *__restrict__ regions, int n, int *__restrict__ status) {
+  pdl_sync();
+  for (int k = blockIdx.y; k < n; k += gridDim.y) {
+    const GuardRegion r = regions[k];
+    const unsigned long long total = (unsigned long long)r.n_blocks * r.len;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (unsigned long long)gridDim.x * blockDim.x) {
+      if (r.base[(i / r.len) * r.stride + (i % r.len)] != GUARD_BYTE) {
+        atomicCAS(status, 0, DEV_GUARD_BASE + k);
+        break;
+      }
+    }
+  }
 }
 
 // 16-byte vector loads of T (8 bf16 or 4 fp32) unpacked to floats.
@@ -91,9 +134,10 @@ template <> struct Vec16<bf16> {
 };
 
 // ----------------------------------------------------------------------------------
-// Patch embedding x[row, f] = sum_i W_emb[f, i] * z[i], z = history token (fp32).
-// grid = (M rows, ceil(d / 128)), block = 128: one output feature per thread, its weight
-// row (P elements, a multiple of 16) read with independent 16-byte loads.
+// Token embedding x[row, f] = sum_i W_emb[f, i] * z[i], z = history token of P values (fp32;
+// P here is the input token length P_in).  grid = (M rows, ceil(d / 128)), block = 128: one
+// output feature per thread, its weight row read with independent 16-byte loads when P is a
+// multiple of the vector width, element by element for short tokens (point tokens: P = 1).
 // ----------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(128)
@@ -102,8 +146,10 @@ embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *
              const float *__restrict__ gain, T *__restrict__ a_out, float *__restrict__ ssq_out) {
   extern __shared__ float zs[];
   pdl_sync();
-  const int row = blockIdx.x, b = row / g.q_len, j = row % g.q_len;
+  const int row = blockIdx.x, slot = row / g.q_len, j = row % g.q_len;
   if (stamp && row == 0 && blockIdx.y == 0 && threadIdx.x == 0) *stamp = globaltimer_ns();
+  if (slot_dead(g, slot)) return;
+  const int b = series_of(g, slot);
   const float *z = hist + ((size_t)b * g.cap + pos0_of(g, b) + j) * P;
   for (int i = threadIdx.x; i < P; i += blockDim.x) zs[i] = z[i];
   __syncthreads();
@@ -112,12 +158,16 @@ embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *
   const T *wr = W + (size_t)f * P;
   constexpr int V = Vec16<T>::N;
   float acc = 0.f;
+  if (P % V == 0) {
 #pragma unroll 4
-  for (int i = 0; i < P; i += V) {
-    float w[V];
-    Vec16<T>::load(wr + i, w);
+    for (int i = 0; i < P; i += V) {
+      float w[V];
+      Vec16<T>::load(wr + i, w);
 #pragma unroll
-    for (int c = 0; c < V; ++c) acc = fmaf(w[c], zs[i + c], acc);
+      for (int c = 0; c < V; ++c) acc = fmaf(w[c], zs[i + c], acc);
+    }
+  } else {
+    for (int i = 0; i < P; ++i) acc = fmaf(to_f32(wr[i]), zs[i], acc);
   }
   x[(size_t)row * d + f] = acc;
   if (a_out) {            // operand of the first contraction, normalised later (see SkNorm); d % 32 == 0
@@ -138,11 +188,12 @@ embed_rows_kernel(const float *__restrict__ hist, PassGeom g, int M, int P, int 
   pdl_sync();
   const int row0 = blockIdx.x * R;
   if (stamp && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *stamp = globaltimer_ns();
+  if (slot_dead(g, row0 / g.q_len)) return;                   // every row of this CTA is past the live ones
   for (int i = threadIdx.x; i < R * P; i += blockDim.x) {
     const int row = row0 + i / P;
     float v = 0.f;
-    if (row < M) {
-      const int b = row / g.q_len, j = row % g.q_len;
+    if (row < M && !slot_dead(g, row / g.q_len)) {
+      const int b = series_of(g, row / g.q_len), j = row % g.q_len;
       v = hist[((size_t)b * g.cap + pos0_of(g, b) + j) * P + i % P];
     }
     zs[i] = v;
@@ -155,14 +206,22 @@ embed_rows_kernel(const float *__restrict__ hist, PassGeom g, int M, int P, int 
   float acc[R];
 #pragma unroll
   for (int r = 0; r < R; ++r) acc[r] = 0.f;
+  if (P % V == 0) {
 #pragma unroll 2
-  for (int i = 0; i < P; i += V) {
-    float w[V];
-    Vec16<T>::load(wr + i, w);
+    for (int i = 0; i < P; i += V) {
+      float w[V];
+      Vec16<T>::load(wr + i, w);
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+      for (int r = 0; r < R; ++r)
 #pragma unroll
-      for (int c = 0; c < V; ++c) acc[r] = fmaf(w[c], zs[r * P + i + c], acc[r]);
+        for (int c = 0; c < V; ++c) acc[r] = fmaf(w[c], zs[r * P + i + c], acc[r]);
+    }
+  } else {
+    for (int i = 0; i < P; ++i) {
+      const float w1 = to_f32(wr[i]);
+#pragma unroll
+      for (int r = 0; r < R; ++r) acc[r] = fmaf(w1, zs[r * P + i], acc[r]);
+    }
   }
 #pragma unroll
   for (int r = 0; r < R; ++r)
@@ -189,12 +248,12 @@ __device__ __forceinline__ void store4(bf16 *o, float a, float b, float c, float
 template <typename T>
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float *__restrict__ x, const float *__restrict__ gain, int M, int d, float eps,
-               T *__restrict__ a) {
+               T *__restrict__ a, LiveRows lr) {
   constexpr int CACHE = 16;                                   // float4 per lane kept in registers
   pdl_sync();
   const int lane = threadIdx.x & 31;
   const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (row >= (size_t)M) return;
+  if (row >= (size_t)live_rows(lr, M)) return;
   const float4 *xr = reinterpret_cast<const float4 *>(x + row * d);
   const float4 *gr = reinterpret_cast<const float4 *>(gain);
   const int nv = d / 4;
@@ -456,11 +515,13 @@ __global__ void __launch_bounds__(128)
 kv_append_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
                  const float2 *__restrict__ rope, PassGeom g, int n_heads) {
   constexpr int HALF = DH / 2;
-  const int h = blockIdx.x, b = blockIdx.y, d = n_heads * DH;
+  const int h = blockIdx.x, slot = blockIdx.y, d = n_heads * DH;
   pdl_sync();
+  if (slot_dead(g, slot)) return;
+  const int b = series_of(g, slot);
   const int p0 = pos0_of(g, b);
   const int j_lo = blockIdx.z * 16, j_hi = min(g.q_len, j_lo + 16);
-  const size_t row0 = (size_t)b * g.q_len;
+  const size_t row0 = (size_t)slot * g.q_len;
   T *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
   T *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;
   for (int i = threadIdx.x; i < (j_hi - j_lo) * (HALF / 2); i += blockDim.x) {
@@ -529,15 +590,17 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   float *row_max = po + 4 * ATTN_QT * DH;           // [ATTN_QT] maximum score over this CTA's keys
   float *row_sum = row_max + ATTN_QT;               // [ATTN_QT] sum of exp(score - row_max)
 
-  const int h = blockIdx.x, b = blockIdx.y;
+  const int h = blockIdx.x, slot = blockIdx.y;
   const int qt = skv > 1 ? blockIdx.z / skv : blockIdx.z;
   const int rank = skv > 1 ? blockIdx.z % skv : 0;   // == %cluster_ctarank: the cluster spans z only
   const int d = n_heads * DH;
   pdl_sync();
+  if (slot_dead(g, slot)) return;                    // the whole cluster (same y) leaves together
+  const int b = series_of(g, slot);
   const int p0 = pos0_of(g, b);
   const int j_lo = qt * QT;
   const int j_hi = min(g.q_len, j_lo + QT);          // queries [j_lo, j_hi)
-  const size_t row0 = (size_t)b * g.q_len;
+  const size_t row0 = (size_t)slot * g.q_len;
   const int nk_all = p0 + j_hi;                      // keys visible to the tile's last query
   const int chunk = skv > 1 ? (((nk_all + skv - 1) / skv + 15) & ~15) : nk_all;
   const int k_lo = min(rank * chunk, nk_all);        // this CTA holds keys [k_lo, k_hi) at rows t - k_lo
@@ -668,9 +731,11 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
 // Final RMSNorm + mean head for selected tokens: o = W_head[P, d] . (g_f * x * rstd).
 // Normalised activations stay fp32 here.  grid = (rows, ceil(P / 8)), block = 256: each warp
 // produces one output element with 16-byte weight loads.
-// only_last = 1: one row per series, the pass's last token, written to the series' next
-//   history slot hist[b, pos0 + q_len, :]  (draft steps, target-only steps);
-// only_last = 0: every token, written to vout[b, j, :]  (verification; vout [B, q_len, P]).
+// only_last = 1: one row per series, the pass's last token, written behind the pass in the
+//   series' history: the P values from token pos0 + q_len on (tok_len values per token)
+//   (draft steps, target-only steps);
+// only_last = 0: the boundary tokens head_step - 1, 2 head_step - 1, ... of the pass, boundary i
+//   written to vout[b, i, :]  (verification; vout [B, q_len / head_step, P]); grid.x = B * that.
 // ----------------------------------------------------------------------------------
 __device__ float head_normal(const DevState *st, int series, int k_pos, int e);   // accept.cuh
 
@@ -678,14 +743,18 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T *__restrict__ Wh, int d,
             int P, float eps, PassGeom g, int only_last, float *__restrict__ hist,
-            float *__restrict__ vout, const DevState *__restrict__ st, float *__restrict__ muq, int k_pos, int K) {
+            float *__restrict__ vout, const DevState *__restrict__ st, float *__restrict__ muq, int k_pos, int K,
+            int tok_len) {
   extern __shared__ __align__(16) float xs[];
   __shared__ float red[32];
   pdl_sync();
-  int b, j;
-  if (only_last) { b = blockIdx.x; j = g.q_len - 1; }
-  else { b = blockIdx.x / g.q_len; j = blockIdx.x % g.q_len; }
-  const float *xr = x + ((size_t)b * g.q_len + j) * d;
+  const int nb = g.q_len / g.head_step;                // boundaries per series
+  int slot, j, ib = 0;
+  if (only_last) { slot = blockIdx.x; j = g.q_len - 1; }
+  else { slot = blockIdx.x / nb; ib = blockIdx.x % nb; j = (ib + 1) * g.head_step - 1; }
+  if (slot_dead(g, slot)) return;
+  const int b = series_of(g, slot);
+  const float *xr = x + ((size_t)slot * g.q_len + j) * d;
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     const float v = xr[i];
@@ -695,8 +764,8 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
   const float rstd = rsqrtf(block_sum(ss, red) / d + eps);
   for (int i = threadIdx.x; i < d; i += blockDim.x) xs[i] = gain[i] * xs[i] * rstd;
   __syncthreads();
-  float *dst = only_last ? hist + ((size_t)b * g.cap + pos0_of(g, b) + g.q_len) * P
-                         : vout + ((size_t)b * g.q_len + j) * P;
+  float *dst = only_last ? hist + ((size_t)b * g.cap + pos0_of(g, b) + g.q_len) * tok_len
+                         : vout + ((size_t)b * nb + ib) * P;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int p = blockIdx.y * 8 + w;
   if (p >= P) return;
@@ -720,25 +789,29 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
   }
 }
 
-// The head for every token of a pass of many rows (verification: vout[b, j, :]): 8 rows per CTA
-// (one warp normalises one row into shared memory), then each warp produces 4 of the CTA's 32
-// outputs for all 8 rows, so that a weight vector is loaded once per 8 rows.
+// The head for the boundary tokens of a pass of many rows (verification: vout[b, i, :]): 8 rows
+// per CTA (one warp normalises one row into shared memory), then each warp produces 4 of the CTA's
+// 32 outputs for all 8 rows, so that a weight vector is loaded once per 8 rows.  M counts boundary
+// rows (series x boundaries per series).
 // grid = (ceil(M / 8), ceil(P / 32)), block = 256, dynamic shared memory 8 * d floats.
 template <typename T>
 __global__ void __launch_bounds__(256)
 head_rows_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T *__restrict__ Wh, int M,
-                 int d, int P, float eps, float *__restrict__ vout) {
+                 int d, int P, float eps, float *__restrict__ vout, PassGeom g) {
   constexpr int R = 8;
   extern __shared__ __align__(16) float xs[];                  // [R][d] normalised rows
   pdl_sync();
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int row0 = blockIdx.x * R;
+  const int nb = g.q_len / g.head_step;                        // boundaries per series
+  M = live_rows(LiveRows{g.n_live, nb}, M);
+  if (row0 >= M) return;
   {
     const int row = row0 + w;
     float *xw = xs + (size_t)w * d;
     float ss = 0.f;
     if (row < M) {
-      const float *xr = x + (size_t)row * d;
+      const float *xr = x + ((size_t)(row / nb) * g.q_len + (row % nb + 1) * g.head_step - 1) * d;
       for (int i = lane; i < d; i += 32) {
         const float v = xr[i];
         xw[i] = v;
@@ -770,7 +843,10 @@ head_rows_kernel(const float *__restrict__ x, const float *__restrict__ gain, co
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       const float o = warp_sum(acc[r]);
-      if (lane == 0 && row0 + r < M) vout[(size_t)(row0 + r) * P + p] = o;
+      if (lane == 0 && row0 + r < M) {                         // vout is indexed by series, rows by slot
+        const int row = row0 + r, b = series_of(g, row / nb);
+        vout[((size_t)b * nb + row % nb) * P + p] = o;
+      }
     }
   }
 }

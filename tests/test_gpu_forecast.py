@@ -116,6 +116,38 @@ def test_graph_and_stream_execution_give_identical_forecasts_and_traces():
         dec.close()
 
 
+@pytest.mark.parametrize("name", ["fp32", "bf16-small-M", "bf16-many-rows"])
+def test_compaction_of_finished_series_changes_nothing(name):
+    """Rounds run over the unfinished series only (slots of a compacted batch); with the flag that
+    switches this off every round runs over all series.  Series never interact, so forecasts,
+    decisions and counters must be the same -- bit for bit: a row's arithmetic does not depend on
+    where in the batch it sits."""
+    import paper_2511_18191_b200 as tsfm
+    if name == "fp32":
+        wl, K, tau = workload("C0", batch=7, series_recipe="c1", horizon=96 * 9 + 5), 3, 2.0
+    elif name == "bf16-small-M":
+        wl, K, tau = workload("C1", batch=12, horizon=96 * 10), 4, 2.0
+    else:      # enough rows for the large-tile contractions and the shared-load embedding / head kernels
+        wl, K, tau = workload("C3", draft_eps=1e-1, horizon=96 * 9, target=Arch(2, 256, 4, 512),
+                              draft=Arch(2, 256, 4, 512)), 4, 0.3
+    s, ctx = series_on_device(wl)
+    res = []
+    for mode in (tsfm.TSFM_EXEC_GRAPH, tsfm.TSFM_EXEC_GRAPH | tsfm.TSFM_EXEC_NO_COMPACT,
+                 tsfm.TSFM_EXEC_STREAM, tsfm.TSFM_EXEC_STREAM | tsfm.TSFM_EXEC_NO_COMPACT):
+        dec = make_decoder(wl, max_K=K, exec_mode=mode)[0]
+        out, st = dec.forecast(ctx, wl.horizon, K, tau, 5)
+        nacc, ell, logu = dec.last_trace(wl.batch, K)
+        d = st.as_dict()
+        res.append((out.cpu().numpy(), nacc, {k: d[k] for k in ("rounds", "proposals_tested", "proposals_accepted", "L_hist")}))
+        dec.close()
+    finished_at = (res[0][1] >= 0).sum(axis=0)                  # rounds each series took part in
+    assert finished_at.min() < finished_at.max(), "the case must desynchronise the batch"
+    for other in res[1:]:
+        np.testing.assert_array_equal(res[0][1], other[1])
+        np.testing.assert_array_equal(res[0][0], other[0])
+        assert res[0][2] == other[2]
+
+
 def test_launch_counter_counts_replayed_rounds():
     import paper_2511_18191_b200 as tsfm
     wl = workload("C0", batch=3, series_recipe="c1")
@@ -170,6 +202,25 @@ def test_c4_sixteen_series():
     wl = workload("C4")
     res = run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, spread(wl.batch, 16))
     assert res["series"] == 16
+
+
+def test_c5_point_tokens_every_series():
+    """The point-token family: input tokens of one step, a 64-step head, so a committed patch is 64
+    tokens and the verification pass over [pending, x_1..x_K] is read at every 64th token (the
+    prefix boundaries N - 1 + i P / P_in)."""
+    wl = workload("C5")
+    for mode in (1, 0):
+        res = run_and_compare(wl, wl.K, wl.tau, wl.forecast_seed, range(wl.batch), exec_mode=mode)
+    assert res["series"] == wl.batch
+
+
+@pytest.mark.parametrize("P,P_in,K,H", [(16, 4, 3, 16 * 5 + 3), (32, 16, 2, 32 * 4), (16, 1, 4, 16 * 3 + 1)])
+def test_short_input_tokens_fp32(P, P_in, K, H):
+    """Input tokens shorter than the patch on the fp32 path (several tokens per patch, with and
+    without the 16-byte embedding loads), ragged batch, truncated last patch."""
+    wl = workload("C0", batch=5, series_recipe="c1", patch_len=P, patch_in=P_in, ctx_len=P * 6, horizon=H)
+    for mode in (1, 0):
+        run_and_compare(wl, K, 2.0, 13, range(5), exec_mode=mode)
 
 
 @pytest.mark.parametrize("target,draft", [

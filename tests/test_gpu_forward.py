@@ -11,8 +11,9 @@ from tsfm_inputs import Arch, Workload, build_models
 pytestmark = pytest.mark.gpu
 
 
-def small_workload(dtype, target, draft, P=32, mode="separate"):
-    return Workload("T", 5, 8 * P, P, 4 * P, 3, 1.0, dtype, target, draft, mode, "c1", series_seed=77)
+def small_workload(dtype, target, draft, P=32, mode="separate", patch_in=0):
+    return Workload("T", 5, 8 * P, P, 4 * P, 3, 1.0, dtype, target, draft, mode, "c1", series_seed=77,
+                    patch_in=patch_in)
 
 
 def run_forward_case(wl, backend, n_tokens, B=5, seed=0):
@@ -21,9 +22,9 @@ def run_forward_case(wl, backend, n_tokens, B=5, seed=0):
     dec = tsfm.SpecDecoder(tw, dw, wl.target, wl.draft, wl.patch_len, wl.dtype,
                            "layer_skip" if wl.draft_mode == "layer_skip" else "separate",
                            max_batch=B, max_ctx_tokens=n_tokens, max_horizon_patches=4, max_K=4,
-                           gemm_backend=backend)
+                           gemm_backend=backend, patch_in=wl.patch_in)
     rng = np.random.default_rng(seed)
-    z = rng.standard_normal((B, n_tokens, wl.patch_len)).astype(np.float32)
+    z = rng.standard_normal((B, n_tokens, wl.token_len)).astype(np.float32)
     zt = torch.from_numpy(z).cuda()
     got_t = dec.model_forward(0, zt).cpu().numpy()
     got_d = dec.model_forward(1, zt).cpu().numpy()
@@ -61,6 +62,18 @@ def test_bf16_forward_matches_oracle(backend, target, draft, P, n, mode):
     gt, wt, gd, wd = run_forward_case(wl, backend, n)
     assert parity.value_error("rel_rms", gt, wt) < 2e-2
     assert parity.value_error("rel_rms", gd, wd) < 2e-2
+
+
+@pytest.mark.parametrize("dtype,P,P_in,n", [("f32", 16, 1, 70), ("f32", 32, 8, 19), ("bf16", 64, 1, 300), ("bf16", 32, 16, 40)])
+def test_forward_with_input_tokens_shorter_than_the_patch(dtype, P, P_in, n):
+    """Embedding of P_in-step tokens ([d, P_in] weights; 16-byte loads or element by element) under a
+    P-step head: next-patch means at every token."""
+    wl = small_workload(dtype, Arch(2, 128, 2, 256), Arch(1, 64, 2, 128), P, patch_in=P_in)
+    gt, wt, gd, wd = run_forward_case(wl, 0, n, B=3)
+    if dtype == "f32":
+        assert np.abs(gt - wt).max() < 1e-4 and np.abs(gd - wd).max() < 1e-4
+    else:
+        assert parity.value_error("rel_rms", gt, wt) < 2e-2 and parity.value_error("rel_rms", gd, wd) < 2e-2
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 128, 64), (16, 128, 64), (32, 1536, 512), (160, 512, 2048), (33, 96, 128),
