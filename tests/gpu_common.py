@@ -2,6 +2,7 @@
 from __future__ import annotations
 
 import functools
+import os
 
 import numpy as np
 import torch
@@ -18,6 +19,9 @@ def _models(wl_key):
 
 
 def make_decoder(wl, backend=tsfm.TSFM_GEMM_AUTO, max_K=None, batch=None, exec_mode=tsfm.TSFM_EXEC_GRAPH):
+    # TSFM_TEST_CHECK_BOUNDS=1 runs every test of the suite in the decoder's bounds-checking mode
+    if os.environ.get("TSFM_TEST_CHECK_BOUNDS") == "1":
+        exec_mode |= tsfm.TSFM_EXEC_CHECK_BOUNDS
     tw, dw = _models(wl.with_(batch=1, horizon=wl.patch_len, K=1, tau=1.0, ctx_len=2 * wl.patch_len, series_recipe="c1",
                               series_seed=0, forecast_seed=0, K_sweep=(), tau_sweep=(), eps_sweep=()))
     dec = tsfm.SpecDecoder.for_workload(wl, tw, dw, max_K=max_K, batch=batch, gemm_backend=backend,

@@ -148,6 +148,65 @@ def test_compaction_of_finished_series_changes_nothing(name):
         assert res[0][2] == other[2]
 
 
+BOUNDS_CASES = {
+    "fp32-ragged": lambda: (workload("C0", batch=6, series_recipe="c1", horizon=96 * 7 + 5), 4, 4.0),
+    "bf16-small-M": lambda: (workload("C1", batch=12, horizon=96 * 10), 4, 2.0),
+    "bf16-K-beyond-a-tile": lambda: (workload("C1", batch=4, horizon=96 * 6), 20, 2.0),
+    "bf16-long-rows": lambda: (workload("C4", batch=3, horizon=32 * 11 + 7, target=Arch(2, 256, 4, 512),
+                                        draft=Arch(1, 128, 2, 256)), 8, 1.0),
+    "bf16-many-rows": lambda: (workload("C3", draft_eps=1e-1, horizon=96 * 5, target=Arch(2, 256, 4, 512),
+                                        draft=Arch(2, 256, 4, 512)), 4, 0.3),
+    "bf16-point-tokens": lambda: (workload("C5", batch=5, horizon=64 * 3 + 9), 3, 1.0),
+}
+
+
+@pytest.mark.parametrize("name", sorted(BOUNDS_CASES))
+def test_bounds_checking_mode_finds_no_write_outside_any_buffer(name):
+    """In bounds-checking mode every buffer has guard bytes behind it and every (layer, series, head)
+    block of the KV caches and every series' history a spare last token; a kernel inspects them after
+    each call.  Representative forecasts (ragged positions, full rollbacks, K + 1 beyond one query
+    tile, rows of 300 tokens, 1024 series, point tokens), in both execution modes, leave them intact,
+    and give the same numbers as the ordinary mode."""
+    import paper_2511_18191_b200 as tsfm
+    wl, K, tau = BOUNDS_CASES[name]()
+    s, ctx = series_on_device(wl)
+    outs = []
+    for mode in (tsfm.TSFM_EXEC_GRAPH, tsfm.TSFM_EXEC_GRAPH | tsfm.TSFM_EXEC_CHECK_BOUNDS,
+                 tsfm.TSFM_EXEC_STREAM | tsfm.TSFM_EXEC_CHECK_BOUNDS):
+        dec = make_decoder(wl, max_K=K, exec_mode=mode)[0]
+        checked = bool(mode & tsfm.TSFM_EXEC_CHECK_BOUNDS)
+        assert (tsfm.tsfm_spec_debug_guard(dec.h) > 20) == checked
+        out, st = dec.forecast(ctx, wl.horizon, K, tau, 3)           # raises if a guard is damaged
+        assert st.device_status == 0
+        ref, st_t = dec.target_only(ctx, wl.horizon)
+        dro, st_d = dec.draft_only(ctx, wl.horizon)
+        assert st_t.device_status == 0 and st_d.device_status == 0
+        outs.append((out.cpu().numpy(), ref.cpu().numpy(), dro.cpu().numpy()))
+        dec.close()
+    for other in outs[1:]:
+        for a, b in zip(outs[0], other):
+            np.testing.assert_array_equal(a, b)
+
+
+def test_a_damaged_guard_is_reported_by_name_and_the_handle_recovers():
+    """The checker itself: one byte of a guard region overwritten from the host (a write inside the
+    library's own allocation) makes the next call fail with the buffer's name; restored, calls succeed."""
+    import paper_2511_18191_b200 as tsfm
+    wl = workload("C0", batch=2, series_recipe="c1")
+    dec = make_decoder(wl, exec_mode=tsfm.TSFM_EXEC_GRAPH | tsfm.TSFM_EXEC_CHECK_BOUNDS)[0]
+    s, ctx = series_on_device(wl)
+    n = tsfm.tsfm_spec_debug_guard(dec.h)
+    dec.forecast(ctx, wl.horizon, wl.K, 1.0, 1)
+    for region in (0, n // 2, n - 1):
+        tsfm.tsfm_spec_debug_guard(dec.h, region, damage=True)
+        with pytest.raises(tsfm.TsfmError) as e:
+            dec.forecast(ctx, wl.horizon, wl.K, 1.0, 1)
+        assert e.value.code == tsfm.TSFM_ERR_INTERNAL and f"guard region {region})" in str(e.value)
+        tsfm.tsfm_spec_debug_guard(dec.h, region, damage=False)
+        dec.forecast(ctx, wl.horizon, wl.K, 1.0, 1)
+    dec.close()
+
+
 def test_launch_counter_counts_replayed_rounds():
     import paper_2511_18191_b200 as tsfm
     wl = workload("C0", batch=3, series_recipe="c1")
