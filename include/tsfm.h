@@ -57,6 +57,10 @@ extern "C" {
 
 #define TSFM_GEMM_AUTO  0       /* bf16 contractions on tcgen05 tensor cores where shapes allow     */
 #define TSFM_GEMM_SIMT  1       /* force the plain FMA kernels everywhere (differential reference)  */
+#define TSFM_GEMM_WS    2       /* tsfm_gemm_bf16 only: the small-batch kernel that keeps its weight
+                                   tile in shared memory (TSFM_ERR_SHAPE outside its domain: at most
+                                   256 tokens, K a multiple of 64 up to 2048, grid within one wave);
+                                   a decoder picks it by itself where it applies                   */
 
 #define TSFM_EXEC_GRAPH   0       /* a forecast is one CUDA-graph launch: prologue, a device-side WHILE
                                    over the rounds, de-normalisation; no host round trip             */
@@ -260,8 +264,8 @@ int tsfm_model_forward(tsfm_spec *h, int32_t which, const float *tokens, int32_t
                        float *out);
 
 /* C[M, N] = A[M, Kd] * W[N, Kd]^T with bf16 operands and fp32 accumulation, through the
- * tensor-core kernel (backend TSFM_GEMM_AUTO) or the FMA kernel (TSFM_GEMM_SIMT); for
- * differential tests of the contraction.  A, W dev bf16 row-major; C dev fp32 row-major. */
+ * tensor-memory kernel (backend TSFM_GEMM_AUTO), the FMA kernel (TSFM_GEMM_SIMT) or the small-batch
+ * kernel (TSFM_GEMM_WS); for differential tests of the contraction.  A, W dev bf16 row-major; C dev fp32 row-major. */
 int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C,
                    int32_t M, int32_t N, int32_t Kd, int32_t backend);
 

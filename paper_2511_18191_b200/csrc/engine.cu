@@ -4,6 +4,7 @@
 #include "../../include/tsfm.h"
 
 #include <cuda_runtime.h>
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
@@ -21,6 +22,7 @@
 #include "accept.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_sk.cuh"
+#include "gemm_ws.cuh"
 
 using namespace tsfm;
 
@@ -136,7 +138,7 @@ struct tsfm_spec {
   ModelDev tgt, drf;
   // activations (sized for M_max rows)
   int M_max = 0;
-  float *x = nullptr, *qkv = nullptr, *ssq = nullptr;   // ssq: [M_max][d / 32] slice sums of squares
+  float *x = nullptr, *qkv = nullptr, *ssq = nullptr;   // ssq: [M_max][d / 16] slice sums of squares
   void *a = nullptr, *ao = nullptr, *hbuf = nullptr;
   // decoding state
   float *hist = nullptr, *vout = nullptr, *mean = nullptr, *sd = nullptr;
@@ -173,10 +175,11 @@ namespace {
 // Kernel classes for per-launch timing.
 // The tensor-core contraction is one kernel in three regimes: up to 512 tokens it streams weights
 // (HBM / latency bound), from 4096 tokens it is tensor bound, between them it is one wave of tiles.
-enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_TC_SMALL, KC_GEMM_TC_MID, KC_GEMM_TC_LARGE, KC_GEMM_SIMT,
+enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_WS, KC_GEMM_TC_SMALL, KC_GEMM_TC_MID, KC_GEMM_TC_LARGE, KC_GEMM_SIMT,
        KC_ATTN, KC_HEAD, KC_ACCEPT, KC_DENORM, KC_COUNT };
-const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_sk_small_M", "gemm_sk_mid_M",
-                                            "gemm_sk_large_M", "gemm_simt", "attn", "head", "accept", "denorm"};
+const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_ws_small_M", "gemm_sk_small_M",
+                                            "gemm_sk_mid_M", "gemm_sk_large_M", "gemm_simt", "attn", "head", "accept",
+                                            "denorm"};
 
 // Brackets one launch with two events when profiling is on (no-op otherwise).
 struct KTimer {
@@ -299,6 +302,12 @@ int attn_set_attr(size_t bytes) {
 // Short rows with at least this many (series, head) pairs: one warp per pair instead of four
 // (measured: C2's draft, 1024 pairs, 15 % faster that way; no difference at 256 pairs).
 constexpr int kFlashWarpMaxCap = 64, kFlashWarpMinPairs = 512;
+// Long rows with at least this many pairs take one warp per pair too: split four ways, a CTA's life
+// is one pipeline fill (positions -> copies -> scores -> merge) and 1280 CTAs at three per SM need
+// three such fills in a row; 1280 warps at twelve per SM are one wave, each streaming its whole row
+// through its ring (measured on C4's verification pass and decode step: attention 51.7 -> 47.2 ms
+// per forecast).
+constexpr int kFlashWarpLongMinPairs = 1024;
 // one-tile passes: a two-stage ring (each warp has a few chunks only, and a third CTA fits on the SM)
 constexpr int kFlashStShort = 2;
 template <int DH> int flash_set_attr() {
@@ -358,6 +367,9 @@ void prefer_max_smem_all() {
   prefer_max_smem(gemm_sk_kernel<1, false>);
   prefer_max_smem(gemm_sk_kernel<1, true>);
   prefer_max_smem(gemm_sk_kernel<2, false>);
+  prefer_max_smem(gemm_sk_kernel<2, true>);
+  prefer_max_smem(gemm_ws_kernel<false>);
+  prefer_max_smem(gemm_ws_kernel<true>);
   prefer_max_smem(attn_flash_kernel<32, 3>);
   prefer_max_smem(attn_flash_kernel<32, kFlashStShort>);
   prefer_max_smem(attn_flash_kernel<64, 3>);
@@ -433,6 +445,17 @@ void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C,
   const double out_b = (epi == EPI_F32 || epi == EPI_ATOMIC) ? 4.0 : epi == EPI_RESID ? 8.0 : e;
   const double bytes = ((double)N * K + (double)M * K) * e + (double)M * N * out_b;
   const double flops = 2.0 * M * N * K;
+  if (sizeof(T) == 2 && h->use_tc && plan && plan->valid && !(norm && norm->use_tma) && gemm_ws_eligible(A, W, M, N, K)) {
+    // few tokens, short K: the shared-memory-resident weight tile kernel has the shorter chain
+    KTimer kt(h, KC_GEMM_WS, bytes, flops);
+    if (gemm_ws_launch(h->ls, h->pdl, A, W, C, M, N, K, epi, norm, lr)) {
+      LAUNCHED();
+    } else if (h->enqueue_err == TSFM_OK) {
+      h->enqueue_err = TSFM_ERR_CUDA;
+      g_cuda_err = std::string("small-batch contraction could not be launched: ") + cudaGetErrorString(cudaGetLastError());
+    }
+    return;
+  }
   if (sizeof(T) == 2 && h->use_tc && plan && plan->valid) {
     KTimer kt(h, M <= 512 ? KC_GEMM_TC_SMALL : M < 4096 ? KC_GEMM_TC_MID : KC_GEMM_TC_LARGE, bytes, flops);
     if (gemm_sk_launch(h->ls, h->pdl, *plan, C, M, epi, h->dev_status, norm, lr)) {
@@ -466,7 +489,8 @@ void launch_attn(tsfm_spec *h, ModelDev &m, int l, int B, const PassGeom &g) {
   if constexpr (sizeof(T) == 2) {
     const int pairs = B * m.arch.n_heads;
     const int mode = pre ? FLASH_TILES
-                         : (h->cap <= kFlashWarpMaxCap && pairs >= kFlashWarpMinPairs) ? FLASH_WARP : FLASH_SPLIT;
+                         : ((h->cap <= kFlashWarpMaxCap && pairs >= kFlashWarpMinPairs) || pairs >= kFlashWarpLongMinPairs)
+                               ? FLASH_WARP : FLASH_SPLIT;
     const dim3 grid = mode == FLASH_WARP ? dim3((pairs + 3) / 4)
                                          : dim3(m.arch.n_heads, B, pre ? (g.q_len + 4 * ATTN_QT - 1) / (4 * ATTN_QT) : 1);
     // short caches: one stage of 32 or 64 rows per warp instead of the ring, more warps per SM
@@ -520,7 +544,13 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   // rows' slice sums of squares; whoever consumes a' scales its result rows by rstd.
   // (Only for passes of few tokens, where a launch costs more than the extra epilogue work: with
   // large tiles the epilogue is the bottleneck and the separate RMSNorm kernel is the cheaper way.)
-  const bool fold = sizeof(T) == 2 && h->use_tc && m.layers[0].tc_qkv.valid && M <= 512;
+  const bool tc = sizeof(T) == 2 && h->use_tc && m.layers[0].tc_qkv.valid;
+  const bool fold = tc && M <= 512;
+  // Larger passes fold the norms too, in the form that keeps the TMA epilogues of the large tiles
+  // (see gemm_sk.cuh): every RMSNorm but the first one of the pass disappears into the contractions.
+  // (Up to a few thousand rows: beyond that the RMSNorm kernel runs at memory speed and the read-back
+  // in the producers' epilogues costs more than it saves -- measured on C4's prefill, 23.6 -> 25.0 ms.)
+  const bool fold_tma = tc && M > 512 && M < 4096 && d % 128 == 0;
   const int L = m.arch.n_layers;
   const LiveRows lr{g.n_live, g.q_len};
   {
@@ -536,16 +566,19 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
   SkNorm consume{};                 // scale the result rows by rstd of the input rows
   consume.ssq_in = h->ssq;
-  consume.n_part = d / 32;
+  consume.n_part = fold_tma ? d / 128 : d / 16;
   consume.inv_d = 1.f / d;
   consume.eps = eps;
+  consume.use_tma = fold_tma;
+  const bool any_fold = fold || fold_tma;
   for (int l = 0; l < L; ++l) {
     LayerDev &ly = m.layers[l];
-    if (!fold) {
+    const bool norm1_kernel = !fold && !(fold_tma && l > 0);    // first norm of the layer as a kernel of its own
+    if (norm1_kernel) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
       launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g1, M, d, eps, (T *)h->a, lr);
     }
-    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr, lr);
+    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, norm1_kernel ? nullptr : &consume, lr);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
     else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
     else launch_attn<T, 128>(h, m, l, B, g);
@@ -554,15 +587,16 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     produce.ssq_out = h->ssq;
     produce.a_out = (bf16 *)h->a;
     produce.gain = ly.g2;
-    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, fold ? &produce : nullptr, lr);
-    if (!fold) {
+    produce.use_tma = fold_tma;
+    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, any_fold ? &produce : nullptr, lr);
+    if (!any_fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
       launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g2, M, d, eps, (T *)h->a, lr);
     }
-    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, fold ? &consume : nullptr, lr);
+    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, any_fold ? &consume : nullptr, lr);
     produce.gain = l + 1 < L ? m.layers[l + 1].g1 : nullptr;
     if (l + 1 == L) produce.a_out = nullptr, produce.ssq_out = nullptr;   // the head kernel norms the final rows itself
-    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID, fold && l + 1 < L ? &produce : nullptr, lr);
+    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID, any_fold && l + 1 < L ? &produce : nullptr, lr);
   }
   const int Mb = B * (g.q_len / g.head_step);          // boundary rows the head reads (verification)
   const double rows = head_mode == HEAD_LAST_TO_HIST ? B : Mb;
@@ -1004,7 +1038,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   const size_t Mx = h->M_max;
   if ((rc = dev_alloc(h, &h->x, Mx * dmax, "x"))) return fail(rc);
   if ((rc = dev_alloc(h, &h->qkv, Mx * 3 * dmax, "qkv"))) return fail(rc);
-  if ((rc = dev_alloc(h, &h->ssq, Mx * (dmax / 32 + 1), "ssq"))) return fail(rc);
+  if ((rc = dev_alloc(h, &h->ssq, Mx * (dmax / 16 + 1), "ssq"))) return fail(rc);
   if ((rc = dev_alloc(h, (char **)&h->a, Mx * dmax * e, "a"))) return fail(rc);
   if ((rc = dev_alloc(h, (char **)&h->ao, Mx * dmax * e, "ao"))) return fail(rc);
   if ((rc = dev_alloc(h, (char **)&h->hbuf, Mx * fmax * e, "hbuf"))) return fail(rc);
@@ -1053,6 +1087,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   prefer_max_smem_all();
   if (h->use_tc) {
     if ((rc = gemm_sk_init())) return fail(rc);
+    if ((rc = gemm_ws_init())) return fail(rc);
     for (ModelDev *m : {&h->tgt, &h->drf}) {
       const int d = m->arch.d_model, f = m->arch.d_ff;
       for (LayerDev &ly : m->layers) {
@@ -1269,6 +1304,14 @@ int tsfm_gemm_bf16(void *stream, const void *A, const void *W, float *C, int32_t
   cudaStream_t s = (cudaStream_t)stream;
   if (backend == TSFM_GEMM_SIMT) {
     launch_gemm_simt<bf16>(s, false, (const bf16 *)A, (const bf16 *)W, C, M, N, Kd, EPI_F32);
+    CU_TRY(cudaGetLastError());
+    return TSFM_OK;
+  }
+  if (backend == TSFM_GEMM_WS) {
+    if (!gemm_ws_eligible(A, W, M, N, Kd)) return TSFM_ERR_SHAPE;
+    if (int rc = gemm_ws_init()) return rc;
+    if (!gemm_ws_launch(s, false, A, W, C, M, N, Kd, EPI_F32, nullptr, LiveRows{nullptr, 0})) CU_TRY(cudaGetLastError());
+    LAUNCHED();
     CU_TRY(cudaGetLastError());
     return TSFM_OK;
   }

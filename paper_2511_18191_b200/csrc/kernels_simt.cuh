@@ -170,10 +170,14 @@ embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *
     for (int i = 0; i < P; ++i) acc = fmaf(to_f32(wr[i]), zs[i], acc);
   }
   x[(size_t)row * d + f] = acc;
-  if (a_out) {            // operand of the first contraction, normalised later (see SkNorm); d % 32 == 0
+  if (a_out) {            // operand of the first contraction, normalised later (see SkNorm); d % 64 == 0
     a_out[(size_t)row * d + f] = from_f32<T>(gain[f] * acc);
-    const float sq = warp_sum(acc * acc);
-    if ((threadIdx.x & 31) == 0) ssq_out[(size_t)row * (d >> 5) + (f >> 5)] = sq;
+    float sq = acc * acc;                                       // sums of squares over slices of 16 features
+    sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+    sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+    sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+    sq += __shfl_xor_sync(0xffffffffu, sq, 8);
+    if ((threadIdx.x & 15) == 0) ssq_out[(size_t)row * (d >> 4) + (f >> 4)] = sq;
   }
 }
 

@@ -26,8 +26,9 @@ def run_gemm(a):
     Ws = [(torch.randn((a.N, a.K), generator=g) / a.K ** 0.5).to(torch.bfloat16).cuda() for _ in range(n_w)]
     C = torch.empty((a.M, a.N), device="cuda")
     s = torch.cuda.current_stream().cuda_stream
+    backend = tsfm.TSFM_GEMM_WS if a.backend == "ws" else tsfm.TSFM_GEMM_AUTO
     for i in range(a.reps):
-        tsfm.tsfm_gemm_bf16(s, A, Ws[i % n_w], C, a.M, a.N, a.K, tsfm.TSFM_GEMM_AUTO)
+        tsfm.tsfm_gemm_bf16(s, A, Ws[i % n_w], C, a.M, a.N, a.K, backend)
     torch.cuda.synchronize()
     print(f"gemm M={a.M} N={a.N} K={a.K}: {a.reps} launches over {n_w} weight matrices, "
           f"checksum {float(C.double().sum()):.6g}")
@@ -80,6 +81,8 @@ def main(argv=None):
     g.add_argument("--K", type=int, required=True)
     g.add_argument("--reps", type=int, default=3)
     g.add_argument("--ring", type=int, default=1, help="number of distinct weight matrices cycled through")
+    g.add_argument("--backend", default="auto", choices=["auto", "ws"],
+                   help="auto: tensor-memory kernel; ws: the small-batch kernel with a resident weight tile")
     f = sub.add_parser("forecast")
     f.add_argument("--workload", default="C1")
     f.add_argument("--mode", default="spec", choices=["spec", "target_only"])

@@ -94,3 +94,28 @@ def test_tensor_core_gemm_matches_fp64_product_and_fma_kernel(M, N, K):
         assert np.isfinite(outs[name]).all(), name
         assert np.abs(outs[name] - want).max() < 2e-5 * K ** 0.5 + 1e-5, name
     assert np.abs(outs["tc"] - outs["simt"]).max() < 2e-5 * K ** 0.5 + 1e-5
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 128, 64), (16, 130, 64), (32, 1536, 512), (33, 96, 128), (40, 512, 192), (64, 384, 1536),
+                                   (128, 1152, 384), (31, 512, 2048), (256, 66, 448), (160, 1536, 512)])
+def test_small_batch_gemm_matches_fp64_product(M, N, K):
+    """The kernel that keeps its weight tile in shared memory (few tokens, K up to 2048): ragged token
+    and feature tiles, every k step distribution over its eight warps, and the refusal outside its domain."""
+    import paper_2511_18191_b200 as tsfm
+    g = torch.Generator(device="cpu").manual_seed(M * 11 + N)
+    A = torch.randn((M, K), generator=g).to(torch.bfloat16)
+    W = (torch.randn((N, K), generator=g) / K ** 0.5).to(torch.bfloat16)
+    Ad, Wd = A.cuda(), W.cuda()
+    Cd = torch.full((M, N), float("nan"), device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    if (M, N, K) == (160, 1536, 512):                     # 480 CTAs: more than one wave, not this kernel's job
+        with pytest.raises(tsfm.TsfmError) as e:
+            tsfm.tsfm_gemm_bf16(s, Ad, Wd, Cd, M, N, K, tsfm.TSFM_GEMM_WS)
+        assert e.value.code == tsfm.TSFM_ERR_SHAPE
+        return
+    tsfm.tsfm_gemm_bf16(s, Ad, Wd, Cd, M, N, K, tsfm.TSFM_GEMM_WS)
+    torch.cuda.synchronize()
+    got = Cd.cpu().numpy()
+    want = (A.double() @ W.double().T).numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - want).max() < 2e-5 * K ** 0.5 + 1e-5
