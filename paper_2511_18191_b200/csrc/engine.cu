@@ -367,7 +367,6 @@ void prefer_max_smem_all() {
   prefer_max_smem(gemm_sk_kernel<1, false>);
   prefer_max_smem(gemm_sk_kernel<1, true>);
   prefer_max_smem(gemm_sk_kernel<2, false>);
-  prefer_max_smem(gemm_sk_kernel<2, true>);
   prefer_max_smem(gemm_ws_kernel<false>);
   prefer_max_smem(gemm_ws_kernel<true>);
   prefer_max_smem(attn_flash_kernel<32, 3>);
@@ -445,7 +444,7 @@ void gemm(tsfm_spec *h, GemmSkPlan *plan, const void *A, const void *W, void *C,
   const double out_b = (epi == EPI_F32 || epi == EPI_ATOMIC) ? 4.0 : epi == EPI_RESID ? 8.0 : e;
   const double bytes = ((double)N * K + (double)M * K) * e + (double)M * N * out_b;
   const double flops = 2.0 * M * N * K;
-  if (sizeof(T) == 2 && h->use_tc && plan && plan->valid && !(norm && norm->use_tma) && gemm_ws_eligible(A, W, M, N, K)) {
+  if (sizeof(T) == 2 && h->use_tc && plan && plan->valid && gemm_ws_eligible(A, W, M, N, K)) {
     // few tokens, short K: the shared-memory-resident weight tile kernel has the shorter chain
     KTimer kt(h, KC_GEMM_WS, bytes, flops);
     if (gemm_ws_launch(h->ls, h->pdl, A, W, C, M, N, K, epi, norm, lr)) {
@@ -544,13 +543,13 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   // rows' slice sums of squares; whoever consumes a' scales its result rows by rstd.
   // (Only for passes of few tokens, where a launch costs more than the extra epilogue work: with
   // large tiles the epilogue is the bottleneck and the separate RMSNorm kernel is the cheaper way.)
-  const bool tc = sizeof(T) == 2 && h->use_tc && m.layers[0].tc_qkv.valid;
-  const bool fold = tc && M <= 512;
-  // Larger passes fold the norms too, in the form that keeps the TMA epilogues of the large tiles
-  // (see gemm_sk.cuh): every RMSNorm but the first one of the pass disappears into the contractions.
-  // (Up to a few thousand rows: beyond that the RMSNorm kernel runs at memory speed and the read-back
-  // in the producers' epilogues costs more than it saves -- measured on C4's prefill, 23.6 -> 25.0 ms.)
-  const bool fold_tma = tc && M > 512 && M < 4096 && d % 128 == 0;
+  // On the bf16 path the RMSNorms of passes of up to 512 tokens are folded into the contractions
+  // around them (SkNorm): whoever produces the residual stream also writes the next operand
+  // a' = bf16(gain * x) and the rows' sums of squares over 16-feature slices; whoever consumes a'
+  // scales its result rows by rstd.  (Only for few tokens, where a launch costs more than the extra
+  // epilogue work.  With the large tiles' TMA epilogues a producer would have to load its block of x
+  // back after the reduction: measured on C2-C4, that costs what the RMSNorm kernel costs.)
+  const bool fold = sizeof(T) == 2 && h->use_tc && m.layers[0].tc_qkv.valid && M <= 512;
   const int L = m.arch.n_layers;
   const LiveRows lr{g.n_live, g.q_len};
   {
@@ -566,19 +565,16 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
   SkNorm consume{};                 // scale the result rows by rstd of the input rows
   consume.ssq_in = h->ssq;
-  consume.n_part = fold_tma ? d / 128 : d / 16;
+  consume.n_part = d / 16;
   consume.inv_d = 1.f / d;
   consume.eps = eps;
-  consume.use_tma = fold_tma;
-  const bool any_fold = fold || fold_tma;
   for (int l = 0; l < L; ++l) {
     LayerDev &ly = m.layers[l];
-    const bool norm1_kernel = !fold && !(fold_tma && l > 0);    // first norm of the layer as a kernel of its own
-    if (norm1_kernel) {
+    if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
       launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g1, M, d, eps, (T *)h->a, lr);
     }
-    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, norm1_kernel ? nullptr : &consume, lr);
+    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr, lr);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
     else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
     else launch_attn<T, 128>(h, m, l, B, g);
@@ -587,28 +583,35 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     produce.ssq_out = h->ssq;
     produce.a_out = (bf16 *)h->a;
     produce.gain = ly.g2;
-    produce.use_tma = fold_tma;
-    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, any_fold ? &produce : nullptr, lr);
-    if (!any_fold) {
+    gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, fold ? &produce : nullptr, lr);
+    if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
       launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g2, M, d, eps, (T *)h->a, lr);
     }
-    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, any_fold ? &consume : nullptr, lr);
+    gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, fold ? &consume : nullptr, lr);
     produce.gain = l + 1 < L ? m.layers[l + 1].g1 : nullptr;
     if (l + 1 == L) produce.a_out = nullptr, produce.ssq_out = nullptr;   // the head kernel norms the final rows itself
-    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID, any_fold && l + 1 < L ? &produce : nullptr, lr);
+    gemm<T>(h, &ly.tc_2, h->hbuf, ly.W2, h->x, M, d, f, EPI_RESID, fold && l + 1 < L ? &produce : nullptr, lr);
   }
   const int Mb = B * (g.q_len / g.head_step);          // boundary rows the head reads (verification)
   const double rows = head_mode == HEAD_LAST_TO_HIST ? B : Mb;
   KTimer kt(h, head_mode == HEAD_NONE ? -1 : KC_HEAD, rows * d * 4 + (double)P * d * sizeof(T) + rows * P * 4,
             2.0 * rows * P * d);
-  if (head_mode == HEAD_LAST_TO_HIST) {
+  const bool rows_fit = (size_t)8 * d * sizeof(float) <= 200 * 1024;
+  if (head_mode == HEAD_LAST_TO_HIST && B >= kManyRows && rows_fit) {
+    PassGeom gl = g;                                    // one boundary per series: the pass's last token
+    gl.head_step = g.q_len;
+    launch_ex(s, h->pdl, head_rows_kernel<T>, dim3((B + 7) / 8, (P + 31) / 32), dim3(256), (size_t)8 * d * sizeof(float),
+              h->x, m.g_f, (const T *)m.W_head, B, d, P, eps, (float *)nullptr, gl, h->hist, Pi,
+              ds.k_pos >= 0 ? (const DevState *)h->st : (const DevState *)nullptr, h->muq, ds.k_pos, ds.K);
+  } else if (head_mode == HEAD_LAST_TO_HIST) {
     launch_ex(s, h->pdl, head_kernel<T>, dim3(B, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
               (const T *)m.W_head, d, P, eps, g, 1, h->hist, (float *)nullptr,
               ds.k_pos >= 0 ? (const DevState *)h->st : (const DevState *)nullptr, h->muq, ds.k_pos, ds.K, Pi);
-  } else if (head_mode == HEAD_ALL_TO_VOUT && Mb >= kManyRows && (size_t)8 * d * sizeof(float) <= 200 * 1024) {
+  } else if (head_mode == HEAD_ALL_TO_VOUT && Mb >= kManyRows && rows_fit) {
     launch_ex(s, h->pdl, head_rows_kernel<T>, dim3((Mb + 7) / 8, (P + 31) / 32), dim3(256), (size_t)8 * d * sizeof(float),
-              h->x, m.g_f, (const T *)m.W_head, Mb, d, P, eps, vout, g);
+              h->x, m.g_f, (const T *)m.W_head, Mb, d, P, eps, vout, g, (float *)nullptr, Pi, (const DevState *)nullptr,
+              (float *)nullptr, 0, 0);
   } else if (head_mode == HEAD_ALL_TO_VOUT) {
     launch_ex(s, h->pdl, head_kernel<T>, dim3(Mb, (P + 7) / 8), dim3(256), d * sizeof(float), h->x, m.g_f,
               (const T *)m.W_head, d, P, eps, g, 0, (float *)nullptr, vout, (const DevState *)nullptr, (float *)nullptr, 0, 0,

@@ -47,12 +47,11 @@ __host__ __device__ constexpr uint32_t umma_idesc_rt(int bn) {
 // that CONSUMES a' multiplies its result rows by rstd = rsqrt(sum of the slices / d + eps).
 struct SkNorm {
   const float *ssq_in;      // [M][n_part] slice sums of squares of this contraction's input rows, or NULL
-  float *ssq_out;           // [M][N / 16] (N / 128 in the TMA form) written by a residual epilogue, or NULL
+  float *ssq_out;           // [M][N / 16] written by a residual epilogue, or NULL
   const float *gain;        // [N] gain of the norm that follows the residual epilogue
   bf16 *a_out;              // [M][N] bf16(gain * x_new), or NULL
-  int n_part;               // partial sums per input row (d / 16; d / 128 in the TMA form)
+  int n_part;               // partial sums per input row (d / 16)
   float inv_d, eps;
-  int use_tma;              // keep the TMA epilogues (large tiles): see "folded norm, TMA form" below
 };
 
 struct SkShape {
@@ -60,7 +59,7 @@ struct SkShape {
 };
 // Ring of `stages` x (W tile 16 KB + A tile BN x 128 B); the partial-sum tile (BN x 128 fp32)
 // reuses the ring once the accumulator is complete.
-static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1, bool bf16_copy = false) {
+static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1) {
   SkShape s;
   s.BN = BN;
   const int stage = TC_W_BYTES * wt + BN * TC_BK * 2;
@@ -68,7 +67,6 @@ static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1, b
   if (stages > kb_per_cta) stages = kb_per_cta < 1 ? 1 : kb_per_cta;
   int bytes = stages * stage;
   if (split && bytes < BN * TC_BM * 4) bytes = BN * TC_BM * 4;
-  if (bf16_copy && bytes < BN * TC_BM * 6) bytes = BN * TC_BM * 6;   // + the bf16 copy of the tile (folded norm, TMA form)
   s.stages = stages;
   const int cols = BN * wt;
   s.tmem_cols = cols <= 32 ? 32 : cols <= 64 ? 64 : cols <= 128 ? 128 : cols <= 256 ? 256 : 512;
@@ -93,11 +91,6 @@ __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi)
 // 128-byte lines at once, where per-thread 2-byte stores leave each line to be completed by a
 // second warp later.
 // tma_c = SK_TMA_F32: fp32 output, staged (and summed over the cluster) like SK_TMA_ADD, stored.
-// Folded norm, TMA form (nm.use_tma; large tiles): a consumer scales the staged tile by the rows'
-// rstd before it leaves; a producer (SK_TMA_ADD with nm.a_out), once its reduction into x has
-// completed, loads the same block of x back through mapC, writes bf16(gain * x) through mapD
-// (bf16 [M][N], same boxes as mapC) and one sum of squares per row and 128-feature tile.  Every
-// element of x has exactly one contributor per contraction, so the block it reads back is final.
 enum { SK_TMA_NONE = 0, SK_TMA_ADD = 1, SK_TMA_BF16 = 2, SK_TMA_F32 = 3 };
 __device__ __forceinline__ void sk_tma_store(const CUtensorMap *map, uint32_t src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
@@ -112,45 +105,10 @@ __device__ __forceinline__ void sk_tma_reduce_add(const CUtensorMap *map, uint32
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
-// Producer half of the folded norm in its TMA form, run by the 128 epilogue threads after thread 0's
-// reduction of `rows` token rows x 128 features (staged at `blk`, rows of 512 bytes) into x has
-// completed: x comes back into the same place, bf16(gain * x) is staged behind the CTA's fp32 tile
-// (at `blk16`) and stored, the rows' sums of squares over this feature tile go to ssq_out.
-__device__ __forceinline__ void sk_norm_produce_tma(const CUtensorMap *mapC, const CUtensorMap *mapD, uint32_t blk,
-                                                    float *blk_f, bf16 *blk_h, uint32_t blk16, int rows, int f_tile0,
-                                                    int row0, int M, int N, const float *gain, float *ssq_out,
-                                                    uint32_t rb, uint32_t phase, bool active, int *status) {
-  if (threadIdx.x == 0 && active) {
-    mbar_expect_tx(rb, (uint32_t)rows * (TC_BM * 4));
-    tma_load_2d(blk, mapC, f_tile0, row0, rb);
-  }
-  if (active) {
-    if (!mbar_wait(rb, phase)) { if (threadIdx.x == 0) atomicExch(status, DEV_TIMEOUT_EPILOGUE); active = false; }
-  }
-  if (active) {
-    const int rg = threadIdx.x >> 5, lane = threadIdx.x & 31, c4 = lane * 4;
-    const float4 gg = *reinterpret_cast<const float4 *>(gain + f_tile0 + c4);
-    for (int tl = rg; tl < rows; tl += 4) {
-      const float4 xv = *reinterpret_cast<const float4 *>(blk_f + (size_t)tl * TC_BM + c4);
-      const __nv_bfloat162 lo = __floats2bfloat162_rn(gg.x * xv.x, gg.y * xv.y), hi = __floats2bfloat162_rn(gg.z * xv.z, gg.w * xv.w);
-      uint2 pk;
-      pk.x = *reinterpret_cast<const uint32_t *>(&lo);
-      pk.y = *reinterpret_cast<const uint32_t *>(&hi);
-      *reinterpret_cast<uint2 *>(blk_h + (size_t)tl * TC_BM + c4) = pk;
-      const float sq = warp_sum(xv.x * xv.x + xv.y * xv.y + xv.z * xv.z + xv.w * xv.w);
-      if (lane == 0 && row0 + tl < M) ssq_out[(size_t)(row0 + tl) * (N >> 7) + (f_tile0 >> 7)] = sq;
-    }
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  asm volatile("bar.sync 2, 128;" ::: "memory");
-  if (threadIdx.x == 0 && active) sk_tma_store(mapD, blk16, f_tile0, row0);
-}
-
 template <int WT, bool NORM>
 __global__ void __launch_bounds__(192, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
-               const __grid_constant__ CUtensorMap mapC, const __grid_constant__ CUtensorMap mapD,
-               void *__restrict__ C, int M, int N, int K, int BN,
+               const __grid_constant__ CUtensorMap mapC, void *__restrict__ C, int M, int N, int K, int BN,
                int stages, int tmem_cols, int ring_bytes, int epi, int tma_c, const SkNorm nm,
                int *__restrict__ status, const LiveRows lr) {
   constexpr int wt = WT;
@@ -168,7 +126,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
   extern __shared__ uint8_t smem_raw[];
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = tiles + (uint32_t)ring_bytes;
-  const uint32_t full0 = bars, empty0 = bars + 64, accum = bars + 128, slot = bars + 136, rb = bars + 144;
+  const uint32_t full0 = bars, empty0 = bars + 64, accum = bars + 128, slot = bars + 136;
   uint32_t *slot_ptr = reinterpret_cast<uint32_t *>(smem_raw + (slot - smem_u32(smem_raw)));
   float *rs = reinterpret_cast<float *>(smem_raw + (bars + 256 - smem_u32(smem_raw)));   // [BN] rstd of the tile's rows
   float *stage_f = reinterpret_cast<float *>(smem_raw + (tiles - smem_u32(smem_raw)));
@@ -192,7 +150,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
     asm volatile("prefetch.tensormap [%0];" ::"l"(&mapW) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&mapA) : "memory");
     if (tma_c) asm volatile("prefetch.tensormap [%0];" ::"l"(&mapC) : "memory");
-    if (NORM && nm.use_tma && nm.a_out) asm volatile("prefetch.tensormap [%0];" ::"l"(&mapD) : "memory");
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -200,7 +157,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       mbar_init(empty0 + 8 * s, 1);
     }
     mbar_init(accum, 1);
-    mbar_init(rb, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 5) {
@@ -288,10 +244,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
         if (t0 + cc >= M) break;
         float v[16];
         tmem_ld16(tbase + cc, v);
-        if (NORM && nm.ssq_in && tma_c && S == 1) {            // consumer of a folded norm: rows scaled by rstd
-#pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] *= rs[cc + j];
-        }
         if (tma_c == SK_TMA_BF16) {
           bf16 *stage_h = reinterpret_cast<bf16 *>(stage_f);
 #pragma unroll
@@ -341,10 +293,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
         if (tma_c == SK_TMA_ADD) sk_tma_reduce_add(&mapC, tiles, f0 + q * TC_BM, t0);
         else sk_tma_store(&mapC, tiles, f0 + q * TC_BM, t0);
       }
-      if (NORM && nm.use_tma && nm.a_out && tma_c == SK_TMA_ADD)
-        sk_norm_produce_tma(&mapC, &mapD, tiles, stage_f, reinterpret_cast<bf16 *>(stage_f + (size_t)BN * TC_BM),
-                            tiles + (uint32_t)BN * (TC_BM * 4), BN, f0 + q * TC_BM, t0, M, N, nm.gain, nm.ssq_out, rb,
-                            (uint32_t)(q & 1), acc_ok, status);
       asm volatile("bar.sync 2, 128;" ::: "memory");       // the stage is free again
     }
   }
@@ -376,21 +324,14 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
 #pragma unroll
         for (int r = 1; r < SK_MAX_SPLIT; ++r)
           if (r < S) { sum.x += v[r].x; sum.y += v[r].y; sum.z += v[r].z; sum.w += v[r].w; }
-        if (NORM && nm.ssq_in) { const float k = rs[tl]; sum.x *= k; sum.y *= k; sum.z *= k; sum.w *= k; }
         *reinterpret_cast<float4 *>(stage_f + (size_t)tl * TC_BM + c4) = sum;
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("bar.sync 2, 128;" ::: "memory");
-      const bool mine = t0 + rank * RB < M;
-      if (threadIdx.x == 0 && mine) {
+      if (threadIdx.x == 0 && t0 + rank * RB < M) {
         if (tma_c == SK_TMA_ADD) sk_tma_reduce_add(&mapC, tiles + (uint32_t)(rank * RB) * (TC_BM * 4), f0, t0 + rank * RB);
         else sk_tma_store(&mapC, tiles + (uint32_t)(rank * RB) * (TC_BM * 4), f0, t0 + rank * RB);
       }
-      // (the bf16 copy of this CTA's block is staged behind the BN-row fp32 tile that its peers still read)
-      if (NORM && nm.use_tma && nm.a_out && tma_c == SK_TMA_ADD)
-        sk_norm_produce_tma(&mapC, &mapD, tiles + (uint32_t)(rank * RB) * (TC_BM * 4), stage_f + (size_t)(rank * RB) * TC_BM,
-                            reinterpret_cast<bf16 *>(stage_f + (size_t)BN * TC_BM), tiles + (uint32_t)BN * (TC_BM * 4), RB, f0,
-                            t0 + rank * RB, M, N, nm.gain, nm.ssq_out, rb, 0u, mine, status);
     } else if (warp < 4) {
       // thread -> (row group, 4 consecutive features): one 16-byte load per partial tile, all S
       // loads of a row in flight together, one 16-byte (fp32) or 8-byte (bf16) store per row
@@ -503,8 +444,7 @@ static int gemm_sk_init() {
   if (dev_done[dev]) return 0;
   if (cudaFuncSetAttribute(gemm_sk_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_sk_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_sk_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_sk_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      cudaFuncSetAttribute(gemm_sk_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
     return -4;
   dev_done[dev] = true;
   return 0;
@@ -594,29 +534,28 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   const int KB = (p.K + TC_BK - 1) / TC_BK;
   const int FT = (p.N + TC_BM - 1) / TC_BM, TT = (M + BN - 1) / BN;
   // residual epilogue through the TMA unit: x and its row pitch 16-byte aligned, whole feature tiles
-  // (a folded norm keeps these epilogues only in its TMA form)
   int tma_c = SK_TMA_NONE;
-  if ((!norm || norm->use_tma) && p.N % TC_BM == 0 && BN % S == 0 && !((uintptr_t)C & 15)) {
+  if (!norm && p.N % TC_BM == 0 && BN % S == 0 && !((uintptr_t)C & 15)) {
     if (epi == EPI_RESID) tma_c = SK_TMA_ADD;
     else if (epi == EPI_F32) tma_c = SK_TMA_F32;
     else if ((epi == EPI_T || epi == EPI_GELU_T) && S == 1) tma_c = SK_TMA_BF16;
   }
-  if (norm && norm->use_tma && !tma_c) return false;           // the caller chose the TMA form: it must apply
-  auto c_map = [&](const void *base, bool hb) -> const CUtensorMap * {
+  const CUtensorMap *mapC = &p.mapW;                         // placeholder when unused
+  if (tma_c) {
     const int rows = BN / S;
+    const bool hb = tma_c == SK_TMA_BF16;
+    const GemmSkPlan::CMap *hit = nullptr;
     for (const auto &c : p.mapC)
-      if (c.C == base && c.M == M && c.rows == rows && c.is_bf16 == hb) return &c.map;
-    GemmSkPlan::CMap c{base, M, rows, hb, {}};
-    if (sk_encode_c(&c.map, base, M, p.N, rows, hb)) return nullptr;
-    p.mapC.push_back(c);
-    return &p.mapC.back().map;
-  };
-  const CUtensorMap *mapC = &p.mapW, *mapD = &p.mapW;       // placeholders when unused
-  if (tma_c && !(mapC = c_map(C, tma_c == SK_TMA_BF16))) return false;
-  const bool produce_tma = norm && norm->use_tma && norm->a_out && tma_c == SK_TMA_ADD;
-  if (produce_tma && (((uintptr_t)norm->a_out & 15) || !(mapD = c_map(norm->a_out, true)))) return false;
-  const CUtensorMap mapC_v = *mapC, mapD_v = *mapD;          // (the cache may have grown between the two lookups)
-  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1 || tma_c, wt, produce_tma);
+      if (c.C == C && c.M == M && c.rows == rows && c.is_bf16 == hb) { hit = &c; break; }
+    if (!hit) {
+      GemmSkPlan::CMap c{C, M, rows, hb, {}};
+      if (sk_encode_c(&c.map, C, M, p.N, rows, hb)) return false;
+      p.mapC.push_back(c);
+      hit = &p.mapC.back();
+    }
+    mapC = &hit->map;
+  }
+  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1 || tma_c, wt);
   if (sh.smem_bytes > 227 * 1024) return false;
   const int ring_bytes = sh.smem_bytes - 1024 - 256 - 1024;
   const SkNorm nm = norm ? *norm : SkNorm{};
@@ -635,10 +574,10 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
   cfg.numAttrs = pdl ? 2 : 1;
   int N = p.N, K = p.K, stages = sh.stages, cols = sh.tmem_cols, rb = ring_bytes;
   auto go = [&](auto kernel) {
-    return cudaLaunchKernelEx(&cfg, kernel, p.mapW, p.mapA[idx], mapC_v, mapD_v, C, M, N, K, BN, stages, cols, rb, epi, tc, nm,
-                              status, lr) == cudaSuccess;
+    return cudaLaunchKernelEx(&cfg, kernel, p.mapW, p.mapA[idx], *mapC, C, M, N, K, BN, stages, cols, rb, epi, tc, nm, status,
+                              lr) == cudaSuccess;
   };
-  if (wt == 2) return norm ? go(gemm_sk_kernel<2, true>) : go(gemm_sk_kernel<2, false>);
+  if (wt == 2) return go(gemm_sk_kernel<2, false>);
   return norm ? go(gemm_sk_kernel<1, true>) : go(gemm_sk_kernel<1, false>);
 }
 
