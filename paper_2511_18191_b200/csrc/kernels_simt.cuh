@@ -793,19 +793,15 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
   }
 }
 
-// The head for the boundary tokens of a pass of many rows: 8 rows per CTA (one warp normalises one
-// row into shared memory), then each warp produces 4 of the CTA's 32 outputs for all 8 rows, so that
-// a weight vector is loaded once per 8 rows.  M counts boundary rows (series x boundaries per series,
-// boundaries per series = q_len / head_step).
-//   hist == NULL: boundary i of series b goes to vout[b, i, :]                      (verification)
-//   hist != NULL (one boundary per series, head_step = q_len): the prediction goes behind the pass in
-//                the series' history, as head_kernel's only_last mode does           (draft / decode steps)
+// The head for the boundary tokens of a pass of many rows (verification: vout[b, i, :]): 8 rows
+// per CTA (one warp normalises one row into shared memory), then each warp produces 4 of the CTA's
+// 32 outputs for all 8 rows, so that a weight vector is loaded once per 8 rows.  M counts boundary
+// rows (series x boundaries per series).
 // grid = (ceil(M / 8), ceil(P / 32)), block = 256, dynamic shared memory 8 * d floats.
 template <typename T>
 __global__ void __launch_bounds__(256)
 head_rows_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T *__restrict__ Wh, int M,
-                 int d, int P, float eps, float *__restrict__ vout, PassGeom g, float *__restrict__ hist, int tok_len,
-                 const DevState *__restrict__ st, float *__restrict__ muq, int k_pos, int K) {
+                 int d, int P, float eps, float *__restrict__ vout, PassGeom g) {
   constexpr int R = 8;
   extern __shared__ __align__(16) float xs[];                  // [R][d] normalised rows
   pdl_sync();
@@ -832,7 +828,6 @@ head_rows_kernel(const float *__restrict__ x, const float *__restrict__ gain, co
     for (int i = lane; i < d; i += 32) xw[i] = gain[i] * xw[i] * rstd;   // each lane rewrites what it wrote
   }
   __syncthreads();
-  const bool sample = hist && st && (st->flags & VAR_SAMPLE_PROPOSALS);
   constexpr int V = Vec16<T>::N;
   for (int q = 0; q < 4; ++q) {
     const int p = blockIdx.y * 32 + q * 8 + w;
@@ -851,18 +846,10 @@ head_rows_kernel(const float *__restrict__ x, const float *__restrict__ gain, co
     }
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      float o = warp_sum(acc[r]);
-      if (lane == 0 && row0 + r < M) {                         // outputs are indexed by series, rows by slot
+      const float o = warp_sum(acc[r]);
+      if (lane == 0 && row0 + r < M) {                         // vout is indexed by series, rows by slot
         const int row = row0 + r, b = series_of(g, row / nb);
-        if (hist) {
-          if (sample) {        // sampled proposal x = mu_q + sigma_q eps (Sec. 3.3); the mean is kept for the statistic
-            muq[((size_t)b * K + k_pos) * P + p] = o;
-            o += st->sigma_q * head_normal(st, b, k_pos, p);
-          }
-          hist[((size_t)b * g.cap + pos0_of(g, b) + g.q_len) * tok_len + p] = o;
-        } else {
-          vout[((size_t)b * nb + row % nb) * P + p] = o;
-        }
+        vout[((size_t)b * nb + row % nb) * P + p] = o;
       }
     }
   }

@@ -24,6 +24,7 @@ def _operands(M, N, K, seed):
 
 
 def _both(tsfm, M, N, K, seed):
+    """(static-scratch result, allocating entry point's result, fp64 product of the same operands)."""
     A, W = _operands(M, N, K, seed)
     s = torch.cuda.current_stream().cuda_stream
     want = torch.full((M, N), float("nan"), device="cuda")
@@ -31,7 +32,8 @@ def _both(tsfm, M, N, K, seed):
     got = torch.full((M, N), float("nan"), device="cuda")
     tsfm.tsfm_gemm_bf16_static(s, A, W, got, M, N, K)
     torch.cuda.synchronize()
-    return got.cpu().numpy(), want.cpu().numpy()
+    exact = (A.cpu().double() @ W.cpu().double().T).numpy()
+    return got.cpu().numpy(), want.cpu().numpy(), exact
 
 
 def test_static_scratch_contraction_matches_the_allocating_one_on_calls_in_a_row():
@@ -40,11 +42,13 @@ def test_static_scratch_contraction_matches_the_allocating_one_on_calls_in_a_row
     # the first shape again: stale partial sums from any earlier call would show up as an error
     shapes = [(160, 1536, 512), (32, 512, 2048), (7, 130, 64), (160, 1536, 512)]
     for i, (M, N, K) in enumerate(shapes):
-        got, want = _both(tsfm, M, N, K, seed=10 + i)
+        got, want, exact = _both(tsfm, M, N, K, seed=10 + i)
         assert np.isfinite(got).all()
         # same tolerance as the tensor-core / FMA comparison of the contraction tests: the two
         # differ only in the order in which the K-split partial sums are added
         assert np.abs(got - want).max() < 2e-5 * K ** 0.5 + 1e-5, (i, M, N, K)
+        # and against the product itself, not only against another kernel
+        assert np.abs(got - exact).max() < 2e-5 * K ** 0.5 + 1e-5, (i, M, N, K)
 
 
 def test_outputs_beyond_the_scratch_capacity_are_rejected_with_a_message():
@@ -58,5 +62,6 @@ def test_outputs_beyond_the_scratch_capacity_are_rejected_with_a_message():
     assert e.value.code == tsfm.TSFM_ERR_SHAPE and "capacity" in str(e.value)
     assert float(out.abs().max()) == 0.0           # nothing was written
     # and the entry point still works afterwards
-    got, want = _both(tsfm, 64, 256, 128, seed=4)
+    got, want, exact = _both(tsfm, 64, 256, 128, seed=4)
     assert np.abs(got - want).max() < 2e-5 * 128 ** 0.5 + 1e-5
+    assert np.abs(got - exact).max() < 2e-5 * 128 ** 0.5 + 1e-5
