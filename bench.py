@@ -47,11 +47,16 @@ UNIT = "patches/s"
 # A kernel that has changed since its capture is listed with None.
 NCU_TRAFFIC_RATIO = {
     "gemm_sk_small_M": None,
-    "gemm_sk_mid_M": None,
+    "gemm_sk_mid_M": 0.564,        # 11.36 MB read, 0 written, of 20.15 MB: the fp32 result stays in L2 for its consumer
     "gemm_sk_large_M": None,
-    "attn": None,
+    "gemm_ws_small_M": 0.77,       # 0.949 MB of 1.229 MB
+    "attn": 1.0,                   # 96.5 MB of 96.9 MB: the KV stream
 }
-NCU_TRAFFIC_SOURCE = {}
+NCU_TRAFFIC_SOURCE = {
+    "gemm_sk_mid_M": "profiles/gemm_sk_kernel_mid_M_C4_verification_QKV.txt (M=576, N=3840, K=1280, cold caches)",
+    "gemm_ws_small_M": "profiles/gemm_ws_kernel_draft_step_QKV.txt (M=64, N=1152, K=384, cold caches)",
+    "attn": "profiles/attn_flash_kernel_C4_verify_and_decode.txt (C4 verification pass, 2-layer small case)",
+}
 
 
 def parse_args():
