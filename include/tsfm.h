@@ -83,10 +83,6 @@ extern "C" {
                                    the buffer's name in tsfm_last_cuda_error().  Costs memory and a launch
                                    per call; for test runs                                               */
 
-#define TSFM_EXEC_NO_FUSION 16     /* flag, may be OR-ed in: small passes run one kernel per operation (attention-
-                                   output projection, MLP up, MLP down, QKV) instead of the fused kernel that
-                                   covers everything between two attention steps; differential reference  */
-
 #define TSFM_MAX_K 32           /* hard upper bound on the block size K                             */
 
 typedef struct tsfm_spec tsfm_spec;   /* opaque decoder handle */
@@ -112,7 +108,7 @@ typedef struct {
   float   rms_eps;              /* RMSNorm epsilon (1e-6)                                        */
   float   norm_eps;             /* instance-norm variance epsilon (1e-5)                         */
   float   rope_base;            /* RoPE base (1e4)                                               */
-  int32_t exec_mode;            /* TSFM_EXEC_GRAPH or TSFM_EXEC_STREAM, optionally | the TSFM_EXEC_* flags above        */
+  int32_t exec_mode;            /* TSFM_EXEC_GRAPH or TSFM_EXEC_STREAM, optionally | TSFM_EXEC_NO_PDL | TSFM_EXEC_NO_COMPACT */
   int32_t patch_in;             /* P_in: steps per INPUT token; 0 = patch_len (a token is a whole patch).
                                    Must divide patch_len.  With P_in < P (the point-token family of the
                                    paper's appendix B: P_in = 1, a horizon head of P steps) a committed

@@ -20,7 +20,6 @@ TSFM_F32, TSFM_BF16 = 0, 1
 TSFM_DRAFT_SEPARATE, TSFM_DRAFT_LAYER_SKIP = 0, 1
 TSFM_GEMM_AUTO, TSFM_GEMM_SIMT, TSFM_GEMM_WS = 0, 1, 2
 TSFM_EXEC_GRAPH, TSFM_EXEC_STREAM, TSFM_EXEC_NO_PDL, TSFM_EXEC_NO_COMPACT, TSFM_EXEC_CHECK_BOUNDS = 0, 1, 2, 4, 8
-TSFM_EXEC_NO_FUSION = 16
 TSFM_MAX_K = 32
 
 EXPORTS = [

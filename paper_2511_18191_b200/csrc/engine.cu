@@ -23,7 +23,6 @@
 #include "gemm_tc.cuh"
 #include "gemm_sk.cuh"
 #include "gemm_ws.cuh"
-#include "layer_block.cuh"
 
 using namespace tsfm;
 
@@ -147,7 +146,6 @@ struct tsfm_spec {
   int *done = nullptr;
   int *live = nullptr, *n_live = nullptr;   // [B] slot -> unfinished series, and their number (round_end_kernel)
   bool compact = true;                   // rounds run over the unfinished series only
-  bool fuse = true;                      // small passes take the fused layer-block kernel where it applies
   AcceptCounters *ctr = nullptr;
   int *unfinished = nullptr;             // [max_T + 1]
   int *h_unfinished = nullptr;           // pinned
@@ -177,9 +175,9 @@ namespace {
 // Kernel classes for per-launch timing.
 // The tensor-core contraction is one kernel in three regimes: up to 512 tokens it streams weights
 // (HBM / latency bound), from 4096 tokens it is tensor bound, between them it is one wave of tiles.
-enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_BLOCK, KC_GEMM_WS, KC_GEMM_TC_SMALL, KC_GEMM_TC_MID, KC_GEMM_TC_LARGE, KC_GEMM_SIMT,
+enum { KC_INSTNORM = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_WS, KC_GEMM_TC_SMALL, KC_GEMM_TC_MID, KC_GEMM_TC_LARGE, KC_GEMM_SIMT,
        KC_ATTN, KC_HEAD, KC_ACCEPT, KC_DENORM, KC_COUNT };
-const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "layer_block", "gemm_ws_small_M", "gemm_sk_small_M",
+const char *const kKernelNames[KC_COUNT] = {"instnorm", "embed", "rmsnorm", "gemm_ws_small_M", "gemm_sk_small_M",
                                             "gemm_sk_mid_M", "gemm_sk_large_M", "gemm_simt", "attn", "head", "accept",
                                             "denorm"};
 
@@ -371,7 +369,6 @@ void prefer_max_smem_all() {
   prefer_max_smem(gemm_sk_kernel<2, false>);
   prefer_max_smem(gemm_ws_kernel<false>);
   prefer_max_smem(gemm_ws_kernel<true>);
-  prefer_max_smem(layer_block_kernel);
   prefer_max_smem(attn_flash_kernel<32, 3>);
   prefer_max_smem(attn_flash_kernel<32, kFlashStShort>);
   prefer_max_smem(attn_flash_kernel<64, 3>);
@@ -571,46 +568,17 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   consume.n_part = d / 16;
   consume.inv_d = 1.f / d;
   consume.eps = eps;
-  // Passes of a few tokens on small models: everything between two attention steps (Wo, norm, MLP,
-  // the next layer's QKV) is one cluster kernel (layer_block.cuh): 2 launches per layer instead of 5.
-  int lb_bg = 0, lb_g = 0;
-  const bool blocks = fold && h->fuse && head_mode != HEAD_NONE &&
-                      lb_geometry(d, m.arch.n_heads, f, B, g.q_len, &lb_bg, &lb_g);
   for (int l = 0; l < L; ++l) {
     LayerDev &ly = m.layers[l];
     if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
       launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g1, M, d, eps, (T *)h->a, lr);
     }
-    if (!blocks || l == 0)
-      gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr, lr);
+    gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr, lr);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
     else if (m.dh == 64) launch_attn<T, 64>(h, m, l, B, g);
     else launch_attn<T, 128>(h, m, l, B, g);
     if (l == L - 1 && head_mode == HEAD_NONE) break;   // prefill: only the cache is needed
-    if (blocks) {
-      LbArgs a{};
-      a.ao = (const bf16 *)h->ao;
-      a.x = h->x;
-      a.Wo = (const bf16 *)ly.Wo; a.W1 = (const bf16 *)ly.W1; a.W2 = (const bf16 *)ly.W2;
-      a.g_mid = ly.g2;
-      a.g_next = l + 1 < L ? m.layers[l + 1].g1 : nullptr;
-      a.Wqkv = l + 1 < L ? (const bf16 *)m.layers[l + 1].Wqkv : nullptr;
-      a.qkv = h->qkv;
-      a.d = d; a.ff = f; a.R = m.arch.n_heads;
-      a.q_len = g.q_len; a.Bg = lb_bg; a.B = B;
-      a.n_live = g.n_live;
-      a.eps = eps;
-      const double wts = ((double)d * d + 2.0 * d * f + (l + 1 < L ? 3.0 * d * d : 0.0));
-      KTimer kt(h, KC_BLOCK, wts * 2 + (double)M * d * (2 + 8) + (l + 1 < L ? (double)M * 3 * d * 4 : 0.0), 2.0 * M * wts);
-      if (lb_launch(s, h->pdl, a, lb_g)) {
-        LAUNCHED();
-      } else if (h->enqueue_err == TSFM_OK) {
-        h->enqueue_err = TSFM_ERR_CUDA;
-        g_cuda_err = std::string("layer-block kernel could not be launched: ") + cudaGetErrorString(cudaGetLastError());
-      }
-      continue;
-    }
     SkNorm produce{};               // residual epilogue also emits the next operand and its statistics
     produce.ssq_out = h->ssq;
     produce.a_out = (bf16 *)h->a;
@@ -995,7 +963,7 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   *out_h = nullptr;
   const int P = cfg->patch_len;
   if (cfg->dtype != TSFM_F32 && cfg->dtype != TSFM_BF16) return TSFM_ERR_ARG;
-  if (cfg->exec_mode & ~(TSFM_EXEC_STREAM | TSFM_EXEC_NO_PDL | TSFM_EXEC_NO_COMPACT | TSFM_EXEC_CHECK_BOUNDS | TSFM_EXEC_NO_FUSION))
+  if (cfg->exec_mode & ~(TSFM_EXEC_STREAM | TSFM_EXEC_NO_PDL | TSFM_EXEC_NO_COMPACT | TSFM_EXEC_CHECK_BOUNDS))
     return TSFM_ERR_ARG;
   if (cfg->gemm_backend != TSFM_GEMM_AUTO && cfg->gemm_backend != TSFM_GEMM_SIMT) return TSFM_ERR_ARG;
   if (cfg->draft_mode != TSFM_DRAFT_SEPARATE && cfg->draft_mode != TSFM_DRAFT_LAYER_SKIP) return TSFM_ERR_ARG;
@@ -1031,7 +999,6 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   h->use_tc = cfg->dtype == TSFM_BF16 && cfg->gemm_backend != TSFM_GEMM_SIMT;
   h->pdl = (cfg->exec_mode & TSFM_EXEC_NO_PDL) == 0;
   h->compact = (cfg->exec_mode & TSFM_EXEC_NO_COMPACT) == 0;
-  h->fuse = (cfg->exec_mode & TSFM_EXEC_NO_FUSION) == 0;
   int rc = TSFM_OK;
   auto fail = [&](int code) { tsfm_spec_destroy(h); return code; };
 
@@ -1120,7 +1087,6 @@ int tsfm_spec_create(const tsfm_weights *target_w, const tsfm_weights *draft_w, 
   if (h->use_tc) {
     if ((rc = gemm_sk_init())) return fail(rc);
     if ((rc = gemm_ws_init())) return fail(rc);
-    if ((rc = lb_init())) return fail(rc);
     for (ModelDev *m : {&h->tgt, &h->drf}) {
       const int d = m->arch.d_model, f = m->arch.d_ff;
       for (LayerDev &ly : m->layers) {

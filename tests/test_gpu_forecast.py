@@ -150,40 +150,6 @@ def test_compaction_of_finished_series_changes_nothing(name):
         assert res[0][2] == other[2]
 
 
-@pytest.mark.parametrize("name", ["C1-layer-skip", "C4-draft-shape", "ragged-compacted"])
-def test_fused_layer_block_against_the_oracle_and_the_per_operation_path(name):
-    """Small passes run everything between two attention steps as one cluster kernel.  Both forms are
-    compared with the oracle (all series); they agree with each other to rounding, and the fused one
-    makes fewer launches."""
-    import paper_2511_18191_b200 as tsfm
-    if name == "C1-layer-skip":
-        wl, K, tau = workload("C1", batch=20), 4, 2.0                       # 8 heads: clusters of 8, draft and target
-    elif name == "C4-draft-shape":                                           # 6-head draft (clusters of 6), big target on the per-op path
-        wl, K, tau = workload("C4", batch=9, horizon=32 * 9 + 5, target=Arch(2, 512, 8, 2048)), 5, 2.0
-    else:                                                                    # series finish at different rounds: partial clusters
-        wl, K, tau = workload("C1", batch=37, horizon=96 * 12, target=Arch(3, 256, 4, 1024), draft=Arch(2, 256, 4, 1024)), 3, 1.5
-    s, ctx = series_on_device(wl)
-    outs, launches = [], []
-    for mode in (tsfm.TSFM_EXEC_GRAPH, tsfm.TSFM_EXEC_GRAPH | tsfm.TSFM_EXEC_NO_FUSION):
-        dec, tw, dw = make_decoder(wl, max_K=K, exec_mode=mode)
-        dec.forecast(ctx, wl.horizon, K, tau, 11)                            # captures the graph
-        n0 = tsfm.tsfm_launch_count()
-        out, st = dec.forecast(ctx, wl.horizon, K, tau, 11)
-        launches.append(tsfm.tsfm_launch_count() - n0)
-        check_stats(st, wl.batch, wl.n_patches, K)
-        nacc, ell, logu = dec.last_trace(wl.batch, K)
-        ref, _ = dec.target_only(ctx, wl.horizon)
-        dec.close()
-        tm, dm = parity.oracle_models(wl, tw, dw)
-        parity.compare_forecast(wl, tm, dm, s, wl.horizon, K, tau, 11, out.cpu().numpy(), nacc, range(wl.batch),
-                                gpu_ell=ell, gpu_logu=logu)
-        want_t = parity.oracle_target_only(tm, s, wl.ctx_len, wl.horizon, range(wl.batch))
-        assert parity.per_series_errors("rel_rms", ref.cpu().numpy(), want_t).max() <= 3e-2
-        outs.append(ref.cpu().numpy())
-    assert launches[0] < launches[1]
-    assert parity.per_series_errors("rel_rms", outs[0], outs[1].astype(np.float64)).max() < 2e-2
-
-
 BOUNDS_CASES = {
     "fp32-ragged": lambda: (workload("C0", batch=6, series_recipe="c1", horizon=96 * 7 + 5), 4, 4.0),
     "bf16-small-M": lambda: (workload("C1", batch=12, horizon=96 * 10), 4, 2.0),
