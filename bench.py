@@ -14,8 +14,8 @@ shards by series with no exchange step: weak scaling, no collective); times are 
 times, max over ranks.
 
 On one GPU the line also carries, under `workloads`, the same measurement (fewer steps) of
-C2 (tensor-bound verification), C1 at its three temperatures and four cells of C3's
-K x eps grid, each with target-only and draft-only decoding, phase times, and the speedup
+C2 (tensor-bound verification), C1 at its three temperatures, C1 with a draft that tracks its
+target (acceptance ~0.97, the regime the paper reports) and four cells of C3's K x eps grid, each with target-only and draft-only decoding, phase times, and the speedup
 Eq. 8 predicts from the measured acceptance rate and cost ratios beside the measured one.
 
 `--impl reference` times the CPU oracle (fp64, as it stands) on a bounded sample of the same
@@ -440,6 +440,11 @@ def other_workloads(names):
         if n == "C1":
             wl = workload("C1")
             out += [(f"C1_tau{t:g}", wl, wl.K, t) for t in wl.tau_sweep]
+            # a draft that tracks its target (the regime the paper reports: acceptance 49-97 %): C1's
+            # layer-skip pair with the target's layers beyond the draft's depth damped to a tenth, and a
+            # 15-patch horizon so that a round is not a third of the forecast
+            wt = workload("C1", late_layer_scale=0.1, horizon=1440)
+            out.append(("C1_tracking_draft_H1440", wt, wt.K, 1.0))
         elif n == "C3":
             for eps in (0.0, 1e-3):
                 wl = workload("C3", draft_eps=eps)

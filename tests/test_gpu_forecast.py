@@ -93,6 +93,16 @@ def test_c1_full(tau, backend, exec_mode):
     run_and_compare(wl, wl.K, tau, wl.forecast_seed, range(wl.batch), backend=backend, exec_mode=exec_mode)
 
 
+def test_c1_with_a_draft_that_tracks_its_target():
+    """The regime the paper reports (acceptance 49-97 %): C1's layer-skip pair with the target's layers
+    beyond the draft's depth damped to a tenth, 15 patches to commit.  Most rounds yield K + 1."""
+    wl = workload("C1", late_layer_scale=0.1, horizon=1440)
+    res = run_and_compare(wl, wl.K, 1.0, wl.forecast_seed, range(0, wl.batch, 2))
+    d = res["stats"]
+    assert d["proposals_accepted"] / d["proposals_tested"] > 0.9
+    assert d["rounds"] <= 6
+
+
 def test_graph_and_stream_execution_give_identical_forecasts_and_traces():
     """The captured graph (device-side WHILE over rounds) replays exactly what the stream path
     launches: same kernels, same arguments -- so forecasts, decisions and counters are identical,

@@ -48,6 +48,7 @@ class Workload:
     eps_sweep: Tuple[float, ...] = ()
     draft_eps: float = 0.0          # perturbation size for "perturbed" drafts
     patch_in: int = 0               # steps per input token; 0 = patch_len (patch tokens)
+    late_layer_scale: float = 1.0   # layer-skip drafts: factor on Wo and W2 of the target layers the draft lacks
     weight_seed: int = 0
     perturb_seed: int = 1
     series_seed: int = 1000

@@ -97,6 +97,12 @@ def perturbed_draft(target: Weights, n_layers: int, eps: float, seed: int, dtype
 def build_models(wl: Workload):
     """(target weights, draft weights) for a workload."""
     tgt = make_model(wl.target, wl.patch_len, wl.weight_seed, wl.dtype, stream=0, patch_in=wl.patch_in)
+    if wl.draft_mode == "layer_skip" and wl.late_layer_scale != 1.0:
+        # a draft that tracks its target: the layers the draft lacks contribute less to the residual stream
+        for l in range(wl.draft.n_layers, wl.target.n_layers):
+            for t in ("Wo", "W2"):
+                w = tgt[f"layers.{l}.{t}"] * np.float32(wl.late_layer_scale)
+                tgt[f"layers.{l}.{t}"] = round_to_bf16(w) if wl.dtype == "bf16" else w.astype(np.float32)
     if wl.draft_mode == "layer_skip":
         drf = layer_skip_draft(tgt, wl.draft.n_layers)
     elif wl.draft_mode == "perturbed":
