@@ -88,10 +88,10 @@ attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__re
   const int warp_bytes = single ? 2 * S_TILE : G::WARP_BYTES;   // shared memory of one warp
   unsigned char *ring = flash_smem + (size_t)w * warp_bytes;
   const uint32_t ring32 = (uint32_t)__cvta_generic_to_shared(ring);
+  const SlotPos sp = slot_lookup(g, slot);                     // before the dependency wait: see SlotPos
   pdl_sync();
-  if (slot_dead(g, slot)) return;                              // per warp (FLASH_WARP) or per CTA: no barrier is pending
-  const int b = series_of(g, slot);
-  const int p0 = pos0_of(g, b);
+  if (sp.dead) return;                                         // per warp (FLASH_WARP) or per CTA: no barrier is pending
+  const int b = sp.b, p0 = sp.p0;
   const size_t row0 = (size_t)slot * g.q_len;
   bf16 *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
   bf16 *Vb = Vc + ((size_t)b * n_heads + h) * g.cap * DH;

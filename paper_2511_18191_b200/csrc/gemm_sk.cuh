@@ -92,17 +92,20 @@ __device__ __forceinline__ void sk_store_rt(void *C, size_t o, float v, int epi)
 // second warp later.
 // tma_c = SK_TMA_F32: fp32 output, staged (and summed over the cluster) like SK_TMA_ADD, stored.
 enum { SK_TMA_NONE = 0, SK_TMA_ADD = 1, SK_TMA_BF16 = 2, SK_TMA_F32 = 3 };
+// (Both wait only until the copy has READ its shared-memory source: the staging tile may then be reused
+// or the CTA may leave.  The writes themselves complete before the grid does, which is what the next
+// kernel's dependency wait waits for.)
 __device__ __forceinline__ void sk_tma_store(const CUtensorMap *map, uint32_t src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 __device__ __forceinline__ void sk_tma_reduce_add(const CUtensorMap *map, uint32_t src, int x, int y) {
   asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
 template <int WT, bool NORM>

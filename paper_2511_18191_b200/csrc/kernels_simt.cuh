@@ -36,6 +36,28 @@ __device__ __forceinline__ int pos0_of(const PassGeom &g, int b) {
 }
 __device__ __forceinline__ bool slot_dead(const PassGeom &g, int slot) { return g.n_live && slot >= *g.n_live; }
 __device__ __forceinline__ int series_of(const PassGeom &g, int slot) { return g.live ? g.live[slot] : slot; }
+// Series, first token position and liveness of a slot in one go.  The live count and the slot's series
+// are two independent loads (issued together); the committed count follows the series index.  The
+// loads are volatile (served by L2) because most kernels do this lookup BEFORE their dependency wait,
+// to take its two L2 round trips off the chain of dependent launches: `live` / `n_live` are written
+// only by round_end_kernel (and the instance-norm kernel), `done` only by accept_kernel, and every
+// kernel of a pass except the embedding that opens a round has at least two kernels between itself
+// and those -- a grid starts only after every CTA of its predecessor has passed its own dependency
+// wait, i.e. after the predecessor's predecessor has finished.  A dead slot's entry of `live` is a
+// stale but valid series index, so the lookup stays in bounds.
+struct SlotPos {
+  int b, p0;
+  bool dead;
+};
+__device__ __forceinline__ SlotPos slot_lookup(const PassGeom &g, int slot) {
+  const int nl = g.n_live ? *reinterpret_cast<const volatile int *>(g.n_live) : 0x7fffffff;
+  const int b = g.live ? reinterpret_cast<const volatile int *>(g.live)[slot] : slot;
+  SlotPos s;
+  s.dead = slot >= nl;
+  s.b = b;
+  s.p0 = (g.done ? reinterpret_cast<const volatile int *>(g.done)[b] * g.tpp : 0) + g.base;
+  return s;
+}
 // Rows of a pass that are in use: n_live * q_len of the M the launch was sized for.
 struct LiveRows {
   const int *n_live;
@@ -148,9 +170,10 @@ embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *
   pdl_sync();
   const int row = blockIdx.x, slot = row / g.q_len, j = row % g.q_len;
   if (stamp && row == 0 && blockIdx.y == 0 && threadIdx.x == 0) *stamp = globaltimer_ns();
-  if (slot_dead(g, slot)) return;
-  const int b = series_of(g, slot);
-  const float *z = hist + ((size_t)b * g.cap + pos0_of(g, b) + j) * P;
+  const SlotPos sp = slot_lookup(g, slot);                      // (after the wait: this kernel may open a round)
+  if (sp.dead) return;
+  const int b = sp.b;
+  const float *z = hist + ((size_t)b * g.cap + sp.p0 + j) * P;
   for (int i = threadIdx.x; i < P; i += blockDim.x) zs[i] = z[i];
   __syncthreads();
   const int f = blockIdx.y * 128 + threadIdx.x;
@@ -520,10 +543,10 @@ kv_append_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restric
                  const float2 *__restrict__ rope, PassGeom g, int n_heads) {
   constexpr int HALF = DH / 2;
   const int h = blockIdx.x, slot = blockIdx.y, d = n_heads * DH;
+  const SlotPos sp = slot_lookup(g, slot);                      // before the dependency wait: see SlotPos
   pdl_sync();
-  if (slot_dead(g, slot)) return;
-  const int b = series_of(g, slot);
-  const int p0 = pos0_of(g, b);
+  if (sp.dead) return;
+  const int b = sp.b, p0 = sp.p0;
   const int j_lo = blockIdx.z * 16, j_hi = min(g.q_len, j_lo + 16);
   const size_t row0 = (size_t)slot * g.q_len;
   T *Kb = Kc + ((size_t)b * n_heads + h) * g.cap * DH;
@@ -598,10 +621,10 @@ attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ V
   const int qt = skv > 1 ? blockIdx.z / skv : blockIdx.z;
   const int rank = skv > 1 ? blockIdx.z % skv : 0;   // == %cluster_ctarank: the cluster spans z only
   const int d = n_heads * DH;
+  const SlotPos sp = slot_lookup(g, slot);           // before the dependency wait: see SlotPos
   pdl_sync();
-  if (slot_dead(g, slot)) return;                    // the whole cluster (same y) leaves together
-  const int b = series_of(g, slot);
-  const int p0 = pos0_of(g, b);
+  if (sp.dead) return;                               // the whole cluster (same y) leaves together
+  const int b = sp.b, p0 = sp.p0;
   const int j_lo = qt * QT;
   const int j_hi = min(g.q_len, j_lo + QT);          // queries [j_lo, j_hi)
   const size_t row0 = (size_t)slot * g.q_len;
@@ -751,13 +774,14 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
             int tok_len) {
   extern __shared__ __align__(16) float xs[];
   __shared__ float red[32];
-  pdl_sync();
   const int nb = g.q_len / g.head_step;                // boundaries per series
   int slot, j, ib = 0;
   if (only_last) { slot = blockIdx.x; j = g.q_len - 1; }
   else { slot = blockIdx.x / nb; ib = blockIdx.x % nb; j = (ib + 1) * g.head_step - 1; }
-  if (slot_dead(g, slot)) return;
-  const int b = series_of(g, slot);
+  const SlotPos sp = slot_lookup(g, slot);             // before the dependency wait: see SlotPos
+  pdl_sync();
+  if (sp.dead) return;
+  const int b = sp.b;
   const float *xr = x + ((size_t)slot * g.q_len + j) * d;
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
@@ -768,7 +792,7 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
   const float rstd = rsqrtf(block_sum(ss, red) / d + eps);
   for (int i = threadIdx.x; i < d; i += blockDim.x) xs[i] = gain[i] * xs[i] * rstd;
   __syncthreads();
-  float *dst = only_last ? hist + ((size_t)b * g.cap + pos0_of(g, b) + g.q_len) * tok_len
+  float *dst = only_last ? hist + ((size_t)b * g.cap + sp.p0 + g.q_len) * tok_len
                          : vout + ((size_t)b * nb + ib) * P;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int p = blockIdx.y * 8 + w;
