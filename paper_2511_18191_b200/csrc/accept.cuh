@@ -85,8 +85,8 @@ struct AcceptArgs {
 // the WHILE node whether another round is needed.  One CTA of 256 threads.
 __global__ void __launch_bounds__(256)
 round_end_kernel(DevState *st, const int *unfinished, int T, cudaGraphConditionalHandle handle, int use_handle,
-                 const int *body_launches, unsigned long long *launch_ctr, const int *__restrict__ done, int B,
-                 int *__restrict__ live, int *__restrict__ n_live) {
+                 const int *body_launches, unsigned long long *launch_ctr, const int *done, int B,
+                 int *live, int *n_live) {
   __shared__ int warp_count[8];
   __shared__ int base;
   pdl_sync();

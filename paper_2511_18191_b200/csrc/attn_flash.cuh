@@ -67,7 +67,7 @@ template <int N> __device__ __forceinline__ void flash_wait() { asm volatile("cp
 
 template <int DH, int NB, int ST>
 __device__ __forceinline__ void
-attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
+attn_flash_body(const float *qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
                 const float2 *__restrict__ rope, const PassGeom &g, int n_heads, int n_pairs, int mode,
                 bf16 *__restrict__ out) {
   constexpr bool single = NB > 0;
@@ -89,7 +89,11 @@ attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__re
   unsigned char *ring = flash_smem + (size_t)w * warp_bytes;
   const uint32_t ring32 = (uint32_t)__cvta_generic_to_shared(ring);
   const SlotPos sp = slot_lookup(g, slot);                     // before the dependency wait: see SlotPos
-  pdl_sync();
+  // Passes of one query tile also start streaming their cached keys before the dependency wait: rows
+  // below pos0 of this layer's cache were written by this layer's attention in an earlier pass, a
+  // whole layer of kernels ago at least.  Passes of several tiles read the rows that the directly
+  // preceding kernel (kv_append_kernel) has just appended: they wait first.
+  if (mode == FLASH_TILES) pdl_sync();
   if (sp.dead) return;                                         // per warp (FLASH_WARP) or per CTA: no barrier is pending
   const int b = sp.b, p0 = sp.p0;
   const size_t row0 = (size_t)slot * g.q_len;
@@ -143,6 +147,10 @@ attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__re
 #pragma unroll
     for (int c = 0; c < G::STAGES - 1; ++c) issue(c);
   }
+  // q, k, v of the pass come from the preceding kernel.  They are read with ld.global.cg: their
+  // addresses are known before the wait, and a load on the read-only path (what a plain load through
+  // a const __restrict__ pointer compiles to) may be scheduled ahead of it.
+  if (mode != FLASH_TILES) pdl_sync();
 
   // rotated, scaled queries as A fragments (rows gr and gr + 8), high and low bf16 parts
   uint32_t qhi[KS][4], qlo[KS][4];
@@ -159,8 +167,8 @@ attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__re
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
           const int c = ks * 16 + hh * 8 + q4 * 2;             // first-half dims c, c + 1; partners c + HALF
-          const float2 q1 = *reinterpret_cast<const float2 *>(src + c);
-          const float2 q2 = *reinterpret_cast<const float2 *>(src + c + HALF);
+          const float2 q1 = __ldcg(reinterpret_cast<const float2 *>(src + c));   // (not a read-only-path load: see below)
+          const float2 q2 = __ldcg(reinterpret_cast<const float2 *>(src + c + HALF));
           const float4 cs = *reinterpret_cast<const float4 *>(rp + c);      // cos0 sin0 cos1 sin1
           float a0 = (q1.x * cs.x - q2.x * cs.y) * sc, a1 = (q1.y * cs.z - q2.y * cs.w) * sc;
           float b0 = (q2.x * cs.x + q1.x * cs.y) * sc, b1 = (q2.y * cs.z + q1.y * cs.w) * sc;
@@ -263,10 +271,10 @@ attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__re
         const float *src = qkv + (row0 + j) * 3 * d + h * DH;
         const int tg = p0 + j;
         const float4 cs = *reinterpret_cast<const float4 *>(rope + (size_t)tg * HALF + c);   // cos0 sin0 cos1 sin1
-        const float2 ka = *reinterpret_cast<const float2 *>(src + d + c);
-        const float2 kb = *reinterpret_cast<const float2 *>(src + d + c + HALF);
-        const float2 va = *reinterpret_cast<const float2 *>(src + 2 * d + c);
-        const float2 vb = *reinterpret_cast<const float2 *>(src + 2 * d + c + HALF);
+        const float2 ka = __ldcg(reinterpret_cast<const float2 *>(src + d + c));
+        const float2 kb = __ldcg(reinterpret_cast<const float2 *>(src + d + c + HALF));
+        const float2 va = __ldcg(reinterpret_cast<const float2 *>(src + 2 * d + c));
+        const float2 vb = __ldcg(reinterpret_cast<const float2 *>(src + 2 * d + c + HALF));
         const uint32_t k1 = pack_bf16x2(ka.x * cs.x - kb.x * cs.y, ka.y * cs.z - kb.y * cs.w);
         const uint32_t k2 = pack_bf16x2(kb.x * cs.x + ka.x * cs.y, kb.y * cs.z + ka.y * cs.w);
         const uint32_t v1 = pack_bf16x2(va.x, va.y), v2 = pack_bf16x2(vb.x, vb.y);
@@ -367,14 +375,14 @@ attn_flash_body(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__re
 // for four CTAs per SM where the head size allows it.
 template <int DH, int ST>
 __global__ void __launch_bounds__(128)
-attn_flash_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
+attn_flash_kernel(const float *qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
                   const float2 *__restrict__ rope, PassGeom g, int n_heads, int n_pairs, int mode,
                   bf16 *__restrict__ out) {
   attn_flash_body<DH, 0, ST>(qkv, Kc, Vc, rope, g, n_heads, n_pairs, mode, out);
 }
 template <int DH, int NB>
 __global__ void __launch_bounds__(128, DH <= 64 ? (NB == 1 ? 4 : 3) : 1)
-attn_flash_single_kernel(const float *__restrict__ qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
+attn_flash_single_kernel(const float *qkv, bf16 *__restrict__ Kc, bf16 *__restrict__ Vc,
                          const float2 *__restrict__ rope, PassGeom g, int n_heads, int n_pairs, int mode,
                          bf16 *__restrict__ out) {
   attn_flash_body<DH, NB, 3>(qkv, Kc, Vc, rope, g, n_heads, n_pairs, mode, out);

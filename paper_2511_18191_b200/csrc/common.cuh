@@ -54,6 +54,11 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
 // until that predecessor has completed and its writes are visible, pdl_release() lets the
 // successor start its own preamble.  Both are no-ops for an ordinary launch.  Every kernel here
 // calls pdl_wait() in every thread before its first access to memory another kernel writes.
+// Pointers to such memory are never `const T *__restrict__` kernel parameters: loads through
+// those compile to the read-only path (ld.global.nc), which promises data that no one writes while
+// the kernel runs, and such a load whose address is known before the wait was seen to be
+// scheduled ahead of it (attention read the previous pass's queries).  Only the constants of a
+// handle (weights, gains, RoPE tables) carry the qualifier pair.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_sync() { pdl_wait(); pdl_release(); }

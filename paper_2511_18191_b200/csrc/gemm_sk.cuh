@@ -111,7 +111,7 @@ __device__ __forceinline__ void sk_tma_reduce_add(const CUtensorMap *map, uint32
 template <int WT, bool NORM>
 __global__ void __launch_bounds__(192, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__ CUtensorMap mapA,
-               const __grid_constant__ CUtensorMap mapC, void *__restrict__ C, int M, int N, int K, int BN,
+               const __grid_constant__ CUtensorMap mapC, void *C, int M, int N, int K, int BN,
                int stages, int tmem_cols, int ring_bytes, int epi, int tma_c, const SkNorm nm,
                int *__restrict__ status, const LiveRows lr) {
   constexpr int wt = WT;

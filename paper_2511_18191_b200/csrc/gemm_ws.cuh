@@ -40,7 +40,7 @@ __device__ __forceinline__ void ws_ldsm4(uint32_t addr, uint32_t (&d)[4]) {
 // NORM: compile the folded-RMSNorm epilogues (SkNorm; slices of 16 features).
 template <bool NORM>
 __global__ void __launch_bounds__(256)
-gemm_ws_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, void *__restrict__ C, int M, int N, int K,
+gemm_ws_kernel(const bf16 *A, const bf16 *__restrict__ W, void *C, int M, int N, int K,
                int epi, const SkNorm nm, const LiveRows lr) {
   extern __shared__ __align__(128) unsigned char ws_smem[];
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;

@@ -104,8 +104,8 @@ __global__ void instnorm_kernel(DevState *__restrict__ st, int ctx_len, int hist
 }
 
 // out[b, s] = hist[b, ctx_len + s] * sd + mean, s < H.   grid = B.
-__global__ void denorm_kernel(const float *__restrict__ hist, int ctx_len, int hist_len, int H,
-                              const float *__restrict__ mean, const float *__restrict__ sd,
+__global__ void denorm_kernel(const float *hist, int ctx_len, int hist_len, int H,
+                              const float *mean, const float *sd,
                               DevState *__restrict__ st) {
   const int b = blockIdx.x;
   pdl_sync();
@@ -163,7 +163,7 @@ template <> struct Vec16<bf16> {
 // ----------------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(128)
-embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *__restrict__ W,
+embed_kernel(const float *hist, PassGeom g, int P, int d, const T *__restrict__ W,
              float *__restrict__ x, unsigned long long *__restrict__ stamp,
              const float *__restrict__ gain, T *__restrict__ a_out, float *__restrict__ ssq_out) {
   extern __shared__ float zs[];
@@ -208,7 +208,7 @@ embed_kernel(const float *__restrict__ hist, PassGeom g, int P, int d, const T *
 // grid = (ceil(M / 8), ceil(d / 128)), block = 128, dynamic shared memory 8 * P floats.
 template <typename T>
 __global__ void __launch_bounds__(128)
-embed_rows_kernel(const float *__restrict__ hist, PassGeom g, int M, int P, int d, const T *__restrict__ W,
+embed_rows_kernel(const float *hist, PassGeom g, int M, int P, int d, const T *__restrict__ W,
                   float *__restrict__ x, unsigned long long *__restrict__ stamp) {
   constexpr int R = 8;
   extern __shared__ float zs[];                               // [R][P]
@@ -274,7 +274,7 @@ __device__ __forceinline__ void store4(bf16 *o, float a, float b, float c, float
 
 template <typename T>
 __global__ void __launch_bounds__(256)
-rmsnorm_kernel(const float *__restrict__ x, const float *__restrict__ gain, int M, int d, float eps,
+rmsnorm_kernel(const float *x, const float *__restrict__ gain, int M, int d, float eps,
                T *__restrict__ a, LiveRows lr) {
   constexpr int CACHE = 16;                                   // float4 per lane kept in registers
   pdl_sync();
@@ -323,7 +323,7 @@ enum { EPI_F32 = 0, EPI_T = 1, EPI_GELU_T = 2, EPI_RESID = 3, EPI_ATOMIC = 4 }; 
 
 template <typename T, int EPI>
 __global__ void __launch_bounds__(256)
-gemm_simt_kernel(const T *__restrict__ A, const T *__restrict__ W, void *__restrict__ Cout,
+gemm_simt_kernel(const T *A, const T *__restrict__ W, void *Cout,
                  int M, int N, int K) {
   __shared__ float As[16][64 + 4];
   __shared__ float Ws[16][64 + 4];
@@ -539,7 +539,7 @@ __device__ __forceinline__ void split_bf16x2(float x, float y, uint32_t &hi, uin
 // rotating the earlier tiles' keys again.  grid = (heads, B, ceil(q_len / 16)), block = 128.
 template <typename T, int DH>
 __global__ void __launch_bounds__(128)
-kv_append_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
+kv_append_kernel(const float *qkv, T *__restrict__ Kc, T *__restrict__ Vc,
                  const float2 *__restrict__ rope, PassGeom g, int n_heads) {
   constexpr int HALF = DH / 2;
   const int h = blockIdx.x, slot = blockIdx.y, d = n_heads * DH;
@@ -600,7 +600,7 @@ __device__ __forceinline__ float attn_peer_f32(const float *local, uint32_t rank
 // the keys and values of this pass into the cache.
 template <typename T, int DH>
 __global__ void __launch_bounds__(128)
-attn_kernel(const float *__restrict__ qkv, T *__restrict__ Kc, T *__restrict__ Vc,
+attn_kernel(const float *qkv, T *Kc, T *Vc,
             const float2 *__restrict__ rope, PassGeom g, int n_heads, int QT, int nk_max, int skv, int pre,
             T *__restrict__ out) {
   constexpr bool BF = sizeof(T) == 2;
@@ -768,9 +768,9 @@ __device__ float head_normal(const DevState *st, int series, int k_pos, int e); 
 
 template <typename T>
 __global__ void __launch_bounds__(256)
-head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T *__restrict__ Wh, int d,
+head_kernel(const float *x, const float *__restrict__ gain, const T *__restrict__ Wh, int d,
             int P, float eps, PassGeom g, int only_last, float *__restrict__ hist,
-            float *__restrict__ vout, const DevState *__restrict__ st, float *__restrict__ muq, int k_pos, int K,
+            float *__restrict__ vout, const DevState *st, float *__restrict__ muq, int k_pos, int K,
             int tok_len) {
   extern __shared__ __align__(16) float xs[];
   __shared__ float red[32];
@@ -824,7 +824,7 @@ head_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T
 // grid = (ceil(M / 8), ceil(P / 32)), block = 256, dynamic shared memory 8 * d floats.
 template <typename T>
 __global__ void __launch_bounds__(256)
-head_rows_kernel(const float *__restrict__ x, const float *__restrict__ gain, const T *__restrict__ Wh, int M,
+head_rows_kernel(const float *x, const float *__restrict__ gain, const T *__restrict__ Wh, int M,
                  int d, int P, float eps, float *__restrict__ vout, PassGeom g) {
   constexpr int R = 8;
   extern __shared__ __align__(16) float xs[];                  // [R][d] normalised rows
