@@ -339,7 +339,8 @@ template <typename F> void prefer_max_smem(F *fn) {
 }
 template <typename T> void prefer_max_smem_typed() {
   prefer_max_smem(embed_kernel<T>);
-  prefer_max_smem(rmsnorm_kernel<T>);
+  prefer_max_smem(rmsnorm_kernel<T, false>);
+  prefer_max_smem(rmsnorm_kernel<T, true>);
   prefer_max_smem(head_kernel<T>);
   prefer_max_smem(embed_rows_kernel<T>);
   prefer_max_smem(head_rows_kernel<T>);
@@ -526,6 +527,8 @@ enum { HEAD_NONE = 0, HEAD_LAST_TO_HIST = 1, HEAD_ALL_TO_VOUT = 2 };
 // Passes of at least this many rows take the embedding and head kernels that share each weight
 // load between 8 rows; below it there are too few rows to fill the SMs that way.
 constexpr int kManyRows = 1024;
+// Up to this many rows the separate RMSNorm kernel fetches its constants before the dependency wait.
+constexpr int kNormEarlyMaxRows = 2048;
 
 // Draft step i of a round (k_pos = i - 1): lets the head kernel turn its mean into a sampled
 // proposal when the call asks for one (Sec. 3.3); target and prefill passes carry none.
@@ -534,7 +537,7 @@ struct DraftStep { int k_pos = -1, K = 0; };
 // One causal pass of a model over q_len new tokens per series (appends to its KV cache).
 template <typename T>
 void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout,
-              unsigned long long *stamp, DraftStep ds) {
+              unsigned long long *stamp, DraftStep ds, bool opens_round) {
   const int M = B * g.q_len, d = m.arch.d_model, f = m.arch.d_ff, P = h->cfg.patch_len, Pi = h->P_in;
   cudaStream_t s = h->ls;
   const float eps = h->cfg.rms_eps;
@@ -552,6 +555,8 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   const bool fold = sizeof(T) == 2 && h->use_tc && m.layers[0].tc_qkv.valid && M <= 512;
   const int L = m.arch.n_layers;
   const LiveRows lr{g.n_live, g.q_len};
+  // the RMSNorm of passes of a few thousand rows is a link in a chain: constants before the wait
+  auto *norm_kernel = M <= kNormEarlyMaxRows && d <= 1280 ? rmsnorm_kernel<T, true> : rmsnorm_kernel<T, false>;
   {
     KTimer kt(h, KC_EMBED, (double)M * Pi * 4 + (double)d * Pi * sizeof(T) + (double)M * d * 4, 2.0 * M * Pi * d);
     if (!fold && M >= kManyRows)
@@ -560,7 +565,7 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     else
       launch_ex(s, h->pdl, embed_kernel<T>, dim3(M, (d + 127) / 128), dim3(128), Pi * sizeof(float), h->hist, g, Pi, d,
                 (const T *)m.W_emb, h->x, stamp, fold ? m.layers[0].g1 : (const float *)nullptr,
-                fold ? (T *)h->a : (T *)nullptr, fold ? h->ssq : (float *)nullptr);
+                fold ? (T *)h->a : (T *)nullptr, fold ? h->ssq : (float *)nullptr, opens_round ? 1 : 0);
   }
   const double norm_bytes = (double)M * d * (4 + sizeof(T)) + d * 4.0;
   SkNorm consume{};                 // scale the result rows by rstd of the input rows
@@ -572,7 +577,7 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     LayerDev &ly = m.layers[l];
     if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g1, M, d, eps, (T *)h->a, lr);
+      launch_ex(s, h->pdl, norm_kernel, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g1, M, d, eps, (T *)h->a, lr);
     }
     gemm<T>(h, &ly.tc_qkv, h->a, ly.Wqkv, h->qkv, M, 3 * d, d, EPI_F32, fold ? &consume : nullptr, lr);
     if (m.dh == 32) launch_attn<T, 32>(h, m, l, B, g);
@@ -586,7 +591,7 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
     gemm<T>(h, &ly.tc_o, h->ao, ly.Wo, h->x, M, d, d, EPI_RESID, fold ? &produce : nullptr, lr);
     if (!fold) {
       KTimer kt(h, KC_RMSNORM, norm_bytes, 3.0 * M * d);
-      launch_ex(s, h->pdl, rmsnorm_kernel<T>, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g2, M, d, eps, (T *)h->a, lr);
+      launch_ex(s, h->pdl, norm_kernel, dim3((M + 7) / 8), dim3(256), 0, h->x, ly.g2, M, d, eps, (T *)h->a, lr);
     }
     gemm<T>(h, &ly.tc_1, h->a, ly.W1, h->hbuf, M, f, d, EPI_GELU_T, fold ? &consume : nullptr, lr);
     produce.gain = l + 1 < L ? m.layers[l + 1].g1 : nullptr;
@@ -615,11 +620,13 @@ void run_pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode
   }
 }
 
+// opens_round: the pass is the first of a round, i.e. its first kernel directly follows the kernel
+// that closed the previous one (and wrote the live list); it then looks its slots up after its wait.
 void pass(tsfm_spec *h, ModelDev &m, int B, const PassGeom &g, int head_mode, float *vout = nullptr,
-          unsigned long long *stamp = nullptr, DraftStep ds = DraftStep{}) {
+          unsigned long long *stamp = nullptr, DraftStep ds = DraftStep{}, bool opens_round = false) {
   if (g.q_len < 1) return;
-  if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout, stamp, ds);
-  else run_pass<float>(h, m, B, g, head_mode, vout, stamp, ds);
+  if (h->cfg.dtype == TSFM_BF16) run_pass<bf16>(h, m, B, g, head_mode, vout, stamp, ds, opens_round);
+  else run_pass<float>(h, m, B, g, head_mode, vout, stamp, ds, opens_round);
 }
 
 int check_call(tsfm_spec *h, const float *series, int B, int ctx_len, int H, float *out, int K) {
@@ -691,7 +698,7 @@ void enqueue_round(tsfm_spec *h, int B, int N, int T, int K, cudaGraphConditiona
   // step 1 re-ingests the last two committed patches (the draft cache may lack the last
   // accepted proposal), steps 2..K ingest the previous proposal; a patch is tpp tokens
   pass(h, h->drf, B, PassGeom{h->done, N - 2 * tpp, 2 * tpp, h->cap, live, n_live, tpp, tpp}, HEAD_LAST_TO_HIST, nullptr,
-       &h->st->t_phase[0], DraftStep{0, K});
+       &h->st->t_phase[0], DraftStep{0, K}, true);
   for (int i = 2; i <= K; ++i)
     pass(h, h->drf, B, PassGeom{h->done, N - tpp + (i - 1) * tpp, tpp, h->cap, live, n_live, tpp, tpp}, HEAD_LAST_TO_HIST,
          nullptr, nullptr, DraftStep{i - 1, K});

@@ -171,6 +171,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = *slot_ptr;
 
+  float g_direct = 0.f;
+  float4 g_vec = make_float4(0.f, 0.f, 0.f, 0.f);
   if (warp == 4 && lane == 0) {
     // ---------------- TMA producer.  The weights do not depend on the preceding kernel: the
     // first ring-full of weight tiles is requested before waiting for it, the activation tiles
@@ -195,6 +197,12 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
       tma_load_2d(dst + w_bytes, &mapA, (kb_lo + kb) * TC_BK, t0, full0 + 8 * s);
     }
   } else {
+    if (NORM && nm.a_out && warp < 4) {
+      // gains of the features this thread finishes in either epilogue: constants, fetched before the wait
+      const int fd = f0 + threadIdx.x, fv = f0 + (threadIdx.x & 31) * 4;
+      if (fd < N) g_direct = nm.gain[fd];
+      if (N % 4 == 0 && fv + 3 < N) g_vec = *reinterpret_cast<const float4 *>(nm.gain + fv);
+    }
     pdl_sync();
     if (warp < 4) {
       if (NORM && nm.ssq_in) {                                // overlaps the main loop
@@ -268,7 +276,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
               if (NORM && epi == EPI_RESID && nm.a_out) {
                 const float xn = ((float *)C)[o] + v[j];
                 ((float *)C)[o] = xn;
-                nm.a_out[o] = __float2bfloat16_rn(nm.gain[f] * xn);
+                nm.a_out[o] = __float2bfloat16_rn(g_direct * xn);
                 v[j] = xn * xn;
               } else {
                 sk_store_rt(C, o, v[j], epi);
@@ -370,7 +378,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_constant__
             old.x += sum.x; old.y += sum.y; old.z += sum.z; old.w += sum.w;
             *reinterpret_cast<float4 *>((float *)C + o) = old;
             if (NORM && nm.a_out) {
-              const float4 gg = *reinterpret_cast<const float4 *>(nm.gain + f);
+              const float4 gg = g_vec;
               const __nv_bfloat162 lo = __floats2bfloat162_rn(gg.x * old.x, gg.y * old.y), hi = __floats2bfloat162_rn(gg.z * old.z, gg.w * old.w);
               uint2 pk;
               pk.x = *reinterpret_cast<const uint32_t *>(&lo);

@@ -64,6 +64,9 @@ gemm_ws_kernel(const bf16 *A, const bf16 *__restrict__ W, void *C, int M, int N,
     else *reinterpret_cast<uint4 *>(Ws + (dst - Ws32)) = make_uint4(0u, 0u, 0u, 0u);
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
+  // the gains of this thread's two output features (folded norm): constants, fetched before the wait
+  float2 gg = make_float2(0.f, 0.f);
+  if (NORM && nm.a_out && f0 + (tid & 7) * 2 < N) gg = *reinterpret_cast<const float2 *>(nm.gain + f0 + (tid & 7) * 2);
   pdl_sync();
   // ---- activation tile (rows past M are zero)
   for (int i = tid; i < WS_MT * cpr; i += 256) {
@@ -138,10 +141,7 @@ gemm_ws_kernel(const bf16 *A, const bf16 *__restrict__ W, void *C, int M, int N,
     if (live) *reinterpret_cast<float2 *>((float *)C + o) = v;
     if (NORM && nm.a_out) {
       // the next contraction's operand bf16(gain * x) and the row's sum of squares over these 16 features
-      if (live) {
-        const float2 gg = *reinterpret_cast<const float2 *>(nm.gain + f);
-        *reinterpret_cast<uint32_t *>(nm.a_out + o) = pack_bf16x2(gg.x * v.x, gg.y * v.y);
-      }
+      if (live) *reinterpret_cast<uint32_t *>(nm.a_out + o) = pack_bf16x2(gg.x * v.x, gg.y * v.y);
       float sq = live ? v.x * v.x + v.y * v.y : 0.f;
       sq += __shfl_xor_sync(0xffffffffu, sq, 1);
       sq += __shfl_xor_sync(0xffffffffu, sq, 2);

@@ -135,17 +135,20 @@ __global__ void guard_check_kernel(const GuardRegion *__restrict__ regions, int 
 
 // 16-byte vector loads of T (8 bf16 or 4 fp32) unpacked to floats.
 template <typename T> struct Vec16;
+// (raw() / unpack() split the load from its use: kernels fetch constants of the model before their
+// dependency wait and unpack them after it.)
 template <> struct Vec16<float> {
   static constexpr int N = 4;
-  static __device__ __forceinline__ void load(const float *p, float *v) {
-    const float4 t = *reinterpret_cast<const float4 *>(p);
-    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-  }
+  using Raw = float4;
+  static __device__ __forceinline__ Raw raw(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+  static __device__ __forceinline__ void unpack(const Raw &t, float *v) { v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+  static __device__ __forceinline__ void load(const float *p, float *v) { unpack(raw(p), v); }
 };
 template <> struct Vec16<bf16> {
   static constexpr int N = 8;
-  static __device__ __forceinline__ void load(const bf16 *p, float *v) {
-    const uint4 t = *reinterpret_cast<const uint4 *>(p);
+  using Raw = uint4;
+  static __device__ __forceinline__ Raw raw(const bf16 *p) { return *reinterpret_cast<const uint4 *>(p); }
+  static __device__ __forceinline__ void unpack(const Raw &t, float *v) {
     const uint32_t w[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -153,6 +156,7 @@ template <> struct Vec16<bf16> {
       v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
     }
   }
+  static __device__ __forceinline__ void load(const bf16 *p, float *v) { unpack(raw(p), v); }
 };
 
 // ----------------------------------------------------------------------------------
@@ -165,25 +169,45 @@ template <typename T>
 __global__ void __launch_bounds__(128)
 embed_kernel(const float *hist, PassGeom g, int P, int d, const T *__restrict__ W,
              float *__restrict__ x, unsigned long long *__restrict__ stamp,
-             const float *__restrict__ gain, T *__restrict__ a_out, float *__restrict__ ssq_out) {
+             const float *__restrict__ gain, T *__restrict__ a_out, float *__restrict__ ssq_out, int opens_round) {
   extern __shared__ float zs[];
-  pdl_sync();
+  constexpr int V = Vec16<T>::N, PRE = 12;                     // weight vectors fetched before the wait
   const int row = blockIdx.x, slot = row / g.q_len, j = row % g.q_len;
+  const int f = blockIdx.y * 128 + threadIdx.x;
+  // Before the dependency wait: what does not depend on the preceding kernel -- the start of this
+  // thread's weight row, its gain, and (unless this pass opens a round, when the kernel that closed
+  // the previous round is the predecessor itself) the slot lookup.
+  const T *wr = W + (size_t)min(f, d - 1) * P;
+  typename Vec16<T>::Raw wpre[PRE];
+  if (P % V == 0) {
+#pragma unroll
+    for (int k = 0; k < PRE; ++k)
+      if (k * V < P) wpre[k] = Vec16<T>::raw(wr + k * V);
+  }
+  const float gf = a_out ? gain[min(f, d - 1)] : 0.f;
+  SlotPos sp;
+  if (!opens_round) sp = slot_lookup(g, slot);
+  pdl_sync();
   if (stamp && row == 0 && blockIdx.y == 0 && threadIdx.x == 0) *stamp = globaltimer_ns();
-  const SlotPos sp = slot_lookup(g, slot);                      // (after the wait: this kernel may open a round)
+  if (opens_round) sp = slot_lookup(g, slot);
   if (sp.dead) return;
   const int b = sp.b;
   const float *z = hist + ((size_t)b * g.cap + sp.p0 + j) * P;
   for (int i = threadIdx.x; i < P; i += blockDim.x) zs[i] = z[i];
   __syncthreads();
-  const int f = blockIdx.y * 128 + threadIdx.x;
   if (f >= d) return;
-  const T *wr = W + (size_t)f * P;
-  constexpr int V = Vec16<T>::N;
   float acc = 0.f;
   if (P % V == 0) {
+#pragma unroll
+    for (int k = 0; k < PRE; ++k)
+      if (k * V < P) {
+        float w[V];
+        Vec16<T>::unpack(wpre[k], w);
+#pragma unroll
+        for (int c = 0; c < V; ++c) acc = fmaf(w[c], zs[k * V + c], acc);
+      }
 #pragma unroll 4
-    for (int i = 0; i < P; i += V) {
+    for (int i = PRE * V; i < P; i += V) {
       float w[V];
       Vec16<T>::load(wr + i, w);
 #pragma unroll
@@ -194,7 +218,7 @@ embed_kernel(const float *hist, PassGeom g, int P, int d, const T *__restrict__ 
   }
   x[(size_t)row * d + f] = acc;
   if (a_out) {            // operand of the first contraction, normalised later (see SkNorm); d % 64 == 0
-    a_out[(size_t)row * d + f] = from_f32<T>(gain[f] * acc);
+    a_out[(size_t)row * d + f] = from_f32<T>(gf * acc);
     float sq = acc * acc;                                       // sums of squares over slices of 16 features
     sq += __shfl_xor_sync(0xffffffffu, sq, 1);
     sq += __shfl_xor_sync(0xffffffffu, sq, 2);
@@ -272,18 +296,31 @@ __device__ __forceinline__ void store4(bf16 *o, float a, float b, float c, float
   *reinterpret_cast<uint2 *>(o) = pk;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(256)
+// EARLY (passes of up to a few thousand rows, where the launch is a link in a chain and not a
+// stream of bytes): the gain and the live-row count are fetched before the dependency wait, which
+// takes two L2 round trips out of the chain at the price of registers (rows of at most 1280
+// features, so that two CTAs still fit on an SM).  The count was written by the kernel that closed
+// the previous round, at least two kernels back.
+template <typename T, bool EARLY>
+__global__ void __launch_bounds__(256, 2)
 rmsnorm_kernel(const float *x, const float *__restrict__ gain, int M, int d, float eps,
                T *__restrict__ a, LiveRows lr) {
-  constexpr int CACHE = 16;                                   // float4 per lane kept in registers
-  pdl_sync();
+  constexpr int CACHE = EARLY ? 10 : 16;                      // float4 per lane kept in registers
   const int lane = threadIdx.x & 31;
   const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (row >= (size_t)live_rows(lr, M)) return;
-  const float4 *xr = reinterpret_cast<const float4 *>(x + row * d);
   const float4 *gr = reinterpret_cast<const float4 *>(gain);
   const int nv = d / 4;
+  float4 gpre[EARLY ? CACHE : 1];
+  if (EARLY) {
+    if (lr.n_live) M = min(M, *reinterpret_cast<const volatile int *>(lr.n_live) * lr.q_len);
+    if (row >= (size_t)M) return;
+#pragma unroll
+    for (int k = 0; k < CACHE; ++k)
+      if (lane + 32 * k < nv) gpre[EARLY ? k : 0] = gr[lane + 32 * k];
+  }
+  pdl_sync();
+  if (!EARLY && row >= (size_t)live_rows(lr, M)) return;
+  const float4 *xr = reinterpret_cast<const float4 *>(x + row * d);
   float4 v[CACHE];
   float ss = 0.f;
 #pragma unroll
@@ -304,7 +341,7 @@ rmsnorm_kernel(const float *x, const float *__restrict__ gain, int M, int d, flo
   for (int k = 0; k < CACHE; ++k) {
     const int i = lane + 32 * k;
     if (i < nv) {
-      const float4 gg = gr[i];
+      const float4 gg = EARLY ? gpre[EARLY ? k : 0] : gr[i];
       store4(ar + 4 * i, gg.x * v[k].x * rstd, gg.y * v[k].y * rstd, gg.z * v[k].z * rstd, gg.w * v[k].w * rstd);
     }
   }
@@ -774,11 +811,25 @@ head_kernel(const float *x, const float *__restrict__ gain, const T *__restrict_
             int tok_len) {
   extern __shared__ __align__(16) float xs[];
   __shared__ float red[32];
+  constexpr int V = Vec16<T>::N, WPRE = 6, GPRE = 6;   // weight vectors per lane / gains per thread fetched early
   const int nb = g.q_len / g.head_step;                // boundaries per series
   int slot, j, ib = 0;
   if (only_last) { slot = blockIdx.x; j = g.q_len - 1; }
   else { slot = blockIdx.x / nb; ib = blockIdx.x % nb; j = (ib + 1) * g.head_step - 1; }
   const SlotPos sp = slot_lookup(g, slot);             // before the dependency wait: see SlotPos
+  // also before the wait: the constants this thread needs -- the start of its warp's weight row and
+  // its gains (two L2 round trips that would otherwise follow the normalisation one after the other)
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int p = blockIdx.y * 8 + w;
+  const T *wr = Wh + (size_t)min(p, P - 1) * d;
+  typename Vec16<T>::Raw wpre[WPRE];
+  float gpre[GPRE];
+#pragma unroll
+  for (int k = 0; k < WPRE; ++k)
+    if ((lane + 32 * k) * V < d) wpre[k] = Vec16<T>::raw(wr + (lane + 32 * k) * V);
+#pragma unroll
+  for (int k = 0; k < GPRE; ++k)
+    if ((int)threadIdx.x + 256 * k < d) gpre[k] = gain[threadIdx.x + 256 * k];
   pdl_sync();
   if (sp.dead) return;
   const int b = sp.b;
@@ -790,17 +841,26 @@ head_kernel(const float *x, const float *__restrict__ gain, const T *__restrict_
     ss = fmaf(v, v, ss);
   }
   const float rstd = rsqrtf(block_sum(ss, red) / d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x) xs[i] = gain[i] * xs[i] * rstd;
+#pragma unroll
+  for (int k = 0; k < GPRE; ++k)
+    if ((int)threadIdx.x + 256 * k < d) xs[threadIdx.x + 256 * k] = gpre[k] * xs[threadIdx.x + 256 * k] * rstd;
+  for (int i = threadIdx.x + 256 * GPRE; i < d; i += blockDim.x) xs[i] = gain[i] * xs[i] * rstd;
   __syncthreads();
   float *dst = only_last ? hist + ((size_t)b * g.cap + sp.p0 + g.q_len) * tok_len
                          : vout + ((size_t)b * nb + ib) * P;
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int p = blockIdx.y * 8 + w;
   if (p >= P) return;
-  const T *wr = Wh + (size_t)p * d;
-  constexpr int V = Vec16<T>::N;
   float acc = 0.f;
-  for (int i = lane * V; i < d; i += 32 * V) {
+#pragma unroll
+  for (int k = 0; k < WPRE; ++k) {
+    const int i = (lane + 32 * k) * V;
+    if (i < d) {
+      float wv[V];
+      Vec16<T>::unpack(wpre[k], wv);
+#pragma unroll
+      for (int c = 0; c < V; ++c) acc = fmaf(wv[c], xs[i + c], acc);
+    }
+  }
+  for (int i = (lane + 32 * WPRE) * V; i < d; i += 32 * V) {
     float wv[V];
     Vec16<T>::load(wr + i, wv);
 #pragma unroll
@@ -828,12 +888,14 @@ head_rows_kernel(const float *x, const float *__restrict__ gain, const T *__rest
                  int d, int P, float eps, float *__restrict__ vout, PassGeom g) {
   constexpr int R = 8;
   extern __shared__ __align__(16) float xs[];                  // [R][d] normalised rows
-  pdl_sync();
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int row0 = blockIdx.x * R;
   const int nb = g.q_len / g.head_step;                        // boundaries per series
-  M = live_rows(LiveRows{g.n_live, nb}, M);
+  // live rows: read before the dependency wait (written when the previous round closed, a whole
+  // pass of kernels back)
+  if (g.n_live) M = min(M, *reinterpret_cast<const volatile int *>(g.n_live) * nb);
   if (row0 >= M) return;
+  pdl_sync();
   {
     const int row = row0 + w;
     float *xw = xs + (size_t)w * d;

@@ -332,6 +332,14 @@ def test_many_series_short_rows_one_warp_per_series_and_head_bf16():
     run_and_compare(wl, 3, 1.0, 9, [0, 100, 198])
 
 
+@pytest.mark.parametrize("B", [257, 340])
+def test_many_series_long_rows_one_warp_per_series_and_head_bf16(B):
+    """C4's row lengths with more than a thousand (series, head) pairs on small models: one warp per
+    pair streams the whole row through its ring (257 x 4 and 340 x 4 pairs, four per CTA)."""
+    wl = workload("C4", batch=B, horizon=32 * 5 + 3, target=Arch(2, 256, 4, 512), draft=Arch(1, 128, 2, 256))
+    run_and_compare(wl, 4, 2.0, 5, [0, B // 2, B - 1])
+
+
 @pytest.mark.parametrize("name,ids", [("C0", [0]), ("C1", [0, 7, 31]), ("C2", [3, 200])])
 def test_draft_only_forecast_matches_oracle(name, ids):
     """Third arm of the matched three-way protocol: the draft model decoding on its own (Eq. 1)."""
