@@ -15,7 +15,9 @@ times, max over ranks.
 
 On one GPU the line also carries, under `workloads`, the same measurement (fewer steps) of
 C2 (tensor-bound verification), C1 at its three temperatures, C1 with a draft that tracks its
-target (acceptance ~0.97, the regime the paper reports) and four cells of C3's K x eps grid, each with target-only and draft-only decoding, phase times, and the speedup
+target (acceptance ~0.97, the regime the paper reports), four cells of C3's K x eps grid and the
+point-token shape C5 (one step per input token, a 64-step head), each with target-only and draft-only
+decoding, phase times, and the speedup
 Eq. 8 predicts from the measured acceptance rate and cost ratios beside the measured one.
 
 `--impl reference` times the CPU oracle (fp64, as it stands) on a bounded sample of the same
@@ -70,7 +72,7 @@ def parse_args():
     ap.add_argument("--K", type=int, default=None)
     ap.add_argument("--cpu-series", type=int, default=None, help="series per oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--others", default="C2,C1,C3", help="comma list of further workloads measured on one GPU ('' = none)")
+    ap.add_argument("--others", default="C2,C1,C3,C5", help="comma list of further workloads measured on one GPU ('' = none)")
     return ap.parse_args()
 
 
@@ -433,7 +435,7 @@ def roofline_of(m, peaks):
 
 
 def other_workloads(names):
-    """(label, workload, K, tau) of the further entries: C2, C1 at its temperatures, cells of C3's grid."""
+    """(label, workload, K, tau) of the further entries: C2, C1 at its temperatures, cells of C3's grid, C5."""
     from tsfm_inputs import workload
     out = []
     for n in names:
