@@ -59,11 +59,12 @@ struct SkShape {
 };
 // Ring of `stages` x (W tile 16 KB + A tile BN x 128 B); the partial-sum tile (BN x 128 fp32)
 // reuses the ring once the accumulator is complete.
-static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1) {
+// (stages_hint > 0: the ring depth the tile rule asks for instead of the default.)
+static inline SkShape sk_shape(int BN, int kb_per_cta, bool split, int wt = 1, int stages_hint = 0) {
   SkShape s;
   s.BN = BN;
   const int stage = TC_W_BYTES * wt + BN * TC_BK * 2;
-  int stages = wt == 2 ? 3 : BN > 160 ? 4 : BN > 64 ? 3 : 4;
+  int stages = stages_hint > 0 ? stages_hint : wt == 2 ? 3 : BN > 160 ? 4 : BN > 64 ? 3 : 4;
   if (stages > kb_per_cta) stages = kb_per_cta < 1 ? 1 : kb_per_cta;
   int bytes = stages * stage;
   if (split && bytes < BN * TC_BM * 4) bytes = BN * TC_BM * 4;
@@ -477,8 +478,10 @@ static int gemm_sk_plan(GemmSkPlan *plan, const void *W, int N, int K, const voi
 // Tile and split choice for M tokens: one token tile up to 256 rows (rounded up to 16), and
 // as many K splits (a power of two, at most 8, at most the number of K blocks) as it takes to
 // put the grid on most of the 148 SMs.
-static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
+// epi: the epilogue (EPI_*); *STG: ring depth, 0 = the default for the tile.
+static void gemm_sk_geometry(int N, int K, int M, int epi, int *BN, int *S, int *WT, int *STG) {
   *WT = 1;
+  *STG = 0;
   // Measured on B200 (graph replay, dependent launches): up to a few hundred tokens a 32-token
   // tile with K split until the grid has ~150-250 CTAs is fastest (the partial-tile exchange
   // grows with the tile, the latency chain does not shrink); large M takes 128/256-token tiles.
@@ -490,7 +493,28 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
     // token tiles shared in shared memory) still covers most SMs.
     const int ctas_b = ((FT + 1) / 2) * ((M + 255) / 256);
     *S = 1;
-    if (KB >= 32 && ctas_b >= 100) { *BN = 256; *WT = 2; } else { *BN = 128; }
+    if (KB >= 32 && ctas_b >= 100) {
+      // one 256-feature CTA per SM: of 256- and 192-token tiles the one with fewer waves x tile
+      // (C4's prefill W2, M = 16320, N = 1280: 320 CTAs of 256 tokens are 2.2 waves, 183 us;
+      // 425 of 192 are 2.9, 162 us)
+      const int w256 = (ctas_b + 147) / 148, w192 = (((FT + 1) / 2) * ((M + 191) / 192) + 147) / 148;
+      *BN = w192 * 192 < w256 * 256 ? 192 : 256;
+      *WT = 2;
+    } else if (KB >= 32) {
+      *BN = 128;
+    } else if (epi == EPI_T || epi == EPI_GELU_T) {
+      // bf16 outputs (the GELU epilogue is the longest): a two-stage ring lets a third CTA onto the
+      // SM, so that two main loops run under every epilogue (M = 16320, N = 5120, K = 1280: 295 ->
+      // 247 us; M = 7424, N = 4096, K = 1024: 106 -> 93 us)
+      *BN = 128;
+      *STG = 2;
+    } else if (epi == EPI_F32 || FT * ((M + 159) / 160) >= 3 * 296) {
+      // fp32 outputs, and residual updates of at least three waves: 160-token tiles (less shared-
+      // memory fill per flop; M = 16320, N = 3840: 165 -> 152 us, M = 5120, N = 2304: 25.2 -> 20.6 us)
+      *BN = 160;
+    } else {
+      *BN = 128;
+    }
     return;
   }
   if (M > 512 && KB < 32) {
@@ -504,8 +528,16 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
     int best = 96, best_cost = 1 << 30;
     for (int bnc = 64; bnc <= 160; bnc += 16) {
       const int ctas = FT * ((M + bnc - 1) / bnc);
-      const int cost = ((ctas + 295) / 296) * (bnc + 48);
+      const int cost = ((ctas + 295) / 296) * (bnc + 48) * 10;
       if (cost < best_cost) { best = bnc; best_cost = cost; }
+    }
+    // With a two-stage ring a third CTA fits on the SM (444 on the device); such a CTA is about
+    // 30 % slower, which pays where it saves a whole wave (M = 2048, N = 3072 GELU: 384 CTAs of 128
+    // tokens, 23.7 -> 17.2 us; M = 3072, N = 2304: 432 CTAs, 16.9 -> 13.4 us).
+    for (int bnc = 80; bnc <= 128; bnc += 16) {
+      const int ctas = FT * ((M + bnc - 1) / bnc);
+      const int cost = ((ctas + 443) / 444) * (bnc + 48) * 13;
+      if (cost < best_cost) { best = bnc; best_cost = cost; *STG = 2; }
     }
     *BN = best;
     *S = 1;
@@ -535,8 +567,8 @@ static void gemm_sk_geometry(int N, int K, int M, int *BN, int *S, int *WT) {
 static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, int M, int epi, int *status,
                            const SkNorm *norm = nullptr, LiveRows lr = LiveRows{nullptr, 0}) {
   if (!p.valid || M < 1 || M > p.M_max) return false;
-  int BN, S, wt;
-  gemm_sk_geometry(p.N, p.K, M, &BN, &S, &wt);
+  int BN, S, wt, stg;
+  gemm_sk_geometry(p.N, p.K, M, epi, &BN, &S, &wt, &stg);
   const int idx = BN / 16 - 1;
   if (!p.haveA[idx]) {
     if (tc_encode(&p.mapA[idx], p.A, p.M_max, p.K, BN)) return false;
@@ -566,7 +598,7 @@ static bool gemm_sk_launch(cudaStream_t st, bool pdl, GemmSkPlan &p, void *C, in
     }
     mapC = &hit->map;
   }
-  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1 || tma_c, wt);
+  const SkShape sh = sk_shape(BN, (KB + S - 1) / S, S > 1 || tma_c, wt, stg);
   if (sh.smem_bytes > 227 * 1024) return false;
   const int ring_bytes = sh.smem_bytes - 1024 - 256 - 1024;
   const SkNorm nm = norm ? *norm : SkNorm{};
